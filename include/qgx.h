@@ -1,0 +1,227 @@
+/*
+ * qgx -- the data-parallel hot path of Q-GenX (quantized generalized extra-gradient,
+ * arXiv 2308.09187) for one NVIDIA B200 (sm_100a), as a C library.
+ *
+ * The paper's K processors are K slices of one GPU's memory: a "[K][d]" array holds worker
+ * k's vector at offset k*d.  A vector is cut into buckets of `bucket` coordinates (the last
+ * one may be shorter; nb = ceil(d / bucket)); Definition 1 is applied to every bucket on its
+ * own, with the bucket's own norm.
+ *
+ * Conventions for every entry point unless its comment says otherwise:
+ *  - pointers marked [dev] are device pointers, owned by the caller, and must stay valid until
+ *    the context's stream has run the call; pointers marked [host] are read (or written) before
+ *    the call returns;
+ *  - calls are asynchronous on the stream given to qgx_create and return a qgx_status for what
+ *    the host could check; errors found on the device (non-finite norm, capacity, corrupt
+ *    stream, a bounded wait that ran out) are latched in the context and reported by
+ *    qgx_sync_status, which synchronizes the stream.  No call aborts, traps or prints;
+ *  - the library allocates device memory only inside qgx_create and when a call needs a larger
+ *    workspace than any call before it (the fused calls and qgx_update_levels).
+ *
+ * Symbol byte: bits 0..4 level index, bit 7 sign (set only when the level index is nonzero).
+ * Stream: 32-bit words, bit p of a stream is bit (p & 31) of word (p >> 5).
+ */
+#ifndef QGX_H_
+#define QGX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  QGX_OK = 0,
+  QGX_ERR_INVALID_ARG = 1,
+  QGX_ERR_BAD_LEVELS = 2,   /* nlev outside [2,32], endpoints not 0 and 1, or not strictly increasing */
+  QGX_ERR_CAPACITY = 3,     /* a worker's stream does not fit cap_words */
+  QGX_ERR_CORRUPT = 4,      /* a stream that no encoder could have produced */
+  QGX_ERR_NONFINITE = 5,    /* a bucket norm is NaN or infinite */
+  QGX_ERR_TIMEOUT = 6,      /* a bounded device-side wait ran out */
+  QGX_ERR_CUDA = 7          /* the CUDA runtime reported an error */
+} qgx_status;
+
+enum { QGX_NORM_L2 = 0, QGX_NORM_LINF = 1 };
+enum { QGX_CODE_FIXED = 0, QGX_CODE_HUFFMAN = 1 };
+enum { QGX_OP_DENSE_AFFINE = 0, QGX_OP_BILINEAR = 1, QGX_OP_DIAGONAL = 2 };
+enum { QGX_REFIT_NONE = 0, QGX_REFIT_CONTINUE = 1, QGX_REFIT_FIRST = 2 };
+/* flag of qgx_quantize: `norms` is an input (the caller's norms are used as they are) */
+enum { QGX_NORMS_SUPPLIED = 1 };
+
+enum { QGX_MAX_LEVELS = 32, QGX_MAX_CODE_LEN = 12, QGX_MAX_BUCKET = 16384 };
+
+typedef struct qgx_ctx qgx_ctx;
+
+/* Prefix code Psi of App. J over the level indices.  code[j] holds the codeword of level j as an
+ * integer of len[j] bits whose most significant bit is sent first.  subblock = number of
+ * coordinates per sub-block of a bucket (a multiple of 4); <= 0 or >= bucket means none. */
+typedef struct {
+  int32_t nlev;
+  int32_t maxlen;
+  int32_t subblock;
+  uint8_t len[32];
+  uint32_t code[32];
+} qgx_codebook;
+
+/* Quantizer configuration (Definition 1 + Sec. 3.2).  levels[0] = 0 < ... < levels[nlev-1] = 1.
+ * In the paper's counting "s levels" means nlev = s + 2. */
+typedef struct {
+  int32_t nlev;
+  int32_t bucket;           /* multiple of 4, <= QGX_MAX_BUCKET */
+  int32_t norm_type;        /* QGX_NORM_L2 | QGX_NORM_LINF */
+  int32_t code_type;        /* what a refit rebuilds: QGX_CODE_FIXED | QGX_CODE_HUFFMAN */
+  int32_t nbins;            /* histogram bins of the level refit (Sec. 3.3) */
+  int32_t pad;
+  uint64_t seed;            /* key of the counter-based generator */
+  float levels[32];
+  qgx_codebook cb;
+} qgx_quant_cfg;
+
+/* Monotone operator A of the VI (Sec. 2).  DENSE_AFFINE: A(x) = M x + b, M row-major d x d.
+ * BILINEAR: the game min_x max_y x^T A y with z = (x, y), A n x n row-major, d = 2n,
+ * A(z) = (A y, -A^T x).  DIAGONAL: A(x) = D .* x.  mat and bias are [dev]. */
+typedef struct {
+  int32_t kind;
+  int32_t pad;
+  uint64_t d;
+  const float *mat;
+  const float *bias;        /* DENSE_AFFINE only; may be NULL */
+} qgx_operator;
+
+/* State of Algorithm 1.  The vectors are [dev] float[d], caller-owned.  scalars is [dev]
+ * double[2] = { sum of squared differences, gamma_t }; t (host) counts iterations from 1. */
+typedef struct {
+  uint64_t d;
+  int32_t K;
+  int32_t t;
+  float *X;                 /* X_t */
+  float *Y;                 /* Y_t */
+  float *Xbar;              /* (1/t) sum of X_{i+1/2}: the ergodic average of Theorems 3 and 4 */
+  float *Xhalf;             /* X_{t+1/2} of the last step */
+  const float *anchor;      /* X_1; the update is X_{t+1} = anchor + gamma_{t+1} Y_{t+1} */
+  double *scalars;
+} qgx_eg_state;
+
+/* ---- context ------------------------------------------------------------------------------ */
+
+/* Creates a context on `device` whose calls run on `cuda_stream` (a cudaStream_t; NULL = the
+ * default stream).  Allocates a small status block.  Returns QGX_ERR_CUDA if there is no usable
+ * device: there is no CPU fallback. */
+qgx_status qgx_create(qgx_ctx **ctx, int device, void *cuda_stream);
+void qgx_destroy(qgx_ctx *ctx);
+/* Synchronizes the stream and returns the first error latched by a device-side check since the
+ * last call of this function (QGX_OK if none), clearing it. */
+qgx_status qgx_sync_status(qgx_ctx *ctx);
+const char *qgx_status_str(qgx_status s);
+/* How many kernels of this library the context has launched so far. */
+uint64_t qgx_launch_count(const qgx_ctx *ctx);
+
+/* ---- host helpers ------------------------------------------------------------------------- */
+
+/* QGX_OK iff the table is admissible for Definition 1. */
+qgx_status qgx_check_levels(const float *levels /*[host]*/, int nlev);
+/* Worst-case 32-bit words of one worker's stream: per bucket 32 (norm, C_b of App. E) +
+ * 16 per sub-block + (maxlen + 1) per coordinate bits, rounded up to whole words. */
+size_t qgx_stream_capacity_words(size_t d, int bucket, int subblock, int maxlen);
+/* Fixed-length code: every level index costs ceil(log2 nlev) bits. */
+qgx_status qgx_build_codebook_fixed(int nlev, int subblock, qgx_codebook *cb /*[host] out*/);
+/* Huffman code (App. J) for symbol weights p[nlev] [host]; canonical codewords ordered by
+ * (length, index); if the longest codeword would exceed QGX_MAX_CODE_LEN the weights are
+ * flattened by adding 2^(m-16), m = 0, 1, ..., until it fits. */
+qgx_status qgx_build_codebook_huffman(const double *p, int nlev, int subblock, qgx_codebook *cb);
+/* Level fit of Sec. 3.3 on a histogram hist[nbins] [host] of normalized magnitudes, read as a
+ * piecewise-uniform density: coordinate descent on the (QAda) objective, each interior level
+ * moved to the root of the objective's derivative with its neighbours fixed; at most 32 sweeps.
+ * first_fit != 0 starts from the mass quantiles, otherwise from levels[] as passed in.
+ * levels [host] in/out. */
+qgx_status qgx_fit_levels(const double *hist, int nbins, float *levels, int nlev, int first_fit);
+/* Symbol weights p[nlev] [host] out of the proposition on the code pmf (App. E). */
+qgx_status qgx_symbol_pmf(const double *hist, int nbins, const float *levels, int nlev, double *p);
+
+/* ---- the four steps of one exchange (Algorithm 1: quantize, encode | decode, aggregate) ---- */
+
+/* Definition 1 per bucket.  v [dev] float[K][d] -> norms [dev] float[K][nb] (L2: square root
+ * of the fp64 sum of squares, rounded once to fp32; with QGX_NORMS_SUPPLIED in flags norms is
+ * read instead) and sym [dev] uint8[K][d].  Coordinate i of worker k in exchange `exchange_id`
+ * rounds up iff (w >> 8) * 2^-24 < xi, w = word (i & 3) of Philox4x32-10 with key = seed and
+ * counter = (i >> 2 low, i >> 2 high, k, exchange_id).  levels is [host].
+ * Device-side error: QGX_ERR_NONFINITE (that bucket's symbols are all zero). */
+qgx_status qgx_quantize(qgx_ctx *ctx, const float *v, int K, size_t d, int bucket,
+                        const float *levels, int nlev, int norm_type, uint64_t seed,
+                        uint32_t exchange_id, int flags, float *norms, uint8_t *sym);
+
+/* CODE o Q of Sec. 3.2 / App. J.  Worker k's stream is stream[k*cap_words ...] [dev]; bucket b
+ * starts on a word boundary, after the buckets before it, and holds: the 32 bits of the norm;
+ * if sub-blocks are on, one 16-bit length (bits) per sub-block; then per coordinate its
+ * codeword, first code bit first, and one sign bit iff the level index is nonzero.
+ * bucket_bits [dev] uint32[K][nb] receives each bucket's length in bits, total_bits [dev]
+ * uint64[K] their sum.  Words the buckets do not use up to each worker's end are left untouched.
+ * Device-side errors: QGX_ERR_CAPACITY (nothing is written for that worker), QGX_ERR_CORRUPT
+ * for a level index >= nlev in sym. */
+qgx_status qgx_encode(qgx_ctx *ctx, const float *norms, const uint8_t *sym, int K, size_t d,
+                      int bucket, const qgx_codebook *cb /*[host]*/, uint32_t *stream,
+                      size_t cap_words, uint32_t *bucket_bits, uint64_t *total_bits);
+
+/* DEQ o CODE: the exact inverse of qgx_encode, driven by bucket_bits.  Every read is bounded by
+ * the bucket's length; a codeword that runs past it, an unassigned bit pattern, a sub-block whose
+ * length disagrees with its header, or lengths that exceed cap_words latch QGX_ERR_CORRUPT. */
+qgx_status qgx_decode(qgx_ctx *ctx, const uint32_t *stream, size_t cap_words,
+                      const uint32_t *bucket_bits, int K, size_t d, int bucket,
+                      const qgx_codebook *cb /*[host]*/, float *norms, uint8_t *sym);
+
+/* Aggregation of Algorithm 1: out[i] = (1/K) sum_k norm_{k,b(i)} * s * l_idx, the fp32 sum taken
+ * in the order k = 0..K-1 and divided once by K.  out [dev] float[d]. */
+qgx_status qgx_average(qgx_ctx *ctx, const float *norms, const uint8_t *sym, int K, size_t d,
+                       int bucket, const float *levels /*[host]*/, int nlev, float *out);
+
+/* ---- fused exchange ------------------------------------------------------------------------ */
+
+/* quantize -> encode -> decode -> average in two kernels, same streams and same mean as the four
+ * calls above in sequence.  v [dev] float[K][d]; mean_out [dev] float[d]; total_bits [dev]
+ * uint64[K] (may be NULL).  The streams live in the context's workspace (slot 0 or 1, so that
+ * the two exchanges of one iteration can both be kept). */
+qgx_status qgx_exchange(qgx_ctx *ctx, const float *v, int K, size_t d, const qgx_quant_cfg *cfg /*[host]*/,
+                        uint32_t exchange_id, int slot, float *mean_out, uint64_t *total_bits);
+/* Where the last qgx_exchange on `slot` left its streams: all [dev], valid until the next call
+ * that uses the slot.  Any output pointer may be NULL. */
+qgx_status qgx_exchange_streams(qgx_ctx *ctx, int slot, const uint32_t **stream, size_t *cap_words,
+                                const uint32_t **bucket_bits, const uint64_t **total_bits);
+
+/* ---- level adaptation (Sec. 3.3; Algorithm 1, "t in U") ------------------------------------- */
+
+/* Sufficient statistics and refit in one call: hist [dev] double[nbins] receives the histogram of
+ * the normalized magnitudes u of all K*nb buckets of v, each coordinate weighted by its bucket's
+ * squared norm (the weights lambda_j of Eq. QAda); then, on the host, cfg->levels is refitted
+ * (qgx_fit_levels, first fit iff refit == QGX_REFIT_FIRST) and cfg->cb rebuilt per cfg->code_type
+ * from the symbol weights.  Synchronizes the stream.  cfg [host] in/out; hist_host [host]
+ * double[nbins] out, may be NULL. */
+qgx_status qgx_update_levels(qgx_ctx *ctx, const float *v, int K, size_t d, qgx_quant_cfg *cfg,
+                             int refit, double *hist, double *hist_host);
+/* The histogram alone (asynchronous).  weighted == 0 counts coordinates instead. */
+qgx_status qgx_histogram(qgx_ctx *ctx, const float *v, int K, size_t d, int bucket, int norm_type,
+                         int nbins, int weighted, double *hist);
+
+/* ---- the iteration (Algorithm 1, Eq. Q-GenX, step size of Theorem 3) ------------------------ */
+
+/* Sets Y = 0, X = anchor, Xbar = 0, scalars = {0, K}, t = 1 (gamma_1 = K). */
+qgx_status qgx_eg_init(qgx_ctx *ctx, qgx_eg_state *st /*[host]*/);
+/* One iteration in the dual-extrapolation instance (two oracle calls, two exchanges):
+ *   V_{k,t} = A(X_t) + U_{k,t};  [refit of levels and code on V_{.,t} if refit != 0];
+ *   X_{t+1/2} = X_t - gamma_t mean_k Vhat_{k,t};   V_{k,t+1/2} = A(X_{t+1/2}) + U_{k,t+1/2};
+ *   Y_{t+1} = Y_t - mean_k Vhat_{k,t+1/2};  sum += sum_k ||Vhat_{k,t} - Vhat_{k,t+1/2}||^2;
+ *   gamma_{t+1} = K / sqrt(1 + sum);  X_{t+1} = anchor + gamma_{t+1} Y_{t+1};
+ *   Xbar += (X_{t+1/2} - Xbar) / t;  t += 1.
+ * noise_t, noise_half [dev] float[K][d] or NULL; exchange ids are 2t and 2t+1.  cfg [host] is
+ * in/out when refit != 0 (and the call then synchronizes once).  bits [dev] uint64[2][K]
+ * (stream bits of the two exchanges), may be NULL. */
+qgx_status qgx_eg_step(qgx_ctx *ctx, qgx_eg_state *st, const qgx_operator *op,
+                       const float *noise_t, const float *noise_half, qgx_quant_cfg *cfg,
+                       int refit, uint64_t *bits);
+/* A(x) alone: out [dev] float[d]. */
+qgx_status qgx_apply_operator(qgx_ctx *ctx, const qgx_operator *op, const float *x, float *out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QGX_H_ */

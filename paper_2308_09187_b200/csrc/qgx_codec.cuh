@@ -1,0 +1,105 @@
+// Device pieces of the prefix codec (Sec. 3.2 / App. J) shared by the stand-alone and the fused
+// kernels: packing a quad's codewords, placing bits into a shared-memory image of a bucket, and a
+// bounded bit reader with a table-driven decoder.
+#pragma once
+
+#include "qgx_common.cuh"
+
+namespace qgx {
+
+// shared-memory copy of the per-level stream bits: entry = bits | nbits << 16, where bits holds
+// the codeword in stream order followed by the sign bit for a negative nonzero level
+struct EncLut {
+  uint32_t e[2 * QGX_MAX_LEVELS];        // index: level | sign << 5
+};
+
+__device__ __forceinline__ void fill_enc_lut(EncLut* lut, const CodeTable& ct) {
+  for (int i = threadIdx.x; i < 2 * QGX_MAX_LEVELS; i += blockDim.x) {
+    const int idx = i & 31, neg = i >> 5;
+    uint32_t bits = 0, n = 0;
+    if (idx < ct.nlev) {
+      n = ct.len[idx];
+      bits = ct.rev[idx];
+      if (idx != 0) { bits |= (uint32_t)neg << n; n += 1; }
+    }
+    lut->e[i] = bits | (n << 16);
+  }
+}
+
+// stream bits of the four symbols of a quad, concatenated in coordinate order
+__device__ __forceinline__ void pack_quad(uint32_t packed_syms, int nvalid, const EncLut* lut, uint64_t* bits, uint32_t* nbits) {
+  uint64_t acc = 0;
+  uint32_t n = 0;
+#pragma unroll
+  for (int c = 0; c < kQuad; ++c) {
+    if (c < nvalid) {
+      const uint32_t s = (packed_syms >> (8 * c)) & 0xffu;
+      const uint32_t e = lut->e[(s & 31u) | ((s >> 7) << 5)];
+      acc |= (uint64_t)(e & 0xffffu) << n;
+      n += e >> 16;
+    }
+  }
+  *bits = acc;
+  *nbits = n;
+}
+
+// OR `nbits` bits into the bucket image at bit position pos (shared memory, zeroed before)
+__device__ __forceinline__ void put_bits(uint32_t* img, uint32_t pos, uint64_t bits, uint32_t nbits) {
+  if (nbits == 0) return;
+  const uint32_t w = pos >> 5, sh = pos & 31u;
+  const uint64_t lo = bits << sh;
+  const uint32_t x0 = (uint32_t)lo, x1 = (uint32_t)(lo >> 32);
+  const uint32_t x2 = sh ? (uint32_t)(bits >> (64 - sh)) : 0u;
+  if (x0) atomicOr(&img[w], x0);
+  if (x1) atomicOr(&img[w + 1], x1);
+  if (x2) atomicOr(&img[w + 2], x2);
+}
+
+// Decoder table: index = next `maxlen` stream bits, entry = level | codeword length << 8 (0 = no
+// codeword starts with these bits).
+constexpr int kDecLutMax = 1 << QGX_MAX_CODE_LEN;
+
+// Reads a bucket's words with every access bounded by nwords.
+struct BitReader {
+  const uint32_t* w;
+  uint32_t nwords;
+  uint32_t next;          // index of the next word to fetch
+  uint64_t buf;           // bits not yet consumed, next bit at bit 0
+  int avail;
+  __device__ __forceinline__ uint32_t fetch(uint32_t i) const { return i < nwords ? w[i] : 0u; }
+  __device__ __forceinline__ void seek(uint32_t bitpos) {
+    next = bitpos >> 5;
+    const uint32_t sh = bitpos & 31u;
+    buf = (uint64_t)(fetch(next) >> sh);
+    avail = 32 - (int)sh;
+    ++next;
+    refill();
+  }
+  __device__ __forceinline__ void refill() {
+    if (avail <= 32) {
+      buf |= (uint64_t)fetch(next) << avail;
+      avail += 32;
+      ++next;
+    }
+  }
+  __device__ __forceinline__ void skip(int n) { buf >>= n; avail -= n; }
+};
+
+// decodes one symbol; returns false on an unassigned pattern.  *used accumulates consumed bits.
+__device__ __forceinline__ bool decode_symbol(BitReader& br, const uint16_t* lut, uint32_t mask, uint32_t* sym, uint32_t* used) {
+  br.refill();
+  const uint32_t e = lut[(uint32_t)br.buf & mask];
+  const int L = (int)(e >> 8);
+  if (L == 0) return false;
+  const uint32_t idx = e & 0xffu;
+  br.skip(L);
+  uint32_t neg = 0;
+  if (idx != 0) { neg = (uint32_t)br.buf & 1u; br.skip(1); }
+  *sym = idx | (neg << 7);
+  *used += (uint32_t)L + (idx != 0 ? 1u : 0u);
+  return true;
+}
+
+void build_dec_lut_host(const CodeTable& ct, uint16_t* lut /*[1 << maxlen]*/);
+
+}  // namespace qgx

@@ -1,0 +1,151 @@
+// Shared device/host helpers of the qgx CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/qgx.h"
+
+namespace qgx {
+
+constexpr int kWarp = 32;
+constexpr int kNormBits = 32;            // C_b of App. E: the norm travels as an IEEE fp32 pattern
+constexpr int kQuad = 4;                 // coordinates per 128-bit load and per Philox block
+constexpr int kSpinLimit = 1 << 22;      // polls before a device-side wait gives up
+
+// device-resident status block of a context
+struct DevStatus {
+  unsigned int error;                    // first latched qgx_status, 0 if none
+  unsigned int pad;
+};
+
+}  // namespace qgx
+
+struct qgx_ctx {
+  int device;
+  cudaStream_t stream;
+  unsigned int* hstatus;                 // pinned host mirror
+  uint64_t launches;
+  // workspace of the fused calls, grown on demand
+  qgx::DevStatus* dstatus;               // [dev]
+  void* ws[16];
+  size_t ws_bytes[16];
+  // bookkeeping of the exchange slots
+  size_t slot_cap_words[2];
+  int slot_K[2];
+  size_t slot_nb[2];
+};
+
+namespace qgx {
+
+// ---- level table and code tables handed to kernels by value ---------------------------------
+struct LevelTable {
+  int nlev;
+  float lev[QGX_MAX_LEVELS];
+};
+
+struct CodeTable {
+  int nlev;
+  int maxlen;
+  int G;                                 // coordinates per sub-block (== bucket: no header)
+  int has_header;
+  // per level index: stream-order bits (first sent bit at bit 0) and length, without sign
+  uint16_t rev[QGX_MAX_LEVELS];
+  uint8_t len[QGX_MAX_LEVELS];
+};
+
+__host__ __device__ inline uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+
+inline int eff_subblock(int bucket, int subblock) {
+  return (subblock <= 0 || subblock >= bucket) ? bucket : subblock;
+}
+
+// latch the first error
+__device__ __forceinline__ void latch_error(DevStatus* st, unsigned int code) {
+  atomicCAS(&st->error, 0u, code);
+}
+
+// ---- Philox4x32-10 (Salmon et al., SC'11): counter-based, ten rounds ------------------------
+struct PhiloxKey {                       // the ten round keys, the same for every thread
+  uint32_t k0[10];
+  uint32_t k1[10];
+};
+
+inline PhiloxKey make_philox_key(uint64_t seed) {
+  PhiloxKey k;
+  uint32_t a = (uint32_t)seed, b = (uint32_t)(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    k.k0[r] = a;
+    k.k1[r] = b;
+    a += 0x9E3779B9u;                    // Weyl sequence of the golden ratio
+    b += 0xBB67AE85u;                    // Weyl sequence of sqrt(3) - 1
+  }
+  return k;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const PhiloxKey& key) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ key.k0[r];
+    const uint32_t n2 = hi0 ^ c3 ^ key.k1[r];
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// ---- Definition 1 for one normalized coordinate, every operation one IEEE rounding ----------
+// returns the level index; lev points to the table in shared memory
+__device__ __forceinline__ int quantize_level(float absv, float norm, const float* lev, int nlev, uint32_t word) {
+  float u = (norm > 0.0f) ? __fdiv_rn(absv, norm) : 0.0f;
+  u = fminf(u, 1.0f);
+  int tau = 0;
+  for (int j = 1; j <= nlev - 2; ++j) tau = (lev[j] <= u) ? j : tau;
+  const float num = __fsub_rn(u, lev[tau]);
+  const float den = __fsub_rn(lev[tau + 1], lev[tau]);
+  const float xi = __fdiv_rn(num, den);
+  const float r = __fmul_rn(__uint2float_rn(word >> 8), 5.9604644775390625e-8f);   // exact
+  return tau + ((r < xi) ? 1 : 0);
+}
+
+__device__ __forceinline__ uint32_t symbol_of(float v, int idx) {
+  const uint32_t neg = (__float_as_uint(v) >> 31) & (idx != 0 ? 1u : 0u);
+  return (uint32_t)idx | (neg << 7);
+}
+
+__device__ __forceinline__ float dequantize_symbol(uint32_t sym, float norm, const float* lev) {
+  const float val = __fmul_rn(norm, lev[sym & 31u]);
+  return __uint_as_float(__float_as_uint(val) ^ ((sym & 0x80u) << 24));
+}
+
+// ---- reductions ------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t x, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  return x;
+}
+
+// host side
+qgx_status check_levels_host(const float* lev, int nlev);
+qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out);
+void* ws_get(qgx_ctx* c, int which, size_t bytes);          // nullptr on failure
+qgx_status cuda_status(cudaError_t e);
+inline void count_launch(qgx_ctx* c, int n = 1) { c->launches += (uint64_t)n; }
+
+}  // namespace qgx
