@@ -353,3 +353,23 @@ def qgx_apply_operator(ctx, op, x, out=None):
         out = torch.empty((int(op.d),), dtype=torch.float32, device=x.device)
     _chk(lib().qgx_apply_operator(ctx.h, C.byref(op), _ptr(x), _ptr(out)), "qgx_apply_operator")
     return out
+
+
+class _DeviceView:
+    """Wraps a raw device pointer so that torch.as_tensor can view it without a copy."""
+
+    def __init__(self, ptr, n, typestr):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (int(ptr), False), "version": 2}
+
+
+def device_view(ptr, n, dtype):
+    typestr = {torch.int32: "<i4", torch.int64: "<i8", torch.float32: "<f4"}[dtype]
+    return torch.as_tensor(_DeviceView(ptr, n, typestr), device="cuda")
+
+
+def exchange_stream_tensors(ctx, slot, K, nb):
+    """(stream [K, cap_words] int32, bucket_bits [K, nb] int32, total_bits [K] int64) of a slot: views into
+    the context's workspace, valid until the next call that uses the slot."""
+    sp, cap, bp, tp = qgx_exchange_streams(ctx, slot, K, nb)
+    return (device_view(sp, K * cap, torch.int32).view(K, cap), device_view(bp, K * nb, torch.int32).view(K, nb),
+            device_view(tp, K, torch.int64))

@@ -101,7 +101,7 @@ void qgx_destroy(qgx_ctx* c) {
   if (!c) return;
   cudaSetDevice(c->device);
   cudaStreamSynchronize(c->stream);
-  for (int i = 0; i < 16; ++i)
+  for (int i = 0; i < 24; ++i)
     if (c->ws[i]) cudaFree(c->ws[i]);
   cudaFree(c->dstatus);
   cudaFreeHost(c->hstatus);

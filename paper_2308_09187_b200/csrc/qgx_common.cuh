@@ -29,8 +29,8 @@ struct qgx_ctx {
   uint64_t launches;
   // workspace of the fused calls, grown on demand
   qgx::DevStatus* dstatus;               // [dev]
-  void* ws[16];
-  size_t ws_bytes[16];
+  void* ws[24];
+  size_t ws_bytes[24];
   // bookkeeping of the exchange slots
   size_t slot_cap_words[2];
   int slot_K[2];
@@ -140,6 +140,14 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t x, int lane) {
   }
   return x;
 }
+
+// optional state update fused into the decode epilogue of an exchange
+struct ExchangeUpdate {
+  int mode;                      // 0 none, 1: xout = xin - gamma * mean, 2: xout = xin - mean
+  const float* xin;
+  float* xout;
+  const double* scalars;         // scalars[1] = gamma_t
+};
 
 // host side
 qgx_status check_levels_host(const float* lev, int nlev);

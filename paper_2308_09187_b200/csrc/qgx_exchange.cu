@@ -1,0 +1,547 @@
+// Fused exchange: one pass over the dual vectors writes the compact streams (quantize + encode),
+// one pass over the streams writes the mean (decode + average).  Same streams, bit for bit, and
+// the same mean as qgx_quantize -> qgx_encode -> qgx_decode -> qgx_average.
+#include "qgx_bucket.cuh"
+#include "qgx_codec.cuh"
+
+#include <algorithm>
+#include <vector>
+
+namespace qgx {
+
+// ---- chained scan of bucket lengths ("decoupled look-back") ----------------------------------
+// status word of bucket (k, b): bits 62..63 state, bits 0..61 a word count.
+constexpr unsigned long long kStEmpty = 0ull, kStAggregate = 1ull << 62, kStPrefix = 2ull << 62;
+constexpr unsigned long long kStMask = 3ull << 62;
+
+__device__ __forceinline__ unsigned long long ld_status(const unsigned long long* p) {
+  return *reinterpret_cast<const volatile unsigned long long*>(p);
+}
+__device__ __forceinline__ void st_status(unsigned long long* p, unsigned long long v) {
+  *reinterpret_cast<volatile unsigned long long*>(p) = v;
+}
+
+// Exclusive prefix (in words) of bucket b of one worker, by warp 0 of the CTA.  Buckets are handed
+// out by a ticket counter in the order b-major, k-minor, so every predecessor (k, b') with b' < b
+// belongs to a CTA that is already running or done: the wait below always ends; it is bounded all
+// the same, and *timed_out reports a wait that ran out.
+__device__ __forceinline__ unsigned long long lookback_prefix(unsigned long long* row /* status of worker k */, long long b,
+                                                              int lane, bool* timed_out) {
+  unsigned long long prefix = 0;
+  long long hi = b - 1;                                 // nearest predecessor not yet accounted for
+  int spins = 0;
+  bool fail = false;
+  while (hi >= 0 && !fail) {
+    const long long mine = hi - lane;
+    unsigned long long s = kStPrefix;                   // positions before bucket 0 act as a zero prefix
+    if (mine >= 0) s = ld_status(row + mine);
+    const unsigned empty = __ballot_sync(0xffffffffu, (s & kStMask) == kStEmpty);
+    const unsigned pref = __ballot_sync(0xffffffffu, (s & kStMask) == kStPrefix);
+    // lanes are ordered from the nearest predecessor outwards
+    const int first_pref = pref ? __ffs(pref) - 1 : 32;
+    const int first_empty = empty ? __ffs(empty) - 1 : 32;
+    if (first_empty < first_pref) {                     // a predecessor has not published yet
+      if (++spins > kSpinLimit) fail = true;
+      __nanosleep(64);
+      continue;
+    }
+    const int take = first_pref < 32 ? first_pref + 1 : 32;
+    unsigned long long part = lane < take ? (s & ~kStMask) : 0ull;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    prefix += part;
+    if (first_pref < 32) break;
+    hi -= 32;
+  }
+  *timed_out = fail;
+  return prefix;
+}
+
+struct EncodeArgs {
+  DualSource src;
+  size_t d;
+  int bucket;
+  int K;
+  size_t nb;
+  int norm_type;
+  uint32_t xid;
+  bool vec_ok;
+  uint32_t* stream;
+  size_t cap_words;
+  uint32_t* bucket_bits;        // [K][nb]
+  uint32_t* offsets;            // [K][nb] word offset of each bucket
+  unsigned long long* total_bits;   // [K], zeroed before the launch
+  float* norms;                 // [K][nb] (kept for the caller; the streams carry them too)
+  unsigned long long* status;   // [K][nb], zeroed before the launch
+  unsigned int* ticket;         // zeroed before the launch
+  DevStatus* st;
+};
+
+template <int V4>
+__global__ void __launch_bounds__(512) k_exchange_encode(EncodeArgs a, LevelTable lt, CodeTable ct, PhiloxKey key) {
+  extern __shared__ uint32_t s_dyn[];
+  __shared__ EncLut s_lut;
+  __shared__ float s_lev[QGX_MAX_LEVELS];
+  __shared__ double s_red[34];
+  __shared__ uint32_t s_chunk[264];
+  __shared__ unsigned int s_ticket;
+  __shared__ unsigned long long s_prefix;
+  __shared__ int s_skip;
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int img_words = (int)((((uint32_t)a.bucket * (uint32_t)(ct.maxlen + 1) + 16u * (uint32_t)(a.bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4);
+  uint32_t* s_img = s_dyn;
+  uint32_t* s_sub = s_dyn + img_words;
+  const int qps = ct.G / kQuad;
+  const unsigned long long total = (unsigned long long)a.nb * (unsigned long long)a.K;
+
+  fill_enc_lut(&s_lut, ct);
+  if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 1.0f;
+
+  for (;;) {
+    __syncthreads();                                    // shared state of the previous bucket is no longer read
+    if (threadIdx.x == 0) s_ticket = atomicAdd(a.ticket, 1u);
+    __syncthreads();
+    const unsigned long long t = s_ticket;
+    if (t >= total) break;
+    const size_t b = (size_t)(t / (unsigned long long)a.K), k = (size_t)(t % (unsigned long long)a.K);
+    const size_t lo = b * (size_t)a.bucket;
+    const int len = (int)min((size_t)a.bucket, a.d - lo);
+
+    BucketRegs<V4> r;
+    load_bucket<V4>(r, a.src, k, a.d, lo, len, a.vec_ok);
+    const float norm = bucket_norm<V4>(r, a.norm_type, s_red);
+    const bool finite = (norm - norm) == 0.0f;
+    if (threadIdx.x == 0) {
+      a.norms[k * a.nb + b] = norm;
+      if (!finite) latch_error(a.st, QGX_ERR_NONFINITE);
+    }
+
+    uint64_t qbits[V4];
+    uint32_t qn[V4], qexcl[V4];
+#pragma unroll
+    for (int j = 0; j < V4; ++j) {
+      const int q = j * (int)blockDim.x + (int)threadIdx.x;
+      const int nvalid = max(0, min(kQuad, len - q * kQuad));
+      uint32_t packed = 0;
+      if (nvalid > 0 && finite) {
+        const uint64_t ctr = (uint64_t)(lo >> 2) + (uint64_t)q;
+        const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
+        const float4 x = r.x[j];
+        const uint32_t s0 = symbol_of(x.x, quantize_level(fabsf(x.x), norm, s_lev, lt.nlev, w.x));
+        const uint32_t s1 = symbol_of(x.y, quantize_level(fabsf(x.y), norm, s_lev, lt.nlev, w.y));
+        const uint32_t s2 = symbol_of(x.z, quantize_level(fabsf(x.z), norm, s_lev, lt.nlev, w.z));
+        const uint32_t s3 = symbol_of(x.w, quantize_level(fabsf(x.w), norm, s_lev, lt.nlev, w.w));
+        packed = s0 | (s1 << 8) | (s2 << 16) | (s3 << 24);
+      }
+      pack_quad(packed, nvalid, &s_lut, &qbits[j], &qn[j]);
+      const uint32_t incl = warp_incl_scan(qn[j], lane);
+      qexcl[j] = incl - qn[j];
+      if (lane == 31) s_chunk[j * nwarps + warp] = incl;
+    }
+    __syncthreads();
+    const int nchunks = V4 * nwarps;
+    if (warp == 0) {
+      uint32_t carry = 0;
+      for (int base = 0; base < nchunks; base += 32) {
+        const int i = base + lane;
+        const uint32_t x = i < nchunks ? s_chunk[i] : 0u;
+        const uint32_t incl = warp_incl_scan(x, lane);
+        if (i < nchunks) s_chunk[i] = carry + incl - x;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (lane == 0) s_chunk[nchunks] = carry;
+    }
+    __syncthreads();
+    const uint32_t nsub = ct.has_header ? (uint32_t)((len + ct.G - 1) / ct.G) : 0u;
+    const uint32_t hdr_bits = kNormBits + 16u * nsub;
+    const uint32_t nbits = hdr_bits + s_chunk[nchunks];
+    const uint32_t nwords = (nbits + 31) >> 5;
+    unsigned long long* row = a.status + k * a.nb;
+    if (threadIdx.x == 0) {
+      st_status(row + b, kStAggregate | (unsigned long long)nwords);   // publish the length as early as possible
+      a.bucket_bits[k * a.nb + b] = nbits;
+      atomicAdd(a.total_bits + k, (unsigned long long)nbits);
+    }
+    for (uint32_t i = threadIdx.x; i < nwords + 2; i += blockDim.x) s_img[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < V4; ++j) {
+      const int q = j * (int)blockDim.x + (int)threadIdx.x;
+      const uint32_t p = s_chunk[j * nwarps + warp] + qexcl[j];
+      if (nsub && q * kQuad < len && q % qps == 0) s_sub[q / qps] = p;
+      put_bits(s_img, hdr_bits + p, qbits[j], qn[j]);
+    }
+    if (threadIdx.x == 0) {
+      atomicOr(&s_img[0], __float_as_uint(norm));
+      if (nsub) s_sub[nsub] = s_chunk[nchunks];
+    }
+    // meanwhile warp 0 finds where the bucket goes
+    if (warp == 0) {
+      bool timed_out = false;
+      const unsigned long long excl = lookback_prefix(row, (long long)b, lane, &timed_out);
+      if (lane == 0) {
+        st_status(row + b, kStPrefix | (excl + (unsigned long long)nwords));
+        int skip = 0;
+        if (timed_out) { latch_error(a.st, QGX_ERR_TIMEOUT); skip = 1; }
+        if (excl + nwords > (unsigned long long)a.cap_words) { latch_error(a.st, QGX_ERR_CAPACITY); skip = 1; }
+        a.offsets[k * a.nb + b] = (uint32_t)min(excl, (unsigned long long)0xffffffffu);
+        s_prefix = excl;
+        s_skip = skip;
+      }
+    }
+    __syncthreads();
+    for (uint32_t s = threadIdx.x; s < nsub; s += blockDim.x) {
+      const uint32_t L = s_sub[s + 1] - s_sub[s];
+      put_bits(s_img, kNormBits + 16u * s, (uint64_t)(L & 0xffffu), 16u);
+    }
+    __syncthreads();
+    if (!s_skip) {
+      uint32_t* dst = a.stream + k * a.cap_words + s_prefix;
+      for (uint32_t i = threadIdx.x; i < nwords; i += blockDim.x) dst[i] = s_img[i];
+    }
+  }
+}
+
+// ---- decode + average ------------------------------------------------------------------------
+struct DecodeArgs {
+  const uint32_t* stream;       // [K][cap_words]
+  size_t cap_words;
+  const uint32_t* bucket_bits;  // [K][nb]
+  const uint32_t* offsets;      // [K][nb]
+  // second stream set whose decoded vectors are compared with the first (may be null)
+  const uint32_t* stream2;
+  size_t cap_words2;
+  const uint32_t* bucket_bits2;
+  const uint32_t* offsets2;
+  double* sum_sq;               // += sum_k ||vhat - vhat2||^2 (fp32 differences, fp64 sum)
+  size_t d;
+  int bucket;
+  int K;
+  size_t nb;
+  const uint16_t* lut;          // decoder table in global memory
+  float* mean;                  // [d]
+  // optional fused state update (the two axpy of Eq. Q-GenX)
+  int update;                   // 0 none, 1: xout = xin - gamma * mean, 2: xout = xin - mean
+  const float* xin;
+  float* xout;
+  const double* scalars;        // scalars[1] = gamma_t
+  DevStatus* st;
+};
+
+// start of sub-block `s` (bits after the header) = sum of the 16-bit lengths before it; all lanes
+// of the warp share the bucket; returns false if the header is inconsistent with nbits
+__device__ __forceinline__ uint32_t subblock_start(const uint32_t* w, uint32_t s, int lane) {
+  // lengths of sub-blocks [0, s - lane) are summed cooperatively, then a scan inside the warp
+  const uint32_t warp_first = s - (uint32_t)lane;
+  uint32_t before = 0;
+  for (uint32_t i = (uint32_t)lane; i < warp_first; i += 32) {
+    const uint32_t bit = kNormBits + 16u * i;
+    before += (w[bit >> 5] >> (bit & 31u)) & 0xffffu;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+  return before;
+}
+
+template <int G, bool DIFF>
+__global__ void __launch_bounds__(128) k_exchange_decode(DecodeArgs a, LevelTable lt, CodeTable ct) {
+  extern __shared__ uint32_t s_dyn[];
+  __shared__ float s_lev[QGX_MAX_LEVELS];
+  uint16_t* s_lut = reinterpret_cast<uint16_t*>(s_dyn);
+  const int lut_n = 1 << ct.maxlen;
+  for (int i = threadIdx.x; i < lut_n; i += blockDim.x) s_lut[i] = a.lut[i];
+  if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 0.0f;
+  __syncthreads();
+  const uint32_t mask = (uint32_t)lut_n - 1u;
+  const int lane = threadIdx.x & 31;
+  const size_t spb = (size_t)a.bucket / G;              // sub-blocks per full bucket (bucket % G == 0, spb % 32 == 0 or spb < 32 handled by the host)
+  const size_t total_sub = a.nb * spb;
+  const float Kf = (float)a.K;
+  double sq = 0.0;
+  bool bad = false;
+
+  for (size_t gs = (size_t)blockIdx.x * blockDim.x + threadIdx.x; gs - lane < total_sub; gs += (size_t)gridDim.x * blockDim.x) {
+    // the warp's 32 sub-blocks lie in one bucket when spb % 32 == 0; otherwise lanes may differ
+    const bool live = gs < total_sub;
+    const size_t b = live ? gs / spb : a.nb - 1;
+    const uint32_t s = live ? (uint32_t)(gs % spb) : 0u;
+    const size_t lo = b * (size_t)a.bucket;
+    const int len = (int)min((size_t)a.bucket, a.d - lo);
+    const int first = (int)s * G;
+    const int count = live ? max(0, min(G, len - first)) : 0;
+    const uint32_t nsub = (uint32_t)((len + G - 1) / G);
+    const uint32_t hdr_bits = kNormBits + 16u * nsub;
+    const bool uniform = (spb % 32 == 0);
+
+    float acc[G];
+#pragma unroll
+    for (int i = 0; i < G; ++i) acc[i] = 0.0f;
+    // a warp none of whose sub-blocks exists (beyond the end of a short last bucket) reads nothing
+    if (!__any_sync(0xffffffffu, count > 0)) continue;
+
+    for (int k = 0; k < a.K; ++k) {
+      const uint32_t nbits = a.bucket_bits[(size_t)k * a.nb + b];
+      const uint32_t nwords = (nbits + 31) >> 5;
+      const uint32_t* w = a.stream + (size_t)k * a.cap_words + a.offsets[(size_t)k * a.nb + b];
+      const bool hdr_ok = nbits >= hdr_bits && (size_t)a.offsets[(size_t)k * a.nb + b] + nwords <= a.cap_words;
+      uint32_t start = 0, want = 0;
+      float norm = 0.0f;
+      if (hdr_ok) {
+        norm = __uint_as_float(w[0]);
+        if (uniform) {
+          const uint32_t bit = kNormBits + 16u * s;
+          const uint32_t mylen = (count > 0) ? ((w[bit >> 5] >> (bit & 31u)) & 0xffffu) : 0u;
+          const uint32_t incl = warp_incl_scan(mylen, lane);
+          start = subblock_start(w, s, lane) + incl - mylen;
+          want = mylen;
+        } else if (count > 0) {
+          for (uint32_t i = 0; i <= s; ++i) {
+            const uint32_t bit = kNormBits + 16u * i;
+            const uint32_t L = (w[bit >> 5] >> (bit & 31u)) & 0xffffu;
+            if (i < s) start += L; else want = L;
+          }
+        }
+      } else {
+        bad = true;
+      }
+      // second stream set (the other exchange of the iteration), same geometry
+      uint32_t start2 = 0, want2 = 0;
+      float norm2 = 0.0f;
+      const uint32_t* w2 = nullptr;
+      uint32_t nwords2 = 0;
+      bool ok2 = false;
+      if (DIFF) {
+        const uint32_t nbits2 = a.bucket_bits2[(size_t)k * a.nb + b];
+        nwords2 = (nbits2 + 31) >> 5;
+        w2 = a.stream2 + (size_t)k * a.cap_words2 + a.offsets2[(size_t)k * a.nb + b];
+        ok2 = nbits2 >= hdr_bits && (size_t)a.offsets2[(size_t)k * a.nb + b] + nwords2 <= a.cap_words2;
+        if (ok2) {
+          norm2 = __uint_as_float(w2[0]);
+          if (uniform) {
+            const uint32_t bit = kNormBits + 16u * s;
+            const uint32_t mylen = (count > 0) ? ((w2[bit >> 5] >> (bit & 31u)) & 0xffffu) : 0u;
+            const uint32_t incl = warp_incl_scan(mylen, lane);
+            start2 = subblock_start(w2, s, lane) + incl - mylen;
+            want2 = mylen;
+          } else if (count > 0) {
+            for (uint32_t i = 0; i <= s; ++i) {
+              const uint32_t bit = kNormBits + 16u * i;
+              const uint32_t L = (w2[bit >> 5] >> (bit & 31u)) & 0xffffu;
+              if (i < s) start2 += L; else want2 = L;
+            }
+          }
+        } else {
+          bad = true;
+        }
+      }
+      if (count <= 0) continue;
+      if (hdr_ok && hdr_bits + start + want > nbits) { bad = true; continue; }
+      if (DIFF && ok2 && hdr_bits + start2 + want2 > nwords2 * 32u) { bad = true; continue; }
+
+      BitReader br;
+      br.w = w; br.nwords = hdr_ok ? nwords : 0u;
+      br.seek(hdr_bits + start);
+      BitReader br2;
+      if (DIFF) { br2.w = w2; br2.nwords = ok2 ? nwords2 : 0u; br2.seek(hdr_bits + start2); }
+      uint32_t used = 0, used2 = 0;
+      bool ok = hdr_ok, okb = ok2;
+#pragma unroll
+      for (int i = 0; i < G; ++i) {
+        if (i < count) {
+          uint32_t sym = 0;
+          if (ok) ok = decode_symbol(br, s_lut, mask, &sym, &used) && used <= want;
+          if (!ok) sym = 0;
+          const float val = dequantize_symbol(sym, norm, s_lev);
+          acc[i] = __fadd_rn(acc[i], val);
+          if (DIFF) {
+            uint32_t sym2 = 0;
+            if (okb) okb = decode_symbol(br2, s_lut, mask, &sym2, &used2) && used2 <= want2;
+            if (!okb) sym2 = 0;
+            const float dlt = __fsub_rn(val, dequantize_symbol(sym2, norm2, s_lev));
+            sq = fma((double)dlt, (double)dlt, sq);
+          }
+        }
+      }
+      if (!ok || used != want) bad = true;
+      if (DIFF && (!okb || used2 != want2)) bad = true;
+    }
+
+    // mean (and the fused state update) for this sub-block's coordinates
+    if (count > 0) {
+      const size_t e0 = lo + (size_t)first;
+      float gam = 1.0f;
+      if (a.update == 1) gam = (float)a.scalars[1];
+#pragma unroll
+      for (int i = 0; i < G; ++i) {
+        if (i < count) {
+          const float m = __fdiv_rn(acc[i], Kf);
+          a.mean[e0 + i] = m;
+          if (a.update == 1) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], __fmul_rn(gam, m));
+          if (a.update == 2) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], m);
+        }
+      }
+    }
+  }
+  if (DIFF) {
+    sq = warp_sum(sq);
+    if (lane == 0 && sq != 0.0) atomicAdd(a.sum_sq, sq);
+  }
+  if (bad) latch_error(a.st, QGX_ERR_CORRUPT);
+}
+
+}  // namespace qgx
+
+// ---- host side ---------------------------------------------------------------------------------
+namespace qgx {
+
+// workspace slots of a context
+enum { WS_OFF64 = 0, WS_FLAGS = 1, WS_LUT = 2, WS_SLOT0 = 3 /* stream, bits, offsets, total: 3..6 and 7..10 */,
+       WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16 };
+
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const LevelTable& lt, const CodeTable& ct, bool diff);
+
+// the whole exchange; diff_slot >= 0 also accumulates sum_k ||vhat(slot) - vhat(diff_slot)||^2 into sum_sq
+qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
+                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int diff_slot, double* sum_sq) {
+  if (!c || !cfg || !mean_out || K < 1 || K > 65535 || d < 1 || slot < 0 || slot > 1) return QGX_ERR_INVALID_ARG;
+  const int bucket = cfg->bucket;
+  if (bucket < kQuad || bucket > QGX_MAX_BUCKET || bucket % kQuad != 0) return QGX_ERR_INVALID_ARG;
+  if (cfg->norm_type != QGX_NORM_L2 && cfg->norm_type != QGX_NORM_LINF) return QGX_ERR_INVALID_ARG;
+  if (check_levels_host(cfg->levels, cfg->nlev) != QGX_OK) return QGX_ERR_BAD_LEVELS;
+  if (cfg->cb.nlev != cfg->nlev) return QGX_ERR_INVALID_ARG;
+  CodeTable ct;
+  qgx_status rc = make_code_table(&cfg->cb, bucket, &ct);
+  if (rc != QGX_OK) return rc;
+  if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
+  LevelTable lt;
+  lt.nlev = cfg->nlev;
+  for (int j = 0; j < QGX_MAX_LEVELS; ++j) lt.lev[j] = j < cfg->nlev ? cfg->levels[j] : 1.0f;
+
+  const size_t nb = (d + (size_t)bucket - 1) / (size_t)bucket;
+  const size_t cap = qgx_stream_capacity_words(d, bucket, cfg->cb.subblock, QGX_MAX_CODE_LEN);   // fits any codebook
+  const int base = WS_SLOT0 + 4 * slot;
+  uint32_t* stream = (uint32_t*)ws_get(c, base + 0, sizeof(uint32_t) * (size_t)K * cap);
+  uint32_t* bbits = (uint32_t*)ws_get(c, base + 1, sizeof(uint32_t) * (size_t)K * nb);
+  uint32_t* offs = (uint32_t*)ws_get(c, base + 2, sizeof(uint32_t) * (size_t)K * nb);
+  unsigned long long* tot = (unsigned long long*)ws_get(c, base + 3, sizeof(uint64_t) * (size_t)K);
+  unsigned long long* status = (unsigned long long*)ws_get(c, WS_STATUS, sizeof(uint64_t) * ((size_t)K * nb + 2));
+  float* norms = (float*)ws_get(c, WS_NORMS, sizeof(float) * (size_t)K * nb);
+  uint16_t* lut = (uint16_t*)ws_get(c, WS_LUT, sizeof(uint16_t) * kDecLutMax);
+  if (!stream || !bbits || !offs || !tot || !status || !norms || !lut) return QGX_ERR_CUDA;
+  c->slot_cap_words[slot] = cap;
+  c->slot_K[slot] = K;
+  c->slot_nb[slot] = nb;
+
+  if (cudaMemsetAsync(status, 0, sizeof(uint64_t) * ((size_t)K * nb + 2), c->stream) != cudaSuccess ||
+      cudaMemsetAsync(tot, 0, sizeof(uint64_t) * (size_t)K, c->stream) != cudaSuccess)
+    return QGX_ERR_CUDA;
+
+  EncodeArgs ea;
+  ea.src = src; ea.d = d; ea.bucket = bucket; ea.K = K; ea.nb = nb; ea.norm_type = cfg->norm_type; ea.xid = xid;
+  ea.vec_ok = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(src.v) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
+  ea.stream = stream; ea.cap_words = cap; ea.bucket_bits = bbits; ea.offsets = offs; ea.total_bits = tot; ea.norms = norms;
+  ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(status + (size_t)K * nb); ea.st = c->dstatus;
+  const PhiloxKey key = make_philox_key(cfg->seed);
+  const int v4 = bucket_v4(bucket);
+  const int threads = bucket_threads(bucket, v4);
+  const size_t img_words = (((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4;
+  const size_t smem = sizeof(uint32_t) * (img_words + (size_t)(bucket / ct.G) + 2);
+  int per_sm = 1;
+#define QGX_LAUNCH_E(V)                                                                                        \
+  do {                                                                                                         \
+    cudaFuncSetAttribute(k_exchange_encode<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V>, threads, smem);               \
+    if (per_sm < 1) per_sm = 1;                                                                                \
+    const unsigned long long want = (unsigned long long)nb * (unsigned long long)K;                            \
+    const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);   \
+    k_exchange_encode<V><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key);                                  \
+  } while (0)
+  switch (v4) {
+    case 1: QGX_LAUNCH_E(1); break;
+    case 2: QGX_LAUNCH_E(2); break;
+    case 4: QGX_LAUNCH_E(4); break;
+    default: QGX_LAUNCH_E(8); break;
+  }
+#undef QGX_LAUNCH_E
+  count_launch(c);
+  if (cudaGetLastError() != cudaSuccess) return QGX_ERR_CUDA;
+  if (total_bits_out &&
+      cudaMemcpyAsync(total_bits_out, tot, sizeof(uint64_t) * (size_t)K, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
+    return QGX_ERR_CUDA;
+
+  // decoder table
+  std::vector<uint16_t> h_lut((size_t)1 << ct.maxlen);
+  build_dec_lut_host(ct, h_lut.data());
+  if (cudaMemcpyAsync(lut, h_lut.data(), h_lut.size() * sizeof(uint16_t), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+    return QGX_ERR_CUDA;
+
+  DecodeArgs da;
+  da.stream = stream; da.cap_words = cap; da.bucket_bits = bbits; da.offsets = offs;
+  da.stream2 = nullptr; da.cap_words2 = 0; da.bucket_bits2 = nullptr; da.offsets2 = nullptr; da.sum_sq = sum_sq;
+  bool diff = false;
+  if (diff_slot >= 0) {
+    if (diff_slot > 1 || diff_slot == slot || c->slot_K[diff_slot] != K || c->slot_nb[diff_slot] != nb || !sum_sq) return QGX_ERR_INVALID_ARG;
+    const int b2 = WS_SLOT0 + 4 * diff_slot;
+    da.stream2 = (const uint32_t*)c->ws[b2 + 0]; da.cap_words2 = c->slot_cap_words[diff_slot];
+    da.bucket_bits2 = (const uint32_t*)c->ws[b2 + 1]; da.offsets2 = (const uint32_t*)c->ws[b2 + 2];
+    diff = true;
+  }
+  da.d = d; da.bucket = bucket; da.K = K; da.nb = nb; da.lut = lut; da.mean = mean_out;
+  da.update = upd ? upd->mode : 0; da.xin = upd ? upd->xin : nullptr; da.xout = upd ? upd->xout : nullptr;
+  da.scalars = upd ? upd->scalars : nullptr; da.st = c->dstatus;
+  return launch_decode_average(c, da, lt, ct, diff);
+}
+
+template <int G>
+static void launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const LevelTable& lt, const CodeTable& ct, bool diff) {
+  const size_t total_sub = da.nb * ((size_t)da.bucket / G);
+  const int threads = 128;
+  const size_t smem = sizeof(uint16_t) * ((size_t)1 << ct.maxlen);
+  int per_sm = 1;
+  if (diff) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, true>, threads, smem);
+  else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, false>, threads, smem);
+  if (per_sm < 1) per_sm = 1;
+  const size_t want = (total_sub + threads - 1) / threads;
+  const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
+  if (diff) k_exchange_decode<G, true><<<grid, threads, smem, c->stream>>>(da, lt, ct);
+  else k_exchange_decode<G, false><<<grid, threads, smem, c->stream>>>(da, lt, ct);
+  count_launch(c);
+}
+
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const LevelTable& lt, const CodeTable& ct, bool diff) {
+  if (!ct.has_header || da.bucket % ct.G != 0) return QGX_ERR_INVALID_ARG;
+  switch (ct.G) {
+    case 32: launch_decode_g<32>(c, da, lt, ct, diff); break;
+    case 64: launch_decode_g<64>(c, da, lt, ct, diff); break;
+    case 128: launch_decode_g<128>(c, da, lt, ct, diff); break;
+    default: return QGX_ERR_INVALID_ARG;
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace qgx
+
+using namespace qgx;
+
+extern "C" {
+
+qgx_status qgx_exchange(qgx_ctx* c, const float* v, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t exchange_id,
+                        int slot, float* mean_out, uint64_t* total_bits) {
+  if (!v) return QGX_ERR_INVALID_ARG;
+  DualSource src{v, nullptr};
+  return exchange_impl(c, src, K, d, cfg, exchange_id, slot, mean_out, total_bits, nullptr, -1, nullptr);
+}
+
+qgx_status qgx_exchange_streams(qgx_ctx* c, int slot, const uint32_t** stream, size_t* cap_words,
+                                const uint32_t** bucket_bits, const uint64_t** total_bits) {
+  if (!c || slot < 0 || slot > 1 || c->slot_K[slot] == 0) return QGX_ERR_INVALID_ARG;
+  const int base = WS_SLOT0 + 4 * slot;
+  if (stream) *stream = (const uint32_t*)c->ws[base + 0];
+  if (cap_words) *cap_words = c->slot_cap_words[slot];
+  if (bucket_bits) *bucket_bits = (const uint32_t*)c->ws[base + 1];
+  if (total_bits) *total_bits = (const uint64_t*)c->ws[base + 3];
+  return QGX_OK;
+}
+
+}  // extern "C"

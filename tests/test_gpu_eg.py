@@ -1,0 +1,164 @@
+"""Parity of qgx_eg_step and the operator kernels with the oracle: teacher-forced per step (the
+library starts every step from the oracle's state) and free-running over whole trajectories."""
+import numpy as np
+import pytest
+import torch
+
+import qgx_inputs as gen
+from oracle import qgx_oracle as o
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_2308_09187_b200 as qgx
+    ctx = qgx.qgx_create(0)
+    yield qgx, ctx
+    qgx.qgx_destroy(ctx)
+
+
+def _rel(a, b):
+    b = np.asarray(b, dtype=np.float64)
+    return float(np.max(np.abs(np.asarray(a, dtype=np.float64) - b)) / max(np.max(np.abs(b)), 1e-30))
+
+
+def test_operators(q):
+    qgx, ctx = q
+    n = 1000
+    M = gen.gaussian((n, n), 1, "cuda")
+    b = gen.gaussian((n,), 2, "cuda")
+    x = gen.gaussian((n,), 3, "cuda")
+    out = qgx.qgx_apply_operator(ctx, qgx.make_operator(qgx.QGX_OP_DENSE_AFFINE, M, b), x)
+    ref = o.apply_operator(o.Op(o.OP_DENSE_AFFINE, M.cpu().numpy(), b.cpu().numpy()), x.cpu().numpy())
+    assert _rel(out.cpu().numpy(), ref) <= 1e-6
+    A = gen.gaussian((513, 513), 4, "cuda")
+    z = gen.gaussian((1026,), 5, "cuda")
+    out = qgx.qgx_apply_operator(ctx, qgx.make_operator(qgx.QGX_OP_BILINEAR, A), z)
+    ref = o.apply_operator(o.Op(o.OP_BILINEAR, A.cpu().numpy()), z.cpu().numpy())
+    assert _rel(out.cpu().numpy(), ref) <= 1e-6
+    D = gen.uniform((5000,), 6, "cuda", 0.01, 1.0)
+    xx = gen.gaussian((5000,), 7, "cuda")
+    out = qgx.qgx_apply_operator(ctx, qgx.make_operator(qgx.QGX_OP_DIAGONAL, D), xx)
+    assert np.array_equal(out.cpu().numpy(), o.apply_operator(o.Op(o.OP_DIAGONAL, D.cpu().numpy()), xx.cpu().numpy()))
+    qgx.qgx_sync_status(ctx)
+
+
+def _load_state(qgx, st_gpu, st_or):
+    st_gpu.X.copy_(torch.from_numpy(st_or.X))
+    st_gpu.Y.copy_(torch.from_numpy(st_or.Y))
+    st_gpu.Xbar.copy_(torch.from_numpy(st_or.Xbar))
+    st_gpu.scalars.copy_(torch.tensor([st_or.sum_sq, float(st_or.gamma)], dtype=torch.float64))
+    st_gpu.c.t = st_or.t
+
+
+def _compare(st_gpu, st_or, tol=1e-5):
+    s, g = st_gpu.read_scalars()
+    assert _rel(st_gpu.Xhalf.cpu().numpy(), st_or.Xhalf) <= tol
+    assert _rel(st_gpu.Y.cpu().numpy(), st_or.Y) <= tol
+    assert _rel(st_gpu.X.cpu().numpy(), st_or.X) <= tol
+    assert _rel(st_gpu.Xbar.cpu().numpy(), st_or.Xbar) <= tol
+    assert abs(s - st_or.sum_sq) <= tol * max(st_or.sum_sq, 1e-30)
+    assert abs(g - st_or.gamma) <= tol * st_or.gamma
+    assert st_gpu.t == st_or.t
+
+
+def test_bilinear_game_teacher_forced_and_free_running(q):
+    """c1: n = 1024 (d = 2048), K = 4, bucket 512, 9 uniform levels, fixed-length code, 100 iterations."""
+    qgx, ctx = q
+    T = 100
+    g = gen.c1_bilinear(T=T, device="cuda")
+    A, z0, noise = g.A.cpu().numpy(), g.z0.cpu().numpy(), g.noise.cpu().numpy()
+    lev = gen.uniform_levels(9).numpy()
+    cb = qgx.qgx_build_codebook_fixed(9, 128)
+    cbo = o.codebook_from(cb.lengths(), cb.codes(), subblock=128)
+    cfg = qgx.make_quant_cfg(lev, g.bucket, cb, g.seed)
+    op = qgx.make_operator(qgx.QGX_OP_BILINEAR, g.A)
+    opo = o.Op(o.OP_BILINEAR, A)
+    st_f = qgx.EgState(g.z0, g.K)          # free running
+    st_t = qgx.EgState(g.z0, g.K)          # teacher forced
+    qgx.qgx_eg_init(ctx, st_f)
+    qgx.qgx_eg_init(ctx, st_t)
+    st_o = o.EgState(z0, g.K)
+    bits = torch.zeros((2, g.K), dtype=torch.int64, device="cuda")
+    for t in range(T):
+        _load_state(qgx, st_t, st_o)
+        bits_o = o.eg_step(st_o, opo, noise[t, 0], noise[t, 1], g.bucket, lev, cbo, g.seed)
+        qgx.qgx_eg_step(ctx, st_t, op, g.noise[t, 0], g.noise[t, 1], cfg, bits=bits)
+        qgx.qgx_eg_step(ctx, st_f, op, g.noise[t, 0], g.noise[t, 1], cfg)
+        if t % 10 == 0 or t == T - 1:
+            qgx.qgx_sync_status(ctx)
+            _compare(st_t, st_o)
+            assert int(bits.sum().item()) == bits_o
+    qgx.qgx_sync_status(ctx)
+    _compare(st_f, st_o, tol=1e-4)          # free running: the same trajectory up to rare level flips
+    s, gam = st_f.read_scalars()
+    assert abs(1.0 / gam ** 2 - (1.0 + s) / g.K ** 2) <= 1e-6 * (1.0 + s) / g.K ** 2     # step-size identity
+    assert float(st_f.Xbar.norm()) < float(g.z0.norm())                                   # towards z* = 0
+
+
+def test_affine_vi_with_refits_teacher_forced(q):
+    """c4 at reduced size: V(x) = M x + b, K = 8, noise sigma = 1, 17 adaptive levels refitted every 10 steps."""
+    qgx, ctx = q
+    n, T = 512, 40
+    vi = gen.c4_affine(n=n, K=8, device="cuda", bucket=128)
+    M, b = vi.M.cpu().numpy(), vi.b.cpu().numpy()
+    xstar = np.linalg.solve(M.astype(np.float64), -b.astype(np.float64))
+    assert np.linalg.norm(M.astype(np.float64) @ xstar + b) <= 1e-12 * np.linalg.norm(b)
+    lev_o = gen.uniform_levels(17).numpy().copy()
+    cb = qgx.qgx_build_codebook_fixed(17, 32)
+    cbo = o.codebook_fixed(17, 32)
+    cfg = qgx.make_quant_cfg(lev_o, vi.bucket, cb, vi.seed, code_type=qgx.QGX_CODE_HUFFMAN, nbins=256)
+    op = qgx.make_operator(qgx.QGX_OP_DENSE_AFFINE, vi.M, vi.b)
+    opo = o.Op(o.OP_DENSE_AFFINE, M, b)
+    st_t = qgx.EgState(vi.x0, vi.K)
+    qgx.qgx_eg_init(ctx, st_t)
+    st_o = o.EgState(vi.x0.cpu().numpy(), vi.K)
+    for t in range(1, T + 1):
+        nz = vi.noise(t)
+        nzh = nz.cpu().numpy()
+        refit = 2 if t == 1 else (1 if (t - 1) % 10 == 0 else 0)
+        _load_state(qgx, st_t, st_o)
+        # both sides quantize with the same table and code: the library's refit result is handed to the oracle
+        qgx.qgx_eg_step(ctx, st_t, op, nz[0], nz[1], cfg, refit=refit)
+        if refit:
+            lev_ref = lev_o.copy()
+            a = o.apply_operator(opo, st_o.X)
+            V = o.form_dual_vectors(a, nzh[0], vi.K)
+            lev_ref, _ = o.refit(V, vi.bucket, 256, lev_ref, cbo, refit == 2, o.CODE_HUFFMAN)
+            got = np.array(cfg.level_list(), dtype=np.float32)
+            assert np.max(np.abs(got - lev_ref)) < 5e-5
+            lev_o = got.copy()
+            cbo = o.codebook_from(cfg.cb.lengths(), cfg.cb.codes(), subblock=32)
+        o.eg_step(st_o, opo, nzh[0], nzh[1], vi.bucket, lev_o, cbo, vi.seed)
+        qgx.qgx_sync_status(ctx)
+        _compare(st_t, st_o)
+    err = np.linalg.norm(st_t.Xbar.cpu().numpy() - xstar) / np.linalg.norm(xstar)
+    assert err < 1.0
+
+
+def test_diagonal_operator_scale_shape(q):
+    """c5 at reduced size: diagonal operator, mixture noise reused every iteration, bucket 16384."""
+    qgx, ctx = q
+    K, d = 4, 3 * 16384 + 4000
+    c5 = gen.c5_diagonal(K=K, d=d, device="cuda")
+    D, x0, noise = c5.D.cpu().numpy(), c5.x0.cpu().numpy(), c5.noise.cpu().numpy()
+    lev = gen.uniform_levels(17).numpy().copy()
+    cb = qgx.qgx_build_codebook_fixed(17, 128)
+    cfg = qgx.make_quant_cfg(lev, c5.bucket, cb, c5.seed, code_type=qgx.QGX_CODE_HUFFMAN)
+    op = qgx.make_operator(qgx.QGX_OP_DIAGONAL, c5.D)
+    opo = o.Op(o.OP_DIAGONAL, D)
+    st = qgx.EgState(c5.x0, K)
+    qgx.qgx_eg_init(ctx, st)
+    st_o = o.EgState(x0, K)
+    cbo = o.codebook_fixed(17, 128)
+    for t in range(1, 4):
+        refit = 2 if t == 1 else 0
+        _load_state(qgx, st, st_o)
+        qgx.qgx_eg_step(ctx, st, op, c5.noise[0], c5.noise[1], cfg, refit=refit)
+        if refit:
+            lev = np.array(cfg.level_list(), dtype=np.float32)
+            cbo = o.codebook_from(cfg.cb.lengths(), cfg.cb.codes(), subblock=128)
+        o.eg_step(st_o, opo, noise[0], noise[1], c5.bucket, lev, cbo, c5.seed)
+        qgx.qgx_sync_status(ctx)
+        _compare(st, st_o)

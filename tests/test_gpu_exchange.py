@@ -1,0 +1,118 @@
+"""Parity of the fused exchange (quantize+encode kernel, decode+average kernel) with the oracle
+and with the four separate calls, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import qgx_inputs as gen
+from oracle import qgx_oracle as o
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_2308_09187_b200 as qgx
+    ctx = qgx.qgx_create(0)
+    yield qgx, ctx
+    qgx.qgx_destroy(ctx)
+
+
+def _levels(rng, nlev, top=0.2):
+    inner = np.sort(rng.uniform(0.001, top, size=nlev - 2))
+    return np.r_[0.0, inner, 1.0].astype(np.float32)
+
+
+def _used_words(bbits):
+    return ((bbits.astype(np.int64) + 31) // 32).sum(axis=1)
+
+
+CASES = [
+    # K, d, bucket, nlev, subblock, huffman
+    (4, 2048, 512, 9, 128, False),        # c1 shape: 4 sub-blocks per bucket
+    (8, 3 * 8192 + 1000, 8192, 17, 128, True),   # c2 shape, ragged tail
+    (3, 2 * 16384 + 1728, 16384, 17, 128, True), # c5 bucket, short last bucket
+    (16, 1728, 4096, 9, 128, True),       # c3's smallest tensor: one partial bucket
+    (5, 40000, 4096, 17, 64, True),
+    (2, 70000, 2048, 32, 32, False),
+    (2, 1001, 256, 3, 32, True),          # d not a multiple of 4
+]
+
+
+@pytest.mark.parametrize("K,d,bucket,nlev,sub,huff", CASES)
+def test_fused_exchange_matches_oracle_and_steps(q, K, d, bucket, nlev, sub, huff):
+    qgx, ctx = q
+    rng = np.random.default_rng(K * 1000 + nlev)
+    v = gen.gaussian_mixture((K, d), seed=d + 1, device="cuda")
+    v[K - 1, : min(d, bucket)] = 0.0
+    vh = v.cpu().numpy()
+    lev = _levels(rng, nlev)
+    p = rng.dirichlet(np.ones(nlev) * 0.4)
+    cb = qgx.qgx_build_codebook_huffman(list(p), sub) if huff else qgx.qgx_build_codebook_fixed(nlev, sub)
+    cbo = o.codebook_from(cb.lengths(), cb.codes(), subblock=sub)
+    seed, xid = 1005, 41
+    cfg = qgx.make_quant_cfg(lev, bucket, cb, seed)
+    nb = o.nbuckets(d, bucket)
+
+    mean, total = qgx.qgx_exchange(ctx, v, cfg, xid, slot=0)
+    qgx.qgx_sync_status(ctx)
+    stream, bbits, tot2 = qgx.exchange_stream_tensors(ctx, 0, K, nb)
+    stream_h = stream.cpu().numpy().view(np.uint32)
+    bbits_h = bbits.cpu().numpy().view(np.uint32)
+
+    # the separate calls on the same input: same norms (same reduction), then the oracle on those norms
+    norms, sym = qgx.qgx_quantize(ctx, v, bucket, lev, qgx.QGX_NORM_L2, seed, xid)
+    qgx.qgx_sync_status(ctx)
+    n_gpu = norms.cpu().numpy()
+    assert np.all(np.abs(n_gpu - o.bucket_norms(vh, bucket)) <= np.spacing(n_gpu))
+    s_ref = o.quantize(vh, bucket, lev, n_gpu, seed, xid)
+    assert np.array_equal(sym.cpu().numpy(), s_ref)
+    st_ref, bb_ref, tot_ref = o.encode(n_gpu, s_ref, bucket, cbo)
+    assert np.array_equal(bbits_h, bb_ref)
+    assert np.array_equal(total.cpu().numpy().astype(np.uint64), tot_ref)
+    assert np.array_equal(tot2.cpu().numpy().astype(np.uint64), tot_ref)
+    used = _used_words(bb_ref)
+    for k in range(K):
+        assert np.array_equal(stream_h[k, :used[k]], st_ref[k, :used[k]])      # the compact stream, bit for bit
+    assert np.array_equal(mean.cpu().numpy(), o.average(n_gpu, s_ref, bucket, lev))
+    m_or, t_or = o.exchange(vh, bucket, lev, cbo, seed, xid)
+    flips = np.count_nonzero(o.quantize(vh, bucket, lev, o.bucket_norms(vh, bucket), seed, xid) != s_ref)
+    assert flips <= max(1, int(1e-6 * K * d))
+    if flips == 0 and np.array_equal(n_gpu, o.bucket_norms(vh, bucket)):
+        assert np.array_equal(mean.cpu().numpy(), m_or) and np.array_equal(t_or, tot_ref)
+    scale = float(n_gpu.max())
+    assert np.max(np.abs(mean.cpu().numpy() - m_or)) <= 1e-5 * scale
+
+
+def test_second_slot_and_repeatability(q):
+    qgx, ctx = q
+    K, d, bucket = 4, 50000, 4096
+    v = gen.gaussian((K, d), seed=9, device="cuda")
+    lev = np.linspace(0, 1, 17, dtype=np.float32) ** 2
+    cfg = qgx.make_quant_cfg(lev, bucket, qgx.qgx_build_codebook_fixed(17, 128), 77)
+    m0, t0 = qgx.qgx_exchange(ctx, v, cfg, 2, slot=0)
+    m1, t1 = qgx.qgx_exchange(ctx, v, cfg, 3, slot=1)
+    m2, t2 = qgx.qgx_exchange(ctx, v, cfg, 2, slot=1)
+    qgx.qgx_sync_status(ctx)
+    assert torch.equal(m0, m2) and torch.equal(t0, t2)          # same exchange id: same rounding
+    assert not torch.equal(m0, m1)                              # another exchange id: fresh randomness
+    # unbiased: the mean over workers of Q(v_k) is close to the mean of v_k
+    err = (m0 - v.mean(0)).abs().max().item()
+    assert err < 0.5 * v.abs().max().item()
+
+
+def test_fused_capacity_and_nonfinite(q):
+    qgx, ctx = q
+    K, d, bucket = 2, 9000, 1024
+    v = gen.gaussian((K, d), seed=3, device="cuda")
+    v[1, 5000] = float("inf")
+    lev = np.linspace(0, 1, 9, dtype=np.float32)
+    cfg = qgx.make_quant_cfg(lev, bucket, qgx.qgx_build_codebook_fixed(9, 128), 5)
+    qgx.qgx_exchange(ctx, v, cfg, 0, slot=0)
+    assert qgx.qgx_sync_status(ctx, check=False) == qgx.QGX_ERR_NONFINITE
+    v[1, 5000] = 1.0
+    qgx.qgx_exchange(ctx, v, cfg, 0, slot=0)
+    assert qgx.qgx_sync_status(ctx, check=False) == qgx.QGX_OK
+    bad = qgx.make_quant_cfg(lev, bucket, qgx.qgx_build_codebook_fixed(9, 96), 5)      # 96 is not a fused sub-block size
+    with pytest.raises(qgx.QgxError):
+        qgx.qgx_exchange(ctx, v, bad, 0, slot=0)

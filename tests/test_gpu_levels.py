@@ -1,0 +1,66 @@
+"""Parity of the histogram kernel and of qgx_update_levels with the oracle."""
+import numpy as np
+import pytest
+
+import qgx_inputs as gen
+from oracle import qgx_oracle as o
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_2308_09187_b200 as qgx
+    ctx = qgx.qgx_create(0)
+    yield qgx, ctx
+    qgx.qgx_destroy(ctx)
+
+
+@pytest.mark.parametrize("K,d,bucket,nbins", [(3, 5000, 1024, 64), (8, 3 * 8192 + 100, 8192, 1024), (2, 40000, 16384, 1024),
+                                              (4, 2048, 512, 256), (2, 1001, 256, 32)])
+def test_histogram(q, K, d, bucket, nbins):
+    qgx, ctx = q
+    v = gen.student_t3((K, d), seed=d, device="cuda")
+    vh = v.cpu().numpy()
+    hu = qgx.qgx_histogram(ctx, v, bucket, nbins, weighted=False)
+    hw = qgx.qgx_histogram(ctx, v, bucket, nbins, weighted=True)
+    qgx.qgx_sync_status(ctx)
+    n_ref = o.bucket_norms(vh, bucket)
+    ref_u = o.histogram(vh, bucket, nbins, weighted=False)
+    ref_w = o.histogram(vh, bucket, nbins, weighted=True)
+    assert hu.cpu().numpy().sum() == K * d
+    # integer counts agree except where a norm differs in its last bit (bin edges are fp32 products)
+    assert np.abs(hu.cpu().numpy() - ref_u).sum() <= max(2, 1e-6 * K * d)
+    assert np.allclose(hw.cpu().numpy(), ref_w, rtol=1e-6, atol=1e-9 * ref_w.sum())
+    hl = qgx.qgx_histogram(ctx, v, bucket, nbins, norm_type=qgx.QGX_NORM_LINF, weighted=False)
+    qgx.qgx_sync_status(ctx)
+    assert np.array_equal(hl.cpu().numpy(), o.histogram(vh, bucket, nbins, o.LINF, False))
+    assert n_ref.shape == (K, o.nbuckets(d, bucket))
+
+
+def test_update_levels_matches_oracle_refit(q):
+    qgx, ctx = q
+    K, d, bucket, nlev = 8, 4 * 8192, 8192, 17
+    v = gen.gaussian((K, d), seed=1002, device="cuda")
+    vh = v.cpu().numpy()
+    for code_type in (qgx.QGX_CODE_FIXED, qgx.QGX_CODE_HUFFMAN):
+        cfg = qgx.make_quant_cfg(np.linspace(0, 1, nlev), bucket, qgx.qgx_build_codebook_fixed(nlev, 128), 1,
+                                 code_type=code_type, nbins=1024)
+        hist = qgx.qgx_update_levels(ctx, v, cfg, qgx.QGX_REFIT_FIRST)
+        cbo = o.codebook_fixed(nlev, 128)
+        lev_ref, hist_ref = o.refit(vh, bucket, 1024, np.linspace(0, 1, nlev, dtype=np.float32), cbo, True, code_type)
+        assert np.allclose(hist, hist_ref, rtol=1e-6, atol=1e-9 * hist_ref.sum())
+        lev = np.array(cfg.level_list(), dtype=np.float32)
+        assert o.check_levels(lev) == o.OK
+        assert np.max(np.abs(lev - lev_ref)) < 5e-5
+        # the fitted table is as good as the oracle's on the oracle's objective
+        assert o.objective(hist_ref, lev) <= o.objective(hist_ref, lev_ref) * (1 + 1e-4) + 1e-12
+        # same expected code length under the symbol weights; the codes themselves may differ in ties
+        p = o.symbol_pmf(hist_ref, lev_ref)
+        assert abs(np.dot(p, cfg.cb.lengths()) - np.dot(p, cbo.lengths())) < 1e-3
+        assert cfg.cb.subblock == 128 and cfg.cb.nlev == nlev
+        # a second refit continues from the fitted table and keeps it (already converged)
+        qgx.qgx_update_levels(ctx, v, cfg, qgx.QGX_REFIT_CONTINUE)
+        lev2 = np.array(cfg.level_list(), dtype=np.float32)
+        lev_ref2, _ = o.refit(vh, bucket, 1024, lev_ref, cbo, False, code_type)
+        assert np.max(np.abs(lev2 - lev_ref2)) < 5e-5
