@@ -117,6 +117,18 @@ const char *qgx_status_str(qgx_status s);
 /* How many kernels of this library the context has launched so far. */
 uint64_t qgx_launch_count(const qgx_ctx *ctx);
 
+/* Per-kernel device timing for benchmarks (no counterpart in the paper).  qgx_timing_enable
+ * allocates `max_records` event pairs (0 switches timing off and frees them); while on, every
+ * launch of the kernels named below is bracketed by two events on the context's stream.
+ * qgx_timing_read synchronizes, returns the number of recorded launches of `kernel` and their
+ * summed duration in milliseconds, and forgets the records read so far of every kernel when
+ * `reset` is nonzero. */
+enum { QGX_KERNEL_ENCODE = 0, QGX_KERNEL_DECODE = 1, QGX_KERNEL_HISTOGRAM = 2, QGX_KERNEL_OPERATOR = 3,
+       QGX_KERNEL_FINISH = 4, QGX_KERNEL_COUNT = 5 };
+qgx_status qgx_timing_enable(qgx_ctx *ctx, int max_records);
+qgx_status qgx_timing_read(qgx_ctx *ctx, int kernel, int reset, int *launches /*[host] out*/,
+                           double *total_ms /*[host] out*/);
+
 /* ---- host helpers ------------------------------------------------------------------------- */
 
 /* QGX_OK iff the table is admissible for Definition 1. */

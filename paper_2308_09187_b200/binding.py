@@ -28,8 +28,9 @@ EXPORTS = [
     "qgx_build_codebook_huffman", "qgx_fit_levels", "qgx_symbol_pmf",
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
-    "qgx_eg_init", "qgx_eg_step", "qgx_apply_operator",
+    "qgx_eg_init", "qgx_eg_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
 ]
+QGX_KERNEL_ENCODE, QGX_KERNEL_DECODE, QGX_KERNEL_HISTOGRAM, QGX_KERNEL_OPERATOR, QGX_KERNEL_FINISH = range(5)
 
 
 class qgx_codebook(C.Structure):
@@ -155,6 +156,17 @@ def qgx_sync_status(ctx, check=True):
 
 def qgx_launch_count(ctx):
     return int(lib().qgx_launch_count(ctx.h))
+
+
+def qgx_timing_enable(ctx, max_records):
+    _chk(lib().qgx_timing_enable(ctx.h, int(max_records)), "qgx_timing_enable")
+
+
+def qgx_timing_read(ctx, kernel, reset=False):
+    """(launches, total milliseconds) of one instrumented kernel since the last reset."""
+    n, ms = C.c_int(0), C.c_double(0.0)
+    _chk(lib().qgx_timing_read(ctx.h, int(kernel), int(reset), C.byref(n), C.byref(ms)), "qgx_timing_read")
+    return n.value, ms.value
 
 
 # ---------------------------------------------------------------- host helpers

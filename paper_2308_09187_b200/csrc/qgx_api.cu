@@ -72,6 +72,15 @@ void* ws_get(qgx_ctx* c, int which, size_t bytes) {
 
 using namespace qgx;
 
+static void timing_free(qgx_ctx* c) {
+  for (int i = 0; i < 2 * c->timing_cap; ++i) cudaEventDestroy(c->timing_ev[i]);
+  delete[] c->timing_ev;
+  delete[] c->timing_kind;
+  c->timing_ev = nullptr;
+  c->timing_kind = nullptr;
+  c->timing_cap = c->timing_used = c->timing_on = 0;
+}
+
 extern "C" {
 
 qgx_status qgx_create(qgx_ctx** out, int device, void* cuda_stream) {
@@ -101,6 +110,7 @@ void qgx_destroy(qgx_ctx* c) {
   if (!c) return;
   cudaSetDevice(c->device);
   cudaStreamSynchronize(c->stream);
+  if (c->timing_ev) timing_free(c);
   for (int i = 0; i < 24; ++i)
     if (c->ws[i]) cudaFree(c->ws[i]);
   cudaFree(c->dstatus);
@@ -135,6 +145,41 @@ const char* qgx_status_str(qgx_status s) {
 }
 
 uint64_t qgx_launch_count(const qgx_ctx* c) { return c ? c->launches : 0; }
+
+qgx_status qgx_timing_enable(qgx_ctx* c, int max_records) {
+  if (!c || max_records < 0 || max_records > (1 << 20)) return QGX_ERR_INVALID_ARG;
+  if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
+  cudaStreamSynchronize(c->stream);
+  if (c->timing_ev) timing_free(c);
+  if (max_records == 0) return QGX_OK;
+  c->timing_ev = new (std::nothrow) cudaEvent_t[2 * (size_t)max_records];
+  c->timing_kind = new (std::nothrow) int[(size_t)max_records];
+  if (!c->timing_ev || !c->timing_kind) return QGX_ERR_CUDA;
+  for (int i = 0; i < 2 * max_records; ++i)
+    if (cudaEventCreate(&c->timing_ev[i]) != cudaSuccess) { c->timing_cap = i / 2; timing_free(c); return QGX_ERR_CUDA; }
+  c->timing_cap = max_records;
+  c->timing_used = 0;
+  c->timing_on = 1;
+  return QGX_OK;
+}
+
+qgx_status qgx_timing_read(qgx_ctx* c, int kernel, int reset, int* launches, double* total_ms) {
+  if (!c || !launches || !total_ms || kernel < 0 || kernel >= QGX_KERNEL_COUNT) return QGX_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return QGX_ERR_CUDA;
+  int n = 0;
+  double ms = 0.0;
+  for (int i = 0; i < c->timing_used; ++i) {
+    if (c->timing_kind[i] != kernel) continue;
+    float t = 0.0f;
+    if (cudaEventElapsedTime(&t, c->timing_ev[2 * i], c->timing_ev[2 * i + 1]) != cudaSuccess) return QGX_ERR_CUDA;
+    ms += (double)t;
+    ++n;
+  }
+  *launches = n;
+  *total_ms = ms;
+  if (reset) c->timing_used = 0;
+  return QGX_OK;
+}
 
 qgx_status qgx_check_levels(const float* levels, int nlev) { return check_levels_host(levels, nlev); }
 

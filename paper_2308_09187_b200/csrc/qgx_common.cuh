@@ -35,6 +35,12 @@ struct qgx_ctx {
   size_t slot_cap_words[2];
   int slot_K[2];
   size_t slot_nb[2];
+  // optional per-kernel timing: pairs of events recorded around instrumented launches
+  int timing_on;
+  int timing_cap;                        // pairs allocated
+  int timing_used;
+  cudaEvent_t* timing_ev;                // 2 * timing_cap events
+  int* timing_kind;                      // kernel id of each pair
 };
 
 namespace qgx {
@@ -155,5 +161,21 @@ qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out);
 void* ws_get(qgx_ctx* c, int which, size_t bytes);          // nullptr on failure
 qgx_status cuda_status(cudaError_t e);
 inline void count_launch(qgx_ctx* c, int n = 1) { c->launches += (uint64_t)n; }
+
+// Brackets an instrumented kernel launch with two events when timing is on (qgx_timing_enable).
+struct ScopedKernelTimer {
+  qgx_ctx* c;
+  int slot;
+  ScopedKernelTimer(qgx_ctx* ctx, int kind) : c(ctx), slot(-1) {
+    if (c->timing_on && c->timing_used < c->timing_cap) {
+      slot = c->timing_used++;
+      c->timing_kind[slot] = kind;
+      cudaEventRecord(c->timing_ev[2 * slot], c->stream);
+    }
+  }
+  ~ScopedKernelTimer() {
+    if (slot >= 0) cudaEventRecord(c->timing_ev[2 * slot + 1], c->stream);
+  }
+};
 
 }  // namespace qgx

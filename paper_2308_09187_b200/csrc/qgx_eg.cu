@@ -98,6 +98,7 @@ static unsigned grid_for(size_t n, int threads) {
 qgx_status apply_operator_impl(qgx_ctx* c, const qgx_operator* op, const float* x, float* out) {
   if (!c || !op || !x || !out || !op->mat || op->d < 1) return QGX_ERR_INVALID_ARG;
   const size_t d = op->d;
+  ScopedKernelTimer timer(c, QGX_KERNEL_OPERATOR);
   if (op->kind == QGX_OP_DENSE_AFFINE) {
     const bool vec_ok = (d % 4 == 0) && ((reinterpret_cast<uintptr_t>(op->mat) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(x) & 15u) == 0);
     k_gemv_rows<<<grid_for(d * 32, 256), 256, 0, c->stream>>>(op->mat, d, d, x, op->bias, out, vec_ok);
@@ -170,7 +171,10 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
   ExchangeUpdate dual{2, st->Y, st->Y, st->scalars};                          // Y_{t+1} = Y_t - mean
   rc = exchange_impl(c, src2, K, d, cfg, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 0, st->scalars);
   if (rc != QGX_OK) return rc;
-  k_eg_finish<<<grid_for(d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->Xhalf, st->anchor, st->scalars, d, K, st->t);
+  {
+    ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);
+    k_eg_finish<<<grid_for(d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->Xhalf, st->anchor, st->scalars, d, K, st->t);
+  }
   count_launch(c);
   st->t += 1;
   return cuda_status(cudaGetLastError());

@@ -457,11 +457,14 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
     const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);   \
     k_exchange_encode<V><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key);                                  \
   } while (0)
-  switch (v4) {
-    case 1: QGX_LAUNCH_E(1); break;
-    case 2: QGX_LAUNCH_E(2); break;
-    case 4: QGX_LAUNCH_E(4); break;
-    default: QGX_LAUNCH_E(8); break;
+  {
+    ScopedKernelTimer timer(c, QGX_KERNEL_ENCODE);
+    switch (v4) {
+      case 1: QGX_LAUNCH_E(1); break;
+      case 2: QGX_LAUNCH_E(2); break;
+      case 4: QGX_LAUNCH_E(4); break;
+      default: QGX_LAUNCH_E(8); break;
+    }
   }
 #undef QGX_LAUNCH_E
   count_launch(c);
@@ -504,8 +507,11 @@ static void launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const LevelTable& 
   if (per_sm < 1) per_sm = 1;
   const size_t want = (total_sub + threads - 1) / threads;
   const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
-  if (diff) k_exchange_decode<G, true><<<grid, threads, smem, c->stream>>>(da, lt, ct);
-  else k_exchange_decode<G, false><<<grid, threads, smem, c->stream>>>(da, lt, ct);
+  {
+    ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
+    if (diff) k_exchange_decode<G, true><<<grid, threads, smem, c->stream>>>(da, lt, ct);
+    else k_exchange_decode<G, false><<<grid, threads, smem, c->stream>>>(da, lt, ct);
+  }
   count_launch(c);
 }
 

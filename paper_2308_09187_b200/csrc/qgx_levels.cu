@@ -65,6 +65,7 @@ qgx_status launch_histogram(qgx_ctx* c, DualSource src, int K, size_t d, int buc
   const int threads = bucket_threads(bucket, v4);
   const dim3 grid((unsigned)nb, (unsigned)K);
   const size_t smem = sizeof(uint32_t) * (size_t)nbins;
+  ScopedKernelTimer timer(c, QGX_KERNEL_HISTOGRAM);
   switch (v4) {
     case 1: k_histogram<1><<<grid, threads, smem, c->stream>>>(src, d, bucket, norm_type, nbins, weighted, vec_ok, hist, c->dstatus); break;
     case 2: k_histogram<2><<<grid, threads, smem, c->stream>>>(src, d, bucket, norm_type, nbins, weighted, vec_ok, hist, c->dstatus); break;
