@@ -52,6 +52,41 @@ qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out) {
   return QGX_OK;
 }
 
+// tau(u) by definition: the largest j <= nlev - 2 with l_j <= u
+static int tau_of(const float* lev, int nlev, float u) {
+  int tau = 0;
+  for (int j = 1; j <= nlev - 2; ++j)
+    if (lev[j] <= u) tau = j;
+  return tau;
+}
+
+void make_quant_table(const float* lev, int nlev, QuantTable* out) {
+  std::memset(out, 0, sizeof(*out));
+  out->nlev = nlev;
+  for (int j = 0; j < 2 * QGX_MAX_LEVELS; ++j) out->upper[j] = (j <= nlev - 2) ? lev[j] : 3.0f;
+  for (int t = 0; t <= nlev - 2; ++t) {
+    const float width = lev[t + 1] - lev[t];                       // the fp32 difference the exact routine divides by
+    const double scale = 8388608.0 / (double)width;
+    const float margin = (float)(4.0 * (double)lev[t + 1] / (double)width + 8.0) * 1.0001f;
+    out->interval[t] = make_float4(lev[t], (float)scale, margin, 8388608.0f - margin);
+  }
+  for (int t = nlev - 1; t < QGX_MAX_LEVELS; ++t) out->interval[t] = make_float4(0.f, 0.f, 3.0e38f, -3.0e38f);   // never "safe"
+  int steps = 0;
+  for (int b = 0; b < kKeyBins; ++b) {
+    // bin b holds patterns [(b + kKeyMin) << 17, (b + 1 + kKeyMin) << 17); bin 0 also everything below
+    uint32_t lo_bits = (uint32_t)(b + kKeyMin) << kKeyShift, hi_bits = ((uint32_t)(b + 1 + kKeyMin) << kKeyShift) - 1u;
+    float lo, hi;
+    std::memcpy(&lo, &lo_bits, 4);
+    std::memcpy(&hi, &hi_bits, 4);
+    if (b == 0) lo = 0.0f;
+    if (hi > 1.0f) hi = 1.0f;
+    const int t_lo = tau_of(lev, nlev, lo), t_hi = tau_of(lev, nlev, hi);
+    out->start[b] = (uint8_t)t_lo;
+    steps = std::max(steps, t_hi - t_lo);
+  }
+  out->steps = steps;
+}
+
 void* ws_get(qgx_ctx* c, int which, size_t bytes) {
   if (bytes == 0) bytes = 16;
   if (c->ws_bytes[which] >= bytes) return c->ws[which];

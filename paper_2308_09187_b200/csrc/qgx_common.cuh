@@ -51,6 +51,20 @@ struct LevelTable {
   float lev[QGX_MAX_LEVELS];
 };
 
+// Tables of the fast rounding path (see quantize_fast): a 1025-entry map from the top bits of the
+// float pattern of u to a lower bound of tau(u), and per interval the level, 2^23 / width, the
+// rounding margin and 2^23 - margin.
+constexpr int kKeyShift = 17;                       // 64 bins per octave of u
+constexpr int kKeyMin = 0x37800000 >> kKeyShift;    // pattern of 2^-16: everything below shares bin 0
+constexpr int kKeyBins = (0x3F800000 >> kKeyShift) - kKeyMin + 1;   // up to u = 1.0: 1025 bins
+struct QuantTable {
+  int nlev;
+  int steps;                             // compare steps after the table look-up
+  float4 interval[QGX_MAX_LEVELS];       // {l_tau, 2^23 / (l_{tau+1} - l_tau), margin, 2^23 - margin}
+  float upper[2 * QGX_MAX_LEVELS];       // upper[j] = l_j for j <= nlev - 2, then a value above 1
+  uint8_t start[kKeyBins + 3];
+};
+
 struct CodeTable {
   int nlev;
   int maxlen;
@@ -117,6 +131,33 @@ __device__ __forceinline__ int quantize_level(float absv, float norm, const floa
   return tau + ((r < xi) ? 1 : 0);
 }
 
+// Same decision as quantize_level, without divisions in the common case.  With rn = RN(1/norm),
+// u' = RN(|v| rn) differs from the exact u = RN(|v| / norm) by at most 2^-22 u.  tau is found from a
+// table on the float pattern of u' plus `steps` comparisons; T = (u' - l_tau) 2^23 / width differs
+// from xi 2^23 by less than margin = 4 l_{tau+1} / width + 8.  The 24-bit variate m rounds up iff
+// m < xi 2^24; with m' = m >> 1 taken as a float through the 2^23 trick, the sign of T - m' decides
+// whenever |T - m'| > margin and T is further than margin from both ends of the interval (so that
+// u' and u lie in the same interval).  Otherwise (about 1e-5 of coordinates) the exact routine runs.
+__device__ __forceinline__ int quantize_fast(float absv, float rn, float norm, const QuantTable* q, int steps,
+                                             const float* lev, int nlev, uint32_t word) {
+  const float u = fminf(__fmul_rn(absv, rn), 1.0f);
+  const int key = max((int)(__float_as_uint(u) >> kKeyShift), kKeyMin) - kKeyMin;
+  const int tau0 = q->start[key];
+  int tau = tau0;
+  for (int i = 1; i <= steps; ++i) tau += (q->upper[tau0 + i] <= u) ? 1 : 0;
+  const float4 iv = q->interval[tau];
+  const float T = __fmul_rn(__fsub_rn(u, iv.x), iv.y);
+  const float mhalf = __fsub_rn(__uint_as_float(0x4B000000u | (word >> 9)), 8388608.0f);   // (m >> 1), exact
+  const float diff = __fsub_rn(T, mhalf);
+  if (fabsf(diff) > iv.z && T > iv.z && T < iv.w) return tau + (diff > 0.0f ? 1 : 0);
+  return quantize_level(absv, norm, lev, nlev, word);
+}
+
+// reciprocal of a bucket norm for quantize_fast; 0 sends every coordinate to the exact routine
+__device__ __forceinline__ float fast_reciprocal(float norm) {
+  return (norm > 7.9e-31f && norm < 1.2e30f) ? __frcp_rn(norm) : 0.0f;
+}
+
 __device__ __forceinline__ uint32_t symbol_of(float v, int idx) {
   const uint32_t neg = (__float_as_uint(v) >> 31) & (idx != 0 ? 1u : 0u);
   return (uint32_t)idx | (neg << 7);
@@ -158,6 +199,7 @@ struct ExchangeUpdate {
 // host side
 qgx_status check_levels_host(const float* lev, int nlev);
 qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out);
+void make_quant_table(const float* lev, int nlev, QuantTable* out);
 void* ws_get(qgx_ctx* c, int which, size_t bytes);          // nullptr on failure
 qgx_status cuda_status(cudaError_t e);
 inline void count_launch(qgx_ctx* c, int n = 1) { c->launches += (uint64_t)n; }

@@ -77,32 +77,78 @@ struct EncodeArgs {
   DevStatus* st;
 };
 
+// Norm of the bucket held by the CTA, one barrier: per-warp partials go to shared memory and every
+// warp then reduces them in the same order (so all warps hold the same value).
 template <int V4>
-__global__ void __launch_bounds__(512) k_exchange_encode(EncodeArgs a, LevelTable lt, CodeTable ct, PhiloxKey key) {
-  extern __shared__ uint32_t s_dyn[];
+__device__ __forceinline__ float bucket_norm_all(const BucketRegs<V4>& r, int norm_type, double* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  double acc = 0.0;
+  if (norm_type == QGX_NORM_L2) {
+#pragma unroll
+    for (int j = 0; j < V4; ++j) {
+      const double a = r.x[j].x, b = r.x[j].y, c = r.x[j].z, e = r.x[j].w;
+      acc = fma(a, a, acc); acc = fma(b, b, acc); acc = fma(c, c, acc); acc = fma(e, e, acc);
+    }
+    acc = warp_sum(acc);
+  } else {
+    float m = 0.0f;
+    bool bad = false;
+#pragma unroll
+    for (int j = 0; j < V4; ++j) {
+      const float4 x = r.x[j];
+      bad = bad || (x.x != x.x) || (x.y != x.y) || (x.z != x.z) || (x.w != x.w);
+      m = fmaxf(m, fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w))));
+    }
+    m = warp_max(m);
+    acc = __any_sync(0xffffffffu, bad) ? (double)__int_as_float(0x7fc00000) : (double)m;
+  }
+  if (lane == 0) red[warp] = acc;
+  __syncthreads();
+  double t = lane < nwarps ? red[lane] : 0.0;
+  if (norm_type == QGX_NORM_L2) return (float)sqrt(warp_sum(t));
+  const bool bad = __any_sync(0xffffffffu, t != t);
+  const float m = warp_max((float)t);
+  return bad ? __int_as_float(0x7fc00000) : m;
+}
+
+// One persistent CTA per SM slot; each ticket is one bucket (k = ticket % K, b = ticket / K).
+//   load + zero image | barrier | norm, quantize, pack, header fields, warp scans | barrier |
+//   chunk prefixes, bit scatter, look-back (warp 0) | barrier | copy out | barrier
+template <int V4, int G>
+__global__ void __launch_bounds__(V4 == 8 ? 512 : (V4 == 4 ? 512 : 256), V4 == 8 ? 2 : 1)
+k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
+                  const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
+                  const __grid_constant__ QuantTable qt) {
+  extern __shared__ uint32_t s_img[];
+  __shared__ QuantTable s_q;
   __shared__ EncLut s_lut;
   __shared__ float s_lev[QGX_MAX_LEVELS];
-  __shared__ double s_red[34];
-  __shared__ uint32_t s_chunk[264];
-  __shared__ unsigned int s_ticket;
+  __shared__ double s_red[2][32];
+  __shared__ uint32_t s_chunk[2][8 * 16];
+  __shared__ unsigned int s_ticket[2];
   __shared__ unsigned long long s_prefix;
   __shared__ int s_skip;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  const int img_words = (int)((((uint32_t)a.bucket * (uint32_t)(ct.maxlen + 1) + 16u * (uint32_t)(a.bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4);
-  uint32_t* s_img = s_dyn;
-  uint32_t* s_sub = s_dyn + img_words;
-  const int qps = ct.G / kQuad;
+  const int img_words = (int)((((uint32_t)a.bucket * (uint32_t)(ct.maxlen + 1) + 16u * (uint32_t)(a.bucket / G + 1) + kNormBits + 31u) >> 5) + 4);
   const unsigned long long total = (unsigned long long)a.nb * (unsigned long long)a.K;
+  constexpr int kSegLanes = G / kQuad;                  // lanes per sub-block within a warp's 128 coordinates
+  constexpr int kSegs = 32 / kSegLanes;                 // sub-blocks per chunk
 
   fill_enc_lut(&s_lut, ct);
+  {
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(&qt);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(&s_q);
+    for (int i = threadIdx.x; i < (int)(sizeof(QuantTable) / 4); i += blockDim.x) dst[i] = src[i];
+  }
   if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 1.0f;
+  if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
+  __syncthreads();
+  const int steps = s_q.steps;
+  const int nlev = lt.nlev;
 
-  for (;;) {
-    __syncthreads();                                    // shared state of the previous bucket is no longer read
-    if (threadIdx.x == 0) s_ticket = atomicAdd(a.ticket, 1u);
-    __syncthreads();
-    const unsigned long long t = s_ticket;
+  for (int par = 0;; par ^= 1) {
+    const unsigned long long t = s_ticket[par];
     if (t >= total) break;
     const size_t b = (size_t)(t / (unsigned long long)a.K), k = (size_t)(t % (unsigned long long)a.K);
     const size_t lo = b * (size_t)a.bucket;
@@ -110,12 +156,17 @@ __global__ void __launch_bounds__(512) k_exchange_encode(EncodeArgs a, LevelTabl
 
     BucketRegs<V4> r;
     load_bucket<V4>(r, a.src, k, a.d, lo, len, a.vec_ok);
-    const float norm = bucket_norm<V4>(r, a.norm_type, s_red);
+    for (int i = threadIdx.x; i < img_words; i += blockDim.x) s_img[i] = 0;
+    const float norm = bucket_norm_all<V4>(r, a.norm_type, s_red[par]);      // barrier inside: the image is zero
     const bool finite = (norm - norm) == 0.0f;
+    const float rn = fast_reciprocal(norm);
     if (threadIdx.x == 0) {
       a.norms[k * a.nb + b] = norm;
       if (!finite) latch_error(a.st, QGX_ERR_NONFINITE);
+      s_img[0] = __float_as_uint(norm);
     }
+    const uint32_t nsub = (uint32_t)((len + G - 1) / G);
+    const uint32_t hdr_bits = kNormBits + 16u * nsub;
 
     uint64_t qbits[V4];
     uint32_t qn[V4], qexcl[V4];
@@ -123,60 +174,69 @@ __global__ void __launch_bounds__(512) k_exchange_encode(EncodeArgs a, LevelTabl
     for (int j = 0; j < V4; ++j) {
       const int q = j * (int)blockDim.x + (int)threadIdx.x;
       const int nvalid = max(0, min(kQuad, len - q * kQuad));
-      uint32_t packed = 0;
+      uint64_t acc = 0;
+      uint32_t n = 0;
       if (nvalid > 0 && finite) {
         const uint64_t ctr = (uint64_t)(lo >> 2) + (uint64_t)q;
         const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
-        const float4 x = r.x[j];
-        const uint32_t s0 = symbol_of(x.x, quantize_level(fabsf(x.x), norm, s_lev, lt.nlev, w.x));
-        const uint32_t s1 = symbol_of(x.y, quantize_level(fabsf(x.y), norm, s_lev, lt.nlev, w.y));
-        const uint32_t s2 = symbol_of(x.z, quantize_level(fabsf(x.z), norm, s_lev, lt.nlev, w.z));
-        const uint32_t s3 = symbol_of(x.w, quantize_level(fabsf(x.w), norm, s_lev, lt.nlev, w.w));
-        packed = s0 | (s1 << 8) | (s2 << 16) | (s3 << 24);
+        const float xs[kQuad] = {r.x[j].x, r.x[j].y, r.x[j].z, r.x[j].w};
+        const uint32_t ws[kQuad] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int c = 0; c < kQuad; ++c) {
+          if (c < nvalid) {
+            const int idx = quantize_fast(fabsf(xs[c]), rn, norm, &s_q, steps, s_lev, nlev, ws[c]);
+            const uint32_t e = s_lut.e[(uint32_t)idx | ((__float_as_uint(xs[c]) >> 31) << 5)];
+            acc |= (uint64_t)(e & 0xffffu) << n;
+            n += e >> 16;
+          }
+        }
+      } else if (nvalid > 0) {
+        const uint32_t e = s_lut.e[0];                   // non-finite norm: every coordinate is sent as level 0
+        for (int c = 0; c < nvalid; ++c) { acc |= (uint64_t)(e & 0xffffu) << n; n += e >> 16; }
       }
-      pack_quad(packed, nvalid, &s_lut, &qbits[j], &qn[j]);
-      const uint32_t incl = warp_incl_scan(qn[j], lane);
-      qexcl[j] = incl - qn[j];
-      if (lane == 31) s_chunk[j * nwarps + warp] = incl;
+      qbits[j] = acc;
+      qn[j] = n;
+      const uint32_t incl = warp_incl_scan(n, lane);
+      qexcl[j] = incl - n;
+      // sub-block lengths: the last lane of each sub-block knows its total
+      const uint32_t before = __shfl_up_sync(0xffffffffu, incl, kSegLanes);
+      if ((lane + 1) % kSegLanes == 0) {
+        const int sb = (j * nwarps + warp) * kSegs + lane / kSegLanes;
+        if (sb * G < len) {
+          const uint32_t L = incl - (lane >= kSegLanes ? before : 0u);
+          put_bits(s_img, kNormBits + 16u * (uint32_t)sb, (uint64_t)(L & 0xffffu), 16u);
+        }
+      }
+      if (lane == 31) s_chunk[par][j * nwarps + warp] = incl;
     }
     __syncthreads();
-    const int nchunks = V4 * nwarps;
-    if (warp == 0) {
-      uint32_t carry = 0;
-      for (int base = 0; base < nchunks; base += 32) {
-        const int i = base + lane;
-        const uint32_t x = i < nchunks ? s_chunk[i] : 0u;
-        const uint32_t incl = warp_incl_scan(x, lane);
-        if (i < nchunks) s_chunk[i] = carry + incl - x;
-        carry += __shfl_sync(0xffffffffu, incl, 31);
-      }
-      if (lane == 0) s_chunk[nchunks] = carry;
+    // exclusive prefix of the chunk totals, computed by every warp for itself
+    const int nchunks = V4 * nwarps;                     // <= 128
+    uint32_t pre[4];
+    uint32_t carry = 0;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const int i = g * 32 + lane;
+      const uint32_t x = i < nchunks ? s_chunk[par][i] : 0u;
+      const uint32_t incl = warp_incl_scan(x, lane);
+      pre[g] = carry + incl - x;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
     }
-    __syncthreads();
-    const uint32_t nsub = ct.has_header ? (uint32_t)((len + ct.G - 1) / ct.G) : 0u;
-    const uint32_t hdr_bits = kNormBits + 16u * nsub;
-    const uint32_t nbits = hdr_bits + s_chunk[nchunks];
+    const uint32_t nbits = hdr_bits + carry;
     const uint32_t nwords = (nbits + 31) >> 5;
     unsigned long long* row = a.status + k * a.nb;
     if (threadIdx.x == 0) {
-      st_status(row + b, kStAggregate | (unsigned long long)nwords);   // publish the length as early as possible
+      st_status(row + b, kStAggregate | (unsigned long long)nwords);
       a.bucket_bits[k * a.nb + b] = nbits;
       atomicAdd(a.total_bits + k, (unsigned long long)nbits);
     }
-    for (uint32_t i = threadIdx.x; i < nwords + 2; i += blockDim.x) s_img[i] = 0;
-    __syncthreads();
 #pragma unroll
     for (int j = 0; j < V4; ++j) {
-      const int q = j * (int)blockDim.x + (int)threadIdx.x;
-      const uint32_t p = s_chunk[j * nwarps + warp] + qexcl[j];
-      if (nsub && q * kQuad < len && q % qps == 0) s_sub[q / qps] = p;
+      const int c = j * nwarps + warp;
+      const uint32_t sel = (c >> 5) == 0 ? pre[0] : ((c >> 5) == 1 ? pre[1] : ((c >> 5) == 2 ? pre[2] : pre[3]));
+      const uint32_t p = __shfl_sync(0xffffffffu, sel, c & 31) + qexcl[j];
       put_bits(s_img, hdr_bits + p, qbits[j], qn[j]);
     }
-    if (threadIdx.x == 0) {
-      atomicOr(&s_img[0], __float_as_uint(norm));
-      if (nsub) s_sub[nsub] = s_chunk[nchunks];
-    }
-    // meanwhile warp 0 finds where the bucket goes
     if (warp == 0) {
       bool timed_out = false;
       const unsigned long long excl = lookback_prefix(row, (long long)b, lane, &timed_out);
@@ -188,18 +248,15 @@ __global__ void __launch_bounds__(512) k_exchange_encode(EncodeArgs a, LevelTabl
         a.offsets[k * a.nb + b] = (uint32_t)min(excl, (unsigned long long)0xffffffffu);
         s_prefix = excl;
         s_skip = skip;
+        s_ticket[par ^ 1] = atomicAdd(a.ticket, 1u);
       }
-    }
-    __syncthreads();
-    for (uint32_t s = threadIdx.x; s < nsub; s += blockDim.x) {
-      const uint32_t L = s_sub[s + 1] - s_sub[s];
-      put_bits(s_img, kNormBits + 16u * s, (uint64_t)(L & 0xffffu), 16u);
     }
     __syncthreads();
     if (!s_skip) {
       uint32_t* dst = a.stream + k * a.cap_words + s_prefix;
       for (uint32_t i = threadIdx.x; i < nwords; i += blockDim.x) dst[i] = s_img[i];
     }
+    __syncthreads();
   }
 }
 
@@ -443,29 +500,39 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   ea.stream = stream; ea.cap_words = cap; ea.bucket_bits = bbits; ea.offsets = offs; ea.total_bits = tot; ea.norms = norms;
   ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(status + (size_t)K * nb); ea.st = c->dstatus;
   const PhiloxKey key = make_philox_key(cfg->seed);
+  QuantTable qt;
+  make_quant_table(cfg->levels, cfg->nlev, &qt);
+  if (!ct.has_header || bucket % ct.G != 0 || (ct.G != 32 && ct.G != 64 && ct.G != 128)) return QGX_ERR_INVALID_ARG;
   const int v4 = bucket_v4(bucket);
   const int threads = bucket_threads(bucket, v4);
   const size_t img_words = (((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4;
-  const size_t smem = sizeof(uint32_t) * (img_words + (size_t)(bucket / ct.G) + 2);
+  const size_t smem = sizeof(uint32_t) * img_words;
   int per_sm = 1;
-#define QGX_LAUNCH_E(V)                                                                                        \
+#define QGX_LAUNCH_E(V, GG)                                                                                    \
   do {                                                                                                         \
-    cudaFuncSetAttribute(k_exchange_encode<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V>, threads, smem);               \
+    cudaFuncSetAttribute(k_exchange_encode<V, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG>, threads, smem);           \
     if (per_sm < 1) per_sm = 1;                                                                                \
     const unsigned long long want = (unsigned long long)nb * (unsigned long long)K;                            \
     const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);   \
-    k_exchange_encode<V><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key);                                  \
+    k_exchange_encode<V, GG><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                          \
+  } while (0)
+#define QGX_LAUNCH_EG(V)                                   \
+  do {                                                     \
+    if (ct.G == 32) QGX_LAUNCH_E(V, 32);                   \
+    else if (ct.G == 64) QGX_LAUNCH_E(V, 64);              \
+    else QGX_LAUNCH_E(V, 128);                             \
   } while (0)
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_ENCODE);
     switch (v4) {
-      case 1: QGX_LAUNCH_E(1); break;
-      case 2: QGX_LAUNCH_E(2); break;
-      case 4: QGX_LAUNCH_E(4); break;
-      default: QGX_LAUNCH_E(8); break;
+      case 1: QGX_LAUNCH_EG(1); break;
+      case 2: QGX_LAUNCH_EG(2); break;
+      case 4: QGX_LAUNCH_EG(4); break;
+      default: QGX_LAUNCH_EG(8); break;
     }
   }
+#undef QGX_LAUNCH_EG
 #undef QGX_LAUNCH_E
   count_launch(c);
   if (cudaGetLastError() != cudaSuccess) return QGX_ERR_CUDA;

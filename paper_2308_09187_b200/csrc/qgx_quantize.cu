@@ -6,10 +6,17 @@ namespace qgx {
 // One CTA per (bucket, worker).  The bucket stays in registers between the norm reduction and
 // the rounding pass, so v is read from HBM exactly once.
 template <int V4>
-__global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int bucket, LevelTable lt, PhiloxKey key,
+__global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int bucket, const __grid_constant__ LevelTable lt,
+                                                   const __grid_constant__ PhiloxKey key, const __grid_constant__ QuantTable qt,
                                                    uint32_t xid, int norm_type, int norms_supplied, bool vec_ok,
                                                    float* __restrict__ norms, uint8_t* __restrict__ sym, DevStatus* st) {
   __shared__ float s_lev[QGX_MAX_LEVELS];
+  __shared__ QuantTable s_q;
+  {
+    const uint32_t* qsrc = reinterpret_cast<const uint32_t*>(&qt);
+    uint32_t* qdst = reinterpret_cast<uint32_t*>(&s_q);
+    for (int i = threadIdx.x; i < (int)(sizeof(QuantTable) / 4); i += blockDim.x) qdst[i] = qsrc[i];
+  }
   __shared__ double s_red[34];
   const size_t b = blockIdx.x, k = blockIdx.y;
   const size_t nb = gridDim.x;
@@ -29,6 +36,8 @@ __global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int 
   }
   const bool finite = (norm - norm) == 0.0f;
   if (!finite && threadIdx.x == 0) latch_error(st, QGX_ERR_NONFINITE);
+  const float rn = fast_reciprocal(norm);
+  const int steps = s_q.steps;
 
   uint8_t* out = sym + k * d + lo;
   const bool sym_vec = vec_ok;            // d % 4 == 0 and bucket % 4 == 0: every quad is 4-byte aligned
@@ -42,10 +51,10 @@ __global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int 
       const uint64_t ctr = (uint64_t)(lo >> 2) + (uint64_t)q;      // (coordinate index) / 4
       const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, xid, key);
       const float4 x = r.x[j];
-      const uint32_t s0 = symbol_of(x.x, quantize_level(fabsf(x.x), norm, s_lev, lt.nlev, w.x));
-      const uint32_t s1 = symbol_of(x.y, quantize_level(fabsf(x.y), norm, s_lev, lt.nlev, w.y));
-      const uint32_t s2 = symbol_of(x.z, quantize_level(fabsf(x.z), norm, s_lev, lt.nlev, w.z));
-      const uint32_t s3 = symbol_of(x.w, quantize_level(fabsf(x.w), norm, s_lev, lt.nlev, w.w));
+      const uint32_t s0 = symbol_of(x.x, quantize_fast(fabsf(x.x), rn, norm, &s_q, steps, s_lev, lt.nlev, w.x));
+      const uint32_t s1 = symbol_of(x.y, quantize_fast(fabsf(x.y), rn, norm, &s_q, steps, s_lev, lt.nlev, w.y));
+      const uint32_t s2 = symbol_of(x.z, quantize_fast(fabsf(x.z), rn, norm, &s_q, steps, s_lev, lt.nlev, w.z));
+      const uint32_t s3 = symbol_of(x.w, quantize_fast(fabsf(x.w), rn, norm, &s_q, steps, s_lev, lt.nlev, w.w));
       packed = s0 | (s1 << 8) | (s2 << 16) | (s3 << 24);
     }
     if (e + kQuad <= len && sym_vec) {
@@ -105,11 +114,13 @@ qgx_status launch_quantize(qgx_ctx* c, DualSource src, int K, size_t d, int buck
   const bool vec_ok = (d % kQuad == 0) && all_aligned16({src.v, src.a}) &&
                       ((reinterpret_cast<uintptr_t>(sym) & 3u) == 0);
   const PhiloxKey key = make_philox_key(seed);
+  QuantTable qt;
+  make_quant_table(lt.lev, lt.nlev, &qt);
   const int v4 = bucket_v4(bucket);
   const dim3 grid((unsigned)nb, (unsigned)K);
   const int threads = bucket_threads(bucket, v4);
 #define QGX_LAUNCH_Q(V)                                                                                      \
-  k_quantize<V><<<grid, threads, 0, c->stream>>>(src, d, bucket, lt, key, xid, norm_type, norms_supplied,   \
+  k_quantize<V><<<grid, threads, 0, c->stream>>>(src, d, bucket, lt, key, qt, xid, norm_type, norms_supplied, \
                                                  vec_ok, norms, sym, c->dstatus)
   switch (v4) {
     case 1: QGX_LAUNCH_Q(1); break;
