@@ -43,6 +43,29 @@ __device__ __forceinline__ void pack_quad(uint32_t packed_syms, int nvalid, cons
   *nbits = n;
 }
 
+// Pair table: the stream bits of two consecutive symbols in one entry, bits | nbits << 26, indexed by
+// the two 6-bit symbol codes (level | sign << 5) as first | second << 6.
+constexpr int kPairLutSize = 64 * 64;
+__device__ __forceinline__ void fill_pair_lut(uint32_t* pair, const EncLut* lut) {
+  for (int i = threadIdx.x; i < kPairLutSize; i += blockDim.x) {
+    const uint32_t a = lut->e[i & 63], b = lut->e[i >> 6];
+    const uint32_t na = a >> 16, nb = b >> 16;
+    pair[i] = ((a & 0xffffu) | ((b & 0xffffu) << na)) | ((na + nb) << 26);
+  }
+}
+
+// stream bits of a full quad of symbols (bytes: level | sign << 7) through the pair table
+__device__ __forceinline__ void pack_quad_pairs(uint32_t sym4, const uint32_t* pair, uint64_t* bits, uint32_t* nbits) {
+  const uint32_t t = (sym4 & 0x1f1f1f1fu) | ((sym4 >> 2) & 0x20202020u);        // 6-bit code in every byte
+  const uint32_t e01 = pair[(t & 0x3fu) | ((t >> 2) & 0xfc0u)];
+  const uint32_t e23 = pair[((t >> 16) & 0x3fu) | ((t >> 18) & 0xfc0u)];
+  const uint32_t b01 = e01 & 0x3ffffffu, n01 = e01 >> 26, b23 = e23 & 0x3ffffffu, n23 = e23 >> 26;
+  const uint32_t lo = b01 | (b23 << n01);
+  const uint32_t hi = __funnelshift_l(b23, 0u, n01);
+  *bits = ((uint64_t)hi << 32) | lo;
+  *nbits = n01 + n23;
+}
+
 // OR `nbits` bits into the bucket image at bit position pos (shared memory, zeroed before)
 __device__ __forceinline__ void put_bits(uint32_t* img, uint32_t pos, uint64_t bits, uint32_t nbits) {
   if (nbits == 0) return;

@@ -131,31 +131,63 @@ __device__ __forceinline__ int quantize_level(float absv, float norm, const floa
   return tau + ((r < xi) ? 1 : 0);
 }
 
+// The exact routine as one out-of-line copy (it runs for about 1e-5 of the coordinates).
+static __device__ __noinline__ int quantize_level_slow(float absv, float norm, const float* lev, int nlev, uint32_t word) {
+  return quantize_level(absv, norm, lev, nlev, word);
+}
+
 // Same decision as quantize_level, without divisions in the common case.  With rn = RN(1/norm),
 // u' = RN(|v| rn) differs from the exact u = RN(|v| / norm) by at most 2^-22 u.  tau is found from a
-// table on the float pattern of u' plus `steps` comparisons; T = (u' - l_tau) 2^23 / width differs
-// from xi 2^23 by less than margin = 4 l_{tau+1} / width + 8.  The 24-bit variate m rounds up iff
-// m < xi 2^24; with m' = m >> 1 taken as a float through the 2^23 trick, the sign of T - m' decides
-// whenever |T - m'| > margin and T is further than margin from both ends of the interval (so that
-// u' and u lie in the same interval).  Otherwise (about 1e-5 of coordinates) the exact routine runs.
-__device__ __forceinline__ int quantize_fast(float absv, float rn, float norm, const QuantTable* q, int steps,
-                                             const float* lev, int nlev, uint32_t word) {
+// table on the float pattern of u' plus two comparisons (tables that would need more send every
+// coordinate to the exact routine); T = (u' - l_tau) 2^23 / width differs from xi 2^23 by less than
+// margin = 4 l_{tau+1} / width + 8.  The 24-bit variate m rounds up iff m < xi 2^24; with m' = m >> 1
+// taken as a float through the 2^23 trick, the sign of T - m' decides whenever |T - m'| > margin and T
+// is further than margin from both ends of the interval (so that u' and u lie in the same interval).
+// Returns the level index and sets *unsafe when the exact routine has to decide instead.
+__device__ __forceinline__ int quantize_fast(float absv, float rn, const QuantTable* q, uint32_t word, bool* unsafe) {
   const float u = fminf(__fmul_rn(absv, rn), 1.0f);
   const int key = max((int)(__float_as_uint(u) >> kKeyShift), kKeyMin) - kKeyMin;
   const int tau0 = q->start[key];
-  int tau = tau0;
-  for (int i = 1; i <= steps; ++i) tau += (q->upper[tau0 + i] <= u) ? 1 : 0;
+  const int tau = tau0 + ((q->upper[tau0 + 1] <= u) ? 1 : 0) + ((q->upper[tau0 + 2] <= u) ? 1 : 0);
   const float4 iv = q->interval[tau];
   const float T = __fmul_rn(__fsub_rn(u, iv.x), iv.y);
   const float mhalf = __fsub_rn(__uint_as_float(0x4B000000u | (word >> 9)), 8388608.0f);   // (m >> 1), exact
   const float diff = __fsub_rn(T, mhalf);
-  if (fabsf(diff) > iv.z && T > iv.z && T < iv.w) return tau + (diff > 0.0f ? 1 : 0);
-  return quantize_level(absv, norm, lev, nlev, word);
+  // a zero coordinate is level 0 whatever the variate (T = 0, diff <= 0), so it needs no second look
+  *unsafe = (absv != 0.0f) && !(fabsf(diff) > iv.z && T > iv.z && T < iv.w);
+  return tau + (diff > 0.0f ? 1 : 0);
+}
+
+// Level indices of the four coordinates of a quad, packed one per byte (no sign).
+__device__ __forceinline__ uint32_t quantize_quad(const float4 x, const uint4 w, float rn, float norm, const QuantTable* q,
+                                                  const float* lev, int nlev) {
+  bool u0, u1, u2, u3;
+  int i0 = quantize_fast(fabsf(x.x), rn, q, w.x, &u0);
+  int i1 = quantize_fast(fabsf(x.y), rn, q, w.y, &u1);
+  int i2 = quantize_fast(fabsf(x.z), rn, q, w.z, &u2);
+  int i3 = quantize_fast(fabsf(x.w), rn, q, w.w, &u3);
+  if (u0 | u1 | u2 | u3) {
+    if (u0) i0 = quantize_level_slow(fabsf(x.x), norm, lev, nlev, w.x);
+    if (u1) i1 = quantize_level_slow(fabsf(x.y), norm, lev, nlev, w.y);
+    if (u2) i2 = quantize_level_slow(fabsf(x.z), norm, lev, nlev, w.z);
+    if (u3) i3 = quantize_level_slow(fabsf(x.w), norm, lev, nlev, w.w);
+  }
+  return (uint32_t)i0 | ((uint32_t)i1 << 8) | ((uint32_t)i2 << 16) | ((uint32_t)i3 << 24);
+}
+
+// sign bits of the four coordinates, at bits 7, 15, 23, 31, dropped where the level index is zero
+__device__ __forceinline__ uint32_t quad_symbols(const float4 x, uint32_t idx4) {
+  const uint32_t s = ((__float_as_uint(x.x) >> 31) << 7) | ((__float_as_uint(x.y) >> 31) << 15) |
+                     ((__float_as_uint(x.z) >> 31) << 23) | ((__float_as_uint(x.w) >> 31) << 31);
+  // a byte of idx4 is nonzero iff (byte + 0x7f) has bit 7 set (level indices are < 0x80)
+  const uint32_t nz = (idx4 + 0x7f7f7f7fu) & 0x80808080u;
+  return idx4 | (s & nz);
 }
 
 // reciprocal of a bucket norm for quantize_fast; 0 sends every coordinate to the exact routine
-__device__ __forceinline__ float fast_reciprocal(float norm) {
-  return (norm > 7.9e-31f && norm < 1.2e30f) ? __frcp_rn(norm) : 0.0f;
+// (u' = 0 is never further than the margin from the lower end of its interval)
+__device__ __forceinline__ float fast_reciprocal(float norm, int steps) {
+  return (norm > 7.9e-31f && norm < 1.2e30f && steps <= 2) ? __frcp_rn(norm) : 0.0f;
 }
 
 __device__ __forceinline__ uint32_t symbol_of(float v, int idx) {

@@ -122,6 +122,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   extern __shared__ uint32_t s_img[];
   __shared__ QuantTable s_q;
   __shared__ EncLut s_lut;
+  __shared__ uint32_t s_pair[kPairLutSize];
   __shared__ float s_lev[QGX_MAX_LEVELS];
   __shared__ double s_red[2][32];
   __shared__ uint32_t s_chunk[2][8 * 16];
@@ -144,6 +145,8 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 1.0f;
   if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
   __syncthreads();
+  fill_pair_lut(s_pair, &s_lut);
+  __syncthreads();
   const int steps = s_q.steps;
   const int nlev = lt.nlev;
 
@@ -159,7 +162,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     for (int i = threadIdx.x; i < img_words; i += blockDim.x) s_img[i] = 0;
     const float norm = bucket_norm_all<V4>(r, a.norm_type, s_red[par]);      // barrier inside: the image is zero
     const bool finite = (norm - norm) == 0.0f;
-    const float rn = fast_reciprocal(norm);
+    const float rn = fast_reciprocal(norm, steps);
     if (threadIdx.x == 0) {
       a.norms[k * a.nb + b] = norm;
       if (!finite) latch_error(a.st, QGX_ERR_NONFINITE);
@@ -174,40 +177,38 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     for (int j = 0; j < V4; ++j) {
       const int q = j * (int)blockDim.x + (int)threadIdx.x;
       const int nvalid = max(0, min(kQuad, len - q * kQuad));
-      uint64_t acc = 0;
-      uint32_t n = 0;
-      if (nvalid > 0 && finite) {
+      uint32_t sym4 = 0;
+      if (nvalid > 0 && finite && norm != 0.0f) {
         const uint64_t ctr = (uint64_t)(lo >> 2) + (uint64_t)q;
         const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
-        const float xs[kQuad] = {r.x[j].x, r.x[j].y, r.x[j].z, r.x[j].w};
-        const uint32_t ws[kQuad] = {w.x, w.y, w.z, w.w};
+        sym4 = quad_symbols(r.x[j], quantize_quad(r.x[j], w, rn, norm, &s_q, s_lev, nlev));
+      }
+      if (nvalid == kQuad) {
+        pack_quad_pairs(sym4, s_pair, &qbits[j], &qn[j]);
+      } else {
+        pack_quad(sym4, nvalid, &s_lut, &qbits[j], &qn[j]);      // the ragged end of a bucket
+      }
+    }
+    // warp scans of the bit counts, two quads per 32-bit word (a chunk holds at most 32 * 52 bits)
 #pragma unroll
-        for (int c = 0; c < kQuad; ++c) {
-          if (c < nvalid) {
-            const int idx = quantize_fast(fabsf(xs[c]), rn, norm, &s_q, steps, s_lev, nlev, ws[c]);
-            const uint32_t e = s_lut.e[(uint32_t)idx | ((__float_as_uint(xs[c]) >> 31) << 5)];
-            acc |= (uint64_t)(e & 0xffffu) << n;
-            n += e >> 16;
-          }
-        }
-      } else if (nvalid > 0) {
-        const uint32_t e = s_lut.e[0];                   // non-finite norm: every coordinate is sent as level 0
-        for (int c = 0; c < nvalid; ++c) { acc |= (uint64_t)(e & 0xffffu) << n; n += e >> 16; }
-      }
-      qbits[j] = acc;
-      qn[j] = n;
-      const uint32_t incl = warp_incl_scan(n, lane);
-      qexcl[j] = incl - n;
-      // sub-block lengths: the last lane of each sub-block knows its total
+    for (int j = 0; j < V4; j += 2) {
+      const uint32_t both = qn[j] | ((j + 1 < V4 ? qn[j + 1] : 0u) << 16);
+      const uint32_t incl = warp_incl_scan(both, lane);
       const uint32_t before = __shfl_up_sync(0xffffffffu, incl, kSegLanes);
-      if ((lane + 1) % kSegLanes == 0) {
-        const int sb = (j * nwarps + warp) * kSegs + lane / kSegLanes;
-        if (sb * G < len) {
-          const uint32_t L = incl - (lane >= kSegLanes ? before : 0u);
-          put_bits(s_img, kNormBits + 16u * (uint32_t)sb, (uint64_t)(L & 0xffffu), 16u);
+      const uint32_t seg = incl - (lane >= kSegLanes ? before : 0u);   // per field: no borrow, the scans are monotone
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (j + h < V4) {
+          const uint32_t mine = (incl >> (16 * h)) & 0xffffu;
+          qexcl[j + h] = mine - qn[j + h];
+          // sub-block lengths: the last lane of each sub-block knows its total
+          if ((lane + 1) % kSegLanes == 0) {
+            const int sb = ((j + h) * nwarps + warp) * kSegs + lane / kSegLanes;
+            if (sb * G < len) put_bits(s_img, kNormBits + 16u * (uint32_t)sb, (uint64_t)((seg >> (16 * h)) & 0xffffu), 16u);
+          }
+          if (lane == 31) s_chunk[par][(j + h) * nwarps + warp] = mine;
         }
       }
-      if (lane == 31) s_chunk[par][j * nwarps + warp] = incl;
     }
     __syncthreads();
     // exclusive prefix of the chunk totals, computed by every warp for itself

@@ -36,8 +36,7 @@ __global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int 
   }
   const bool finite = (norm - norm) == 0.0f;
   if (!finite && threadIdx.x == 0) latch_error(st, QGX_ERR_NONFINITE);
-  const float rn = fast_reciprocal(norm);
-  const int steps = s_q.steps;
+  const float rn = fast_reciprocal(norm, s_q.steps);
 
   uint8_t* out = sym + k * d + lo;
   const bool sym_vec = vec_ok;            // d % 4 == 0 and bucket % 4 == 0: every quad is 4-byte aligned
@@ -47,15 +46,11 @@ __global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int 
     const int e = q * kQuad;
     if (e >= len) continue;
     uint32_t packed = 0;
-    if (finite) {
+    if (finite && norm != 0.0f) {
       const uint64_t ctr = (uint64_t)(lo >> 2) + (uint64_t)q;      // (coordinate index) / 4
       const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, xid, key);
       const float4 x = r.x[j];
-      const uint32_t s0 = symbol_of(x.x, quantize_fast(fabsf(x.x), rn, norm, &s_q, steps, s_lev, lt.nlev, w.x));
-      const uint32_t s1 = symbol_of(x.y, quantize_fast(fabsf(x.y), rn, norm, &s_q, steps, s_lev, lt.nlev, w.y));
-      const uint32_t s2 = symbol_of(x.z, quantize_fast(fabsf(x.z), rn, norm, &s_q, steps, s_lev, lt.nlev, w.z));
-      const uint32_t s3 = symbol_of(x.w, quantize_fast(fabsf(x.w), rn, norm, &s_q, steps, s_lev, lt.nlev, w.w));
-      packed = s0 | (s1 << 8) | (s2 << 16) | (s3 << 24);
+      packed = quad_symbols(x, quantize_quad(x, w, rn, norm, &s_q, s_lev, lt.nlev));
     }
     if (e + kQuad <= len && sym_vec) {
       *reinterpret_cast<uint32_t*>(out + e) = packed;
