@@ -262,6 +262,14 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
 }
 
 // ---- decode + average ------------------------------------------------------------------------
+// Decoder table of the fused path: index = the next maxlen + 1 stream bits (codeword, then the sign
+// bit of a nonzero level); entry = the signed level value and the bits consumed (bit 7 set: no
+// codeword starts like this, one bit is consumed so that the walk goes on and the lengths disagree).
+struct DecEntry {
+  float val;
+  uint32_t len;
+};
+
 struct DecodeArgs {
   const uint32_t* stream;       // [K][cap_words]
   size_t cap_words;
@@ -277,7 +285,7 @@ struct DecodeArgs {
   int bucket;
   int K;
   size_t nb;
-  const uint16_t* lut;          // decoder table in global memory
+  const DecEntry* lut;          // decoder table in global memory, 1 << (maxlen + 1) entries
   float* mean;                  // [d]
   // optional fused state update (the two axpy of Eq. Q-GenX)
   int update;                   // 0 none, 1: xout = xin - gamma * mean, 2: xout = xin - mean
@@ -287,11 +295,42 @@ struct DecodeArgs {
   DevStatus* st;
 };
 
-// start of sub-block `s` (bits after the header) = sum of the 16-bit lengths before it; all lanes
-// of the warp share the bucket; returns false if the header is inconsistent with nbits
-__device__ __forceinline__ uint32_t subblock_start(const uint32_t* w, uint32_t s, int lane) {
-  // lengths of sub-blocks [0, s - lane) are summed cooperatively, then a scan inside the warp
-  const uint32_t warp_first = s - (uint32_t)lane;
+constexpr int kDecThreads = 128;
+constexpr int kDecChunk = 32;           // coordinates whose running sums a thread keeps in registers
+constexpr uint32_t kStateStep = 1u - (1u << 18);   // adding L * step moves the position up and the bits left down by L
+
+// Bits not yet consumed of one sub-block: a 64-bit window refilled 32 bits at a time.  The streams
+// of the fused path lie in the context's workspace, which extends past every bucket, so a read a
+// few words beyond a (corrupt) sub-block stays inside allocated memory.
+struct Window {
+  const uint32_t* next;
+  uint32_t lo, hi;
+  int avail;
+  __device__ __forceinline__ void open(const uint32_t* words, uint32_t bitpos) {
+    const uint32_t* p = words + (bitpos >> 5);
+    const uint32_t sh = bitpos & 31u;
+    const uint32_t w0 = p[0], w1 = p[1];
+    lo = __funnelshift_r(w0, w1, sh);
+    hi = w1 >> sh;
+    avail = 64 - (int)sh;                               // the window ends on a word boundary
+    next = p + 2;
+  }
+  __device__ __forceinline__ void refill() {            // needs avail <= 32
+    const uint32_t w = *next++;
+    lo |= __funnelshift_lc(0u, w, (uint32_t)avail);     // w << avail, nothing when avail == 32
+    hi |= __funnelshift_lc(w, 0u, (uint32_t)avail);     // the bits of w that do not fit the low word
+    avail += 32;
+  }
+  __device__ __forceinline__ void skip(uint32_t n) {    // n < 32
+    lo = __funnelshift_r(lo, hi, n);
+    hi >>= n;
+    avail -= (int)n;
+  }
+};
+
+// start of sub-block `s` (bits after the header) = sum of the 16-bit lengths before it; all lanes of
+// the warp share the bucket and hold consecutive sub-blocks
+__device__ __forceinline__ uint32_t header_sum_before_warp(const uint32_t* w, uint32_t warp_first, int lane) {
   uint32_t before = 0;
   for (uint32_t i = (uint32_t)lane; i < warp_first; i += 32) {
     const uint32_t bit = kNormBits + 16u * i;
@@ -302,25 +341,67 @@ __device__ __forceinline__ uint32_t subblock_start(const uint32_t* w, uint32_t s
   return before;
 }
 
+// where sub-block s of bucket (k, b) starts and how long it is; false if the bucket's numbers disagree
+__device__ __forceinline__ bool locate_subblock(const uint32_t* stream, size_t cap_words, const uint32_t* bucket_bits,
+                                                const uint32_t* offsets, size_t kb, uint32_t hdr_bits, uint32_t s,
+                                                bool exists, bool uniform, int lane, const uint32_t** words, float* norm,
+                                                uint32_t* start, uint32_t* want) {
+  const uint32_t nbits = bucket_bits[kb];
+  const uint32_t off = offsets[kb];
+  const uint32_t* w = stream + off;
+  *words = w;
+  const bool ok = nbits >= hdr_bits && (size_t)off + ((nbits + 31) >> 5) <= cap_words;
+  uint32_t st = 0, len = 0;
+  float nm = 0.0f;
+  if (ok) {
+    nm = __uint_as_float(w[0]);
+    if (uniform) {
+      const uint32_t bit = kNormBits + 16u * s;
+      len = exists ? ((w[bit >> 5] >> (bit & 31u)) & 0xffffu) : 0u;
+      const uint32_t incl = warp_incl_scan(len, lane);
+      st = header_sum_before_warp(w, s - (uint32_t)lane, lane) + incl - len;
+    } else if (exists) {
+      for (uint32_t i = 0; i <= s; ++i) {
+        const uint32_t bit = kNormBits + 16u * i;
+        const uint32_t L = (w[bit >> 5] >> (bit & 31u)) & 0xffffu;
+        if (i < s) st += L; else len = L;
+      }
+    }
+  }
+  *norm = nm;
+  *start = hdr_bits + st;
+  *want = len;
+  return ok && (!exists || (hdr_bits + st + len <= nbits && nbits < (1u << 18) && len < (1u << 14)));
+}
+
+// One thread per sub-block.  The thread walks its sub-block of every worker's stream 32 coordinates
+// at a time, keeping the 32 running sums in registers and each worker's bit position in shared memory.
 template <int G, bool DIFF>
-__global__ void __launch_bounds__(128) k_exchange_decode(DecodeArgs a, LevelTable lt, CodeTable ct) {
-  extern __shared__ uint32_t s_dyn[];
-  __shared__ float s_lev[QGX_MAX_LEVELS];
-  uint16_t* s_lut = reinterpret_cast<uint16_t*>(s_dyn);
-  const int lut_n = 1 << ct.maxlen;
-  for (int i = threadIdx.x; i < lut_n; i += blockDim.x) s_lut[i] = a.lut[i];
-  if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 0.0f;
+__global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_constant__ DecodeArgs a, const __grid_constant__ CodeTable ct) {
+  extern __shared__ __align__(16) unsigned char s_raw[];
+  const int lut_n = 2 << ct.maxlen;
+  DecEntry* s_lut = reinterpret_cast<DecEntry*>(s_raw);
+  // per worker and thread: bit position in the bucket (low 18 bits) | bits left in the sub-block << 18
+  uint32_t* s_state = reinterpret_cast<uint32_t*>(s_raw + sizeof(DecEntry) * (size_t)lut_n);    // [K][threads]
+  float* s_norm = reinterpret_cast<float*>(s_state + (size_t)a.K * kDecThreads);                // [K][threads]
+  uint32_t* s_state2 = reinterpret_cast<uint32_t*>(s_norm + (size_t)a.K * kDecThreads);
+  float* s_norm2 = reinterpret_cast<float*>(s_state2 + (size_t)a.K * kDecThreads);
+  {
+    const uint2* src = reinterpret_cast<const uint2*>(a.lut);
+    uint2* dst = reinterpret_cast<uint2*>(s_lut);
+    for (int i = threadIdx.x; i < lut_n; i += blockDim.x) dst[i] = src[i];
+  }
   __syncthreads();
   const uint32_t mask = (uint32_t)lut_n - 1u;
-  const int lane = threadIdx.x & 31;
-  const size_t spb = (size_t)a.bucket / G;              // sub-blocks per full bucket (bucket % G == 0, spb % 32 == 0 or spb < 32 handled by the host)
+  const int lane = threadIdx.x & 31, tid = threadIdx.x;
+  const size_t spb = (size_t)a.bucket / G;
   const size_t total_sub = a.nb * spb;
+  const bool uniform = (spb % 32 == 0);
   const float Kf = (float)a.K;
   double sq = 0.0;
   bool bad = false;
 
-  for (size_t gs = (size_t)blockIdx.x * blockDim.x + threadIdx.x; gs - lane < total_sub; gs += (size_t)gridDim.x * blockDim.x) {
-    // the warp's 32 sub-blocks lie in one bucket when spb % 32 == 0; otherwise lanes may differ
+  for (size_t gs = (size_t)blockIdx.x * blockDim.x + tid; gs - lane < total_sub; gs += (size_t)gridDim.x * blockDim.x) {
     const bool live = gs < total_sub;
     const size_t b = live ? gs / spb : a.nb - 1;
     const uint32_t s = live ? (uint32_t)(gs % spb) : 0u;
@@ -330,115 +411,95 @@ __global__ void __launch_bounds__(128) k_exchange_decode(DecodeArgs a, LevelTabl
     const int count = live ? max(0, min(G, len - first)) : 0;
     const uint32_t nsub = (uint32_t)((len + G - 1) / G);
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
-    const bool uniform = (spb % 32 == 0);
+    if (!__any_sync(0xffffffffu, count > 0)) continue;   // beyond the end of a short last bucket
 
-    float acc[G];
-#pragma unroll
-    for (int i = 0; i < G; ++i) acc[i] = 0.0f;
-    // a warp none of whose sub-blocks exists (beyond the end of a short last bucket) reads nothing
-    if (!__any_sync(0xffffffffu, count > 0)) continue;
-
+    // where this sub-block lies in every worker's stream
     for (int k = 0; k < a.K; ++k) {
-      const uint32_t nbits = a.bucket_bits[(size_t)k * a.nb + b];
-      const uint32_t nwords = (nbits + 31) >> 5;
-      const uint32_t* w = a.stream + (size_t)k * a.cap_words + a.offsets[(size_t)k * a.nb + b];
-      const bool hdr_ok = nbits >= hdr_bits && (size_t)a.offsets[(size_t)k * a.nb + b] + nwords <= a.cap_words;
-      uint32_t start = 0, want = 0;
-      float norm = 0.0f;
-      if (hdr_ok) {
-        norm = __uint_as_float(w[0]);
-        if (uniform) {
-          const uint32_t bit = kNormBits + 16u * s;
-          const uint32_t mylen = (count > 0) ? ((w[bit >> 5] >> (bit & 31u)) & 0xffffu) : 0u;
-          const uint32_t incl = warp_incl_scan(mylen, lane);
-          start = subblock_start(w, s, lane) + incl - mylen;
-          want = mylen;
-        } else if (count > 0) {
-          for (uint32_t i = 0; i <= s; ++i) {
-            const uint32_t bit = kNormBits + 16u * i;
-            const uint32_t L = (w[bit >> 5] >> (bit & 31u)) & 0xffffu;
-            if (i < s) start += L; else want = L;
-          }
-        }
-      } else {
-        bad = true;
-      }
-      // second stream set (the other exchange of the iteration), same geometry
-      uint32_t start2 = 0, want2 = 0;
-      float norm2 = 0.0f;
-      const uint32_t* w2 = nullptr;
-      uint32_t nwords2 = 0;
-      bool ok2 = false;
+      const size_t kb = (size_t)k * a.nb + b;
+      const uint32_t* w;
+      float nm;
+      uint32_t st, want;
+      const bool ok = locate_subblock(a.stream + (size_t)k * a.cap_words, a.cap_words, a.bucket_bits, a.offsets, kb, hdr_bits, s,
+                                      count > 0, uniform, lane, &w, &nm, &st, &want);
+      bad = bad || !ok;
+      s_state[k * kDecThreads + tid] = ok ? (st | (want << 18)) : 0u;
+      s_norm[k * kDecThreads + tid] = ok ? nm : 0.0f;
       if (DIFF) {
-        const uint32_t nbits2 = a.bucket_bits2[(size_t)k * a.nb + b];
-        nwords2 = (nbits2 + 31) >> 5;
-        w2 = a.stream2 + (size_t)k * a.cap_words2 + a.offsets2[(size_t)k * a.nb + b];
-        ok2 = nbits2 >= hdr_bits && (size_t)a.offsets2[(size_t)k * a.nb + b] + nwords2 <= a.cap_words2;
-        if (ok2) {
-          norm2 = __uint_as_float(w2[0]);
-          if (uniform) {
-            const uint32_t bit = kNormBits + 16u * s;
-            const uint32_t mylen = (count > 0) ? ((w2[bit >> 5] >> (bit & 31u)) & 0xffffu) : 0u;
-            const uint32_t incl = warp_incl_scan(mylen, lane);
-            start2 = subblock_start(w2, s, lane) + incl - mylen;
-            want2 = mylen;
-          } else if (count > 0) {
-            for (uint32_t i = 0; i <= s; ++i) {
-              const uint32_t bit = kNormBits + 16u * i;
-              const uint32_t L = (w2[bit >> 5] >> (bit & 31u)) & 0xffffu;
-              if (i < s) start2 += L; else want2 = L;
+        const bool ok2 = locate_subblock(a.stream2 + (size_t)k * a.cap_words2, a.cap_words2, a.bucket_bits2, a.offsets2, kb,
+                                         hdr_bits, s, count > 0, uniform, lane, &w, &nm, &st, &want);
+        bad = bad || !ok2;
+        s_state2[k * kDecThreads + tid] = ok2 ? (st | (want << 18)) : 0u;
+        s_norm2[k * kDecThreads + tid] = ok2 ? nm : 0.0f;
+      }
+    }
+    if (count <= 0) continue;
+
+    float gam = 1.0f;
+    if (a.update == 1) gam = (float)a.scalars[1];
+    for (int c0 = 0; c0 < count; c0 += kDecChunk) {
+      const int n = min(kDecChunk, count - c0);
+      float acc[kDecChunk];
+#pragma unroll
+      for (int i = 0; i < kDecChunk; ++i) acc[i] = 0.0f;
+      for (int k = 0; k < a.K; ++k) {
+        const size_t kb = (size_t)k * a.nb + b;
+        const float norm = s_norm[k * kDecThreads + tid];
+        uint32_t state = s_state[k * kDecThreads + tid];
+        Window win;
+        win.open(a.stream + (size_t)k * a.cap_words + a.offsets[kb], state & 0x3ffffu);
+        uint32_t flags = 0;
+        Window win2;
+        float norm2 = 0.0f;
+        uint32_t state2 = 0;
+        if (DIFF) {
+          norm2 = s_norm2[k * kDecThreads + tid];
+          state2 = s_state2[k * kDecThreads + tid];
+          win2.open(a.stream2 + (size_t)k * a.cap_words2 + a.offsets2[kb], state2 & 0x3ffffu);
+        }
+#pragma unroll
+        for (int i = 0; i < kDecChunk; ++i) {
+          if ((i & 1) == 0) {                              // two symbols use at most 26 bits
+            if (win.avail <= 32) win.refill();
+            if (DIFF) { if (win2.avail <= 32) win2.refill(); }
+          }
+          if (i < n) {
+            const DecEntry e = s_lut[win.lo & mask];
+            const uint32_t L = e.len & 31u;
+            flags |= e.len;
+            win.skip(L);
+            state += L * kStateStep;                       // position up, bits left down
+            const float val = __fmul_rn(norm, e.val);
+            acc[i] = __fadd_rn(acc[i], val);
+            if (DIFF) {
+              const DecEntry e2 = s_lut[win2.lo & mask];
+              const uint32_t L2 = e2.len & 31u;
+              flags |= e2.len;
+              win2.skip(L2);
+              state2 += L2 * kStateStep;
+              const float dlt = __fsub_rn(val, __fmul_rn(norm2, e2.val));
+              sq = fma((double)dlt, (double)dlt, sq);
             }
           }
-        } else {
-          bad = true;
         }
+        bad = bad || (flags & 0x80u);
+        s_state[k * kDecThreads + tid] = state;
+        if (DIFF) s_state2[k * kDecThreads + tid] = state2;
       }
-      if (count <= 0) continue;
-      if (hdr_ok && hdr_bits + start + want > nbits) { bad = true; continue; }
-      if (DIFF && ok2 && hdr_bits + start2 + want2 > nwords2 * 32u) { bad = true; continue; }
-
-      BitReader br;
-      br.w = w; br.nwords = hdr_ok ? nwords : 0u;
-      br.seek(hdr_bits + start);
-      BitReader br2;
-      if (DIFF) { br2.w = w2; br2.nwords = ok2 ? nwords2 : 0u; br2.seek(hdr_bits + start2); }
-      uint32_t used = 0, used2 = 0;
-      bool ok = hdr_ok, okb = ok2;
+      // mean (and the fused state update) of these coordinates
+      const size_t e0 = lo + (size_t)first + (size_t)c0;
 #pragma unroll
-      for (int i = 0; i < G; ++i) {
-        if (i < count) {
-          uint32_t sym = 0;
-          if (ok) ok = decode_symbol(br, s_lut, mask, &sym, &used) && used <= want;
-          if (!ok) sym = 0;
-          const float val = dequantize_symbol(sym, norm, s_lev);
-          acc[i] = __fadd_rn(acc[i], val);
-          if (DIFF) {
-            uint32_t sym2 = 0;
-            if (okb) okb = decode_symbol(br2, s_lut, mask, &sym2, &used2) && used2 <= want2;
-            if (!okb) sym2 = 0;
-            const float dlt = __fsub_rn(val, dequantize_symbol(sym2, norm2, s_lev));
-            sq = fma((double)dlt, (double)dlt, sq);
-          }
-        }
-      }
-      if (!ok || used != want) bad = true;
-      if (DIFF && (!okb || used2 != want2)) bad = true;
-    }
-
-    // mean (and the fused state update) for this sub-block's coordinates
-    if (count > 0) {
-      const size_t e0 = lo + (size_t)first;
-      float gam = 1.0f;
-      if (a.update == 1) gam = (float)a.scalars[1];
-#pragma unroll
-      for (int i = 0; i < G; ++i) {
-        if (i < count) {
+      for (int i = 0; i < kDecChunk; ++i) {
+        if (i < n) {
           const float m = __fdiv_rn(acc[i], Kf);
           a.mean[e0 + i] = m;
           if (a.update == 1) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], __fmul_rn(gam, m));
           if (a.update == 2) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], m);
         }
       }
+    }
+    for (int k = 0; k < a.K; ++k) {
+      bad = bad || ((s_state[k * kDecThreads + tid] >> 18) != 0u);       // every sub-block used exactly its length
+      if (DIFF) bad = bad || ((s_state2[k * kDecThreads + tid] >> 18) != 0u);
     }
   }
   if (DIFF) {
@@ -455,9 +516,9 @@ namespace qgx {
 
 // workspace slots of a context
 enum { WS_OFF64 = 0, WS_FLAGS = 1, WS_LUT = 2, WS_SLOT0 = 3 /* stream, bits, offsets, total: 3..6 and 7..10 */,
-       WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16 };
+       WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18 };
 
-qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const LevelTable& lt, const CodeTable& ct, bool diff);
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct, bool diff);
 
 // the whole exchange; diff_slot >= 0 also accumulates sum_k ||vhat(slot) - vhat(diff_slot)||^2 into sum_sq
 qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
@@ -479,13 +540,13 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const size_t nb = (d + (size_t)bucket - 1) / (size_t)bucket;
   const size_t cap = qgx_stream_capacity_words(d, bucket, cfg->cb.subblock, QGX_MAX_CODE_LEN);   // fits any codebook
   const int base = WS_SLOT0 + 4 * slot;
-  uint32_t* stream = (uint32_t*)ws_get(c, base + 0, sizeof(uint32_t) * (size_t)K * cap);
+  uint32_t* stream = (uint32_t*)ws_get(c, base + 0, sizeof(uint32_t) * ((size_t)K * cap + 64));   // slack: see Window
   uint32_t* bbits = (uint32_t*)ws_get(c, base + 1, sizeof(uint32_t) * (size_t)K * nb);
   uint32_t* offs = (uint32_t*)ws_get(c, base + 2, sizeof(uint32_t) * (size_t)K * nb);
   unsigned long long* tot = (unsigned long long*)ws_get(c, base + 3, sizeof(uint64_t) * (size_t)K);
   unsigned long long* status = (unsigned long long*)ws_get(c, WS_STATUS, sizeof(uint64_t) * ((size_t)K * nb + 2));
   float* norms = (float*)ws_get(c, WS_NORMS, sizeof(float) * (size_t)K * nb);
-  uint16_t* lut = (uint16_t*)ws_get(c, WS_LUT, sizeof(uint16_t) * kDecLutMax);
+  DecEntry* lut = (DecEntry*)ws_get(c, WS_DLUT, sizeof(DecEntry) * (size_t)(2 * kDecLutMax));
   if (!stream || !bbits || !offs || !tot || !status || !norms || !lut) return QGX_ERR_CUDA;
   c->slot_cap_words[slot] = cap;
   c->slot_K[slot] = K;
@@ -541,11 +602,23 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
       cudaMemcpyAsync(total_bits_out, tot, sizeof(uint64_t) * (size_t)K, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
     return QGX_ERR_CUDA;
 
-  // decoder table
-  std::vector<uint16_t> h_lut((size_t)1 << ct.maxlen);
-  build_dec_lut_host(ct, h_lut.data());
-  if (cudaMemcpyAsync(lut, h_lut.data(), h_lut.size() * sizeof(uint16_t), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
-    return QGX_ERR_CUDA;
+  // decoder table: the next maxlen + 1 bits -> signed level value and bits consumed
+  {
+    std::vector<uint16_t> by_code((size_t)1 << ct.maxlen);
+    build_dec_lut_host(ct, by_code.data());
+    std::vector<DecEntry> h_lut((size_t)2 << ct.maxlen);
+    for (size_t i = 0; i < h_lut.size(); ++i) {
+      const uint16_t e = by_code[i & (((size_t)1 << ct.maxlen) - 1)];
+      const uint32_t L = e >> 8, idx = e & 0xffu;
+      if (L == 0) { h_lut[i].val = 0.0f; h_lut[i].len = 1u | 0x80u; continue; }
+      if (idx == 0) { h_lut[i].val = 0.0f; h_lut[i].len = L; continue; }
+      const bool neg = (i >> L) & 1u;
+      h_lut[i].val = neg ? -cfg->levels[idx] : cfg->levels[idx];
+      h_lut[i].len = L + 1u;
+    }
+    if (cudaMemcpyAsync(lut, h_lut.data(), h_lut.size() * sizeof(DecEntry), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+      return QGX_ERR_CUDA;
+  }
 
   DecodeArgs da;
   da.stream = stream; da.cap_words = cap; da.bucket_bits = bbits; da.offsets = offs;
@@ -561,37 +634,43 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   da.d = d; da.bucket = bucket; da.K = K; da.nb = nb; da.lut = lut; da.mean = mean_out;
   da.update = upd ? upd->mode : 0; da.xin = upd ? upd->xin : nullptr; da.xout = upd ? upd->xout : nullptr;
   da.scalars = upd ? upd->scalars : nullptr; da.st = c->dstatus;
-  return launch_decode_average(c, da, lt, ct, diff);
+  return launch_decode_average(c, da, ct, diff);
 }
 
 template <int G>
-static void launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const LevelTable& lt, const CodeTable& ct, bool diff) {
+static qgx_status launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, bool diff) {
   const size_t total_sub = da.nb * ((size_t)da.bucket / G);
-  const int threads = 128;
-  const size_t smem = sizeof(uint16_t) * ((size_t)1 << ct.maxlen);
+  const size_t per_set = (sizeof(uint32_t) + sizeof(float)) * (size_t)da.K * kDecThreads;
+  const size_t smem = sizeof(DecEntry) * ((size_t)2 << ct.maxlen) + per_set * (diff ? 2 : 1);
+  if (smem > 200 * 1024) return QGX_ERR_INVALID_ARG;   // too many workers for the per-thread positions
   int per_sm = 1;
-  if (diff) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, true>, threads, smem);
-  else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, false>, threads, smem);
+  if (diff) {
+    cudaFuncSetAttribute(k_exchange_decode<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, true>, kDecThreads, smem);
+  } else {
+    cudaFuncSetAttribute(k_exchange_decode<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, false>, kDecThreads, smem);
+  }
   if (per_sm < 1) per_sm = 1;
-  const size_t want = (total_sub + threads - 1) / threads;
+  const size_t want = (total_sub + kDecThreads - 1) / kDecThreads;
   const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
-    if (diff) k_exchange_decode<G, true><<<grid, threads, smem, c->stream>>>(da, lt, ct);
-    else k_exchange_decode<G, false><<<grid, threads, smem, c->stream>>>(da, lt, ct);
+    if (diff) k_exchange_decode<G, true><<<grid, kDecThreads, smem, c->stream>>>(da, ct);
+    else k_exchange_decode<G, false><<<grid, kDecThreads, smem, c->stream>>>(da, ct);
   }
   count_launch(c);
+  return cuda_status(cudaGetLastError());
 }
 
-qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const LevelTable& lt, const CodeTable& ct, bool diff) {
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, bool diff) {
   if (!ct.has_header || da.bucket % ct.G != 0) return QGX_ERR_INVALID_ARG;
   switch (ct.G) {
-    case 32: launch_decode_g<32>(c, da, lt, ct, diff); break;
-    case 64: launch_decode_g<64>(c, da, lt, ct, diff); break;
-    case 128: launch_decode_g<128>(c, da, lt, ct, diff); break;
+    case 32: return launch_decode_g<32>(c, da, ct, diff);
+    case 64: return launch_decode_g<64>(c, da, ct, diff);
+    case 128: return launch_decode_g<128>(c, da, ct, diff);
     default: return QGX_ERR_INVALID_ARG;
   }
-  return cuda_status(cudaGetLastError());
 }
 
 }  // namespace qgx
