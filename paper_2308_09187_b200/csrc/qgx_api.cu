@@ -128,6 +128,7 @@ qgx_status qgx_create(qgx_ctx** out, int device, void* cuda_stream) {
   if (!c) return QGX_ERR_CUDA;
   std::memset(c, 0, sizeof(*c));
   c->device = device;
+  c->sym_slot = -1;
   c->stream = (cudaStream_t)cuda_stream;
   if (cudaMalloc((void**)&c->dstatus, sizeof(DevStatus)) != cudaSuccess ||
       cudaMemsetAsync(c->dstatus, 0, sizeof(DevStatus), c->stream) != cudaSuccess ||

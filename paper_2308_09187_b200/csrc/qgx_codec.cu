@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(512) k_bit_scatter(const float* __restrict__ n
   __syncthreads();
   for (uint32_t s = threadIdx.x; s < nsub; s += blockDim.x) {
     const uint32_t L = s_sub[s + 1] - s_sub[s];
-    put_bits(s_img, kNormBits + 16u * s, (uint64_t)(L & 0xffffu), 16u);
+    reinterpret_cast<uint16_t*>(s_img)[2 + s] = (uint16_t)(L & 0xffffu);
   }
   __syncthreads();
   uint32_t* dst = stream + k * cap_words + off[k * nb + b];

@@ -66,16 +66,14 @@ __device__ __forceinline__ void pack_quad_pairs(uint32_t sym4, const uint32_t* p
   *nbits = n01 + n23;
 }
 
-// OR `nbits` bits into the bucket image at bit position pos (shared memory, zeroed before)
+// OR `nbits` (<= 52) bits into the bucket image at bit position pos (shared memory, zeroed before).
+// Two words are always touched; a third only when the bits reach it.
 __device__ __forceinline__ void put_bits(uint32_t* img, uint32_t pos, uint64_t bits, uint32_t nbits) {
-  if (nbits == 0) return;
   const uint32_t w = pos >> 5, sh = pos & 31u;
-  const uint64_t lo = bits << sh;
-  const uint32_t x0 = (uint32_t)lo, x1 = (uint32_t)(lo >> 32);
-  const uint32_t x2 = sh ? (uint32_t)(bits >> (64 - sh)) : 0u;
-  if (x0) atomicOr(&img[w], x0);
-  if (x1) atomicOr(&img[w + 1], x1);
-  if (x2) atomicOr(&img[w + 2], x2);
+  const uint32_t blo = (uint32_t)bits, bhi = (uint32_t)(bits >> 32);
+  atomicOr(&img[w], blo << sh);
+  atomicOr(&img[w + 1], __funnelshift_l(blo, bhi, sh));
+  if (sh + nbits > 64u) atomicOr(&img[w + 2], __funnelshift_l(bhi, 0u, sh));
 }
 
 // Decoder table: index = next `maxlen` stream bits, entry = level | codeword length << 8 (0 = no

@@ -35,6 +35,10 @@ struct qgx_ctx {
   size_t slot_cap_words[2];
   int slot_K[2];
   size_t slot_nb[2];
+  // which exchange slot last kept its symbols in the workspace (-1: none), and for what shape
+  int sym_slot;
+  int sym_K;
+  size_t sym_d;
   // optional per-kernel timing: pairs of events recorded around instrumented launches
   int timing_on;
   int timing_cap;                        // pairs allocated
@@ -108,8 +112,10 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
                                                const PhiloxKey& key) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;      // one wide multiply gives both halves
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
     const uint32_t n0 = hi1 ^ c1 ^ key.k0[r];
     const uint32_t n2 = hi0 ^ c3 ^ key.k1[r];
     c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;

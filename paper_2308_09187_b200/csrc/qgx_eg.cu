@@ -7,7 +7,7 @@ namespace qgx {
 
 // declared in qgx_exchange.cu / qgx_levels.cu
 qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
-                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int diff_slot, double* sum_sq);
+                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int sym_mode, double* sum_sq);
 qgx_status refit_from_source(qgx_ctx* c, DualSource src, int K, size_t d, qgx_quant_cfg* cfg, int refit, double* hist,
                              double* hist_host);
 enum { WS_OPVAL = 15, WS_MEAN = 16, WS_HIST = 17 };
@@ -163,13 +163,13 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
   }
   const uint32_t xid = 2u * (uint32_t)st->t;
   ExchangeUpdate half{1, st->X, st->Xhalf, st->scalars};                      // X_{t+1/2} = X_t - gamma_t * mean
-  rc = exchange_impl(c, src, K, d, cfg, xid, 0, mean, bits, &half, -1, nullptr);
+  rc = exchange_impl(c, src, K, d, cfg, xid, 0, mean, bits, &half, 1, nullptr);
   if (rc != QGX_OK) return rc;
   rc = apply_operator_impl(c, op, st->Xhalf, a);                              // A(X_{t+1/2})
   if (rc != QGX_OK) return rc;
   DualSource src2{noise_half, a};
   ExchangeUpdate dual{2, st->Y, st->Y, st->scalars};                          // Y_{t+1} = Y_t - mean
-  rc = exchange_impl(c, src2, K, d, cfg, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 0, st->scalars);
+  rc = exchange_impl(c, src2, K, d, cfg, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 2, st->scalars);
   if (rc != QGX_OK) return rc;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);

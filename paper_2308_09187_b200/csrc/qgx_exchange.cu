@@ -74,6 +74,13 @@ struct EncodeArgs {
   float* norms;                 // [K][nb] (kept for the caller; the streams carry them too)
   unsigned long long* status;   // [K][nb], zeroed before the launch
   unsigned int* ticket;         // zeroed before the launch
+  // optional: keep this exchange's symbols (1 byte per coordinate) ...
+  uint8_t* sym_out;             // [K][d] or null
+  // ... and compare with the symbols and norms kept by an earlier exchange:
+  // *sum_sq += sum_k ||Q(V_k) of that exchange - Q(V_k) of this one||^2 (fp32 differences, fp64 sum)
+  const uint8_t* sym_prev;      // [K][d] or null
+  const float* norms_prev;      // [K][nb]
+  double* sum_sq;
   DevStatus* st;
 };
 
@@ -114,7 +121,8 @@ __device__ __forceinline__ float bucket_norm_all(const BucketRegs<V4>& r, int no
 // One persistent CTA per SM slot; each ticket is one bucket (k = ticket % K, b = ticket / K).
 //   load + zero image | barrier | norm, quantize, pack, header fields, warp scans | barrier |
 //   chunk prefixes, bit scatter, look-back (warp 0) | barrier | copy out | barrier
-template <int V4, int G>
+// SYM: 0 plain, 1 also keeps the symbols, 2 also compares with the kept symbols of the other exchange
+template <int V4, int G, int SYM>
 __global__ void __launch_bounds__(V4 == 8 ? 512 : (V4 == 4 ? 512 : 256), V4 == 8 ? 2 : 1)
 k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
@@ -149,6 +157,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   __syncthreads();
   const int steps = s_q.steps;
   const int nlev = lt.nlev;
+  double sq = 0.0;
 
   for (int par = 0;; par ^= 1) {
     const unsigned long long t = s_ticket[par];
@@ -170,6 +179,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     const uint32_t nsub = (uint32_t)((len + G - 1) / G);
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
+    const float norm_prev = SYM == 2 ? a.norms_prev[k * a.nb + b] : 0.0f;
 
     uint64_t qbits[V4];
     uint32_t qn[V4], qexcl[V4];
@@ -182,6 +192,26 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
         const uint64_t ctr = (uint64_t)(lo >> 2) + (uint64_t)q;
         const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
         sym4 = quad_symbols(r.x[j], quantize_quad(r.x[j], w, rn, norm, &s_q, s_lev, nlev));
+      }
+      if (SYM == 1 && nvalid > 0) {
+        uint8_t* o = a.sym_out + k * a.d + lo + (size_t)q * kQuad;
+        if (nvalid == kQuad && a.vec_ok) *reinterpret_cast<uint32_t*>(o) = sym4;
+        else for (int c = 0; c < nvalid; ++c) o[c] = (uint8_t)(sym4 >> (8 * c));
+      }
+      if (SYM == 2 && nvalid > 0) {
+        const uint8_t* o = a.sym_prev + k * a.d + lo + (size_t)q * kQuad;
+        uint32_t prev4 = 0;
+        if (nvalid == kQuad && a.vec_ok) prev4 = __ldcs(reinterpret_cast<const uint32_t*>(o));
+        else for (int c = 0; c < nvalid; ++c) prev4 |= (uint32_t)o[c] << (8 * c);
+#pragma unroll
+        for (int c = 0; c < kQuad; ++c) {
+          if (c < nvalid) {
+            const float d1 = dequantize_symbol((prev4 >> (8 * c)) & 0xffu, norm_prev, s_lev);
+            const float d2 = dequantize_symbol((sym4 >> (8 * c)) & 0xffu, finite ? norm : 0.0f, s_lev);
+            const float dlt = __fsub_rn(d1, d2);
+            sq = fma((double)dlt, (double)dlt, sq);
+          }
+        }
       }
       if (nvalid == kQuad) {
         pack_quad_pairs(sym4, s_pair, &qbits[j], &qn[j]);
@@ -204,7 +234,8 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
           // sub-block lengths: the last lane of each sub-block knows its total
           if ((lane + 1) % kSegLanes == 0) {
             const int sb = ((j + h) * nwarps + warp) * kSegs + lane / kSegLanes;
-            if (sb * G < len) put_bits(s_img, kNormBits + 16u * (uint32_t)sb, (uint64_t)((seg >> (16 * h)) & 0xffffu), 16u);
+            // the 16-bit length fields are halfword aligned: a plain store
+            if (sb * G < len) reinterpret_cast<uint16_t*>(s_img)[2 + sb] = (uint16_t)((seg >> (16 * h)) & 0xffffu);
           }
           if (lane == 31) s_chunk[par][(j + h) * nwarps + warp] = mine;
         }
@@ -259,6 +290,10 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     __syncthreads();
   }
+  if (SYM == 2) {
+    sq = warp_sum(sq);
+    if (lane == 0 && sq != 0.0) atomicAdd(a.sum_sq, sq);
+  }
 }
 
 // ---- decode + average ------------------------------------------------------------------------
@@ -275,12 +310,6 @@ struct DecodeArgs {
   size_t cap_words;
   const uint32_t* bucket_bits;  // [K][nb]
   const uint32_t* offsets;      // [K][nb]
-  // second stream set whose decoded vectors are compared with the first (may be null)
-  const uint32_t* stream2;
-  size_t cap_words2;
-  const uint32_t* bucket_bits2;
-  const uint32_t* offsets2;
-  double* sum_sq;               // += sum_k ||vhat - vhat2||^2 (fp32 differences, fp64 sum)
   size_t d;
   int bucket;
   int K;
@@ -376,7 +405,7 @@ __device__ __forceinline__ bool locate_subblock(const uint32_t* stream, size_t c
 
 // One thread per sub-block.  The thread walks its sub-block of every worker's stream 32 coordinates
 // at a time, keeping the 32 running sums in registers and each worker's bit position in shared memory.
-template <int G, bool DIFF>
+template <int G>
 __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_constant__ DecodeArgs a, const __grid_constant__ CodeTable ct) {
   extern __shared__ __align__(16) unsigned char s_raw[];
   const int lut_n = 2 << ct.maxlen;
@@ -384,8 +413,6 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
   // per worker and thread: bit position in the bucket (low 18 bits) | bits left in the sub-block << 18
   uint32_t* s_state = reinterpret_cast<uint32_t*>(s_raw + sizeof(DecEntry) * (size_t)lut_n);    // [K][threads]
   float* s_norm = reinterpret_cast<float*>(s_state + (size_t)a.K * kDecThreads);                // [K][threads]
-  uint32_t* s_state2 = reinterpret_cast<uint32_t*>(s_norm + (size_t)a.K * kDecThreads);
-  float* s_norm2 = reinterpret_cast<float*>(s_state2 + (size_t)a.K * kDecThreads);
   {
     const uint2* src = reinterpret_cast<const uint2*>(a.lut);
     uint2* dst = reinterpret_cast<uint2*>(s_lut);
@@ -398,7 +425,6 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
   const size_t total_sub = a.nb * spb;
   const bool uniform = (spb % 32 == 0);
   const float Kf = (float)a.K;
-  double sq = 0.0;
   bool bad = false;
 
   for (size_t gs = (size_t)blockIdx.x * blockDim.x + tid; gs - lane < total_sub; gs += (size_t)gridDim.x * blockDim.x) {
@@ -424,13 +450,6 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
       bad = bad || !ok;
       s_state[k * kDecThreads + tid] = ok ? (st | (want << 18)) : 0u;
       s_norm[k * kDecThreads + tid] = ok ? nm : 0.0f;
-      if (DIFF) {
-        const bool ok2 = locate_subblock(a.stream2 + (size_t)k * a.cap_words2, a.cap_words2, a.bucket_bits2, a.offsets2, kb,
-                                         hdr_bits, s, count > 0, uniform, lane, &w, &nm, &st, &want);
-        bad = bad || !ok2;
-        s_state2[k * kDecThreads + tid] = ok2 ? (st | (want << 18)) : 0u;
-        s_norm2[k * kDecThreads + tid] = ok2 ? nm : 0.0f;
-      }
     }
     if (count <= 0) continue;
 
@@ -448,19 +467,10 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
         Window win;
         win.open(a.stream + (size_t)k * a.cap_words + a.offsets[kb], state & 0x3ffffu);
         uint32_t flags = 0;
-        Window win2;
-        float norm2 = 0.0f;
-        uint32_t state2 = 0;
-        if (DIFF) {
-          norm2 = s_norm2[k * kDecThreads + tid];
-          state2 = s_state2[k * kDecThreads + tid];
-          win2.open(a.stream2 + (size_t)k * a.cap_words2 + a.offsets2[kb], state2 & 0x3ffffu);
-        }
 #pragma unroll
         for (int i = 0; i < kDecChunk; ++i) {
           if ((i & 1) == 0) {                              // two symbols use at most 26 bits
             if (win.avail <= 32) win.refill();
-            if (DIFF) { if (win2.avail <= 32) win2.refill(); }
           }
           if (i < n) {
             const DecEntry e = s_lut[win.lo & mask];
@@ -470,20 +480,10 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
             state += L * kStateStep;                       // position up, bits left down
             const float val = __fmul_rn(norm, e.val);
             acc[i] = __fadd_rn(acc[i], val);
-            if (DIFF) {
-              const DecEntry e2 = s_lut[win2.lo & mask];
-              const uint32_t L2 = e2.len & 31u;
-              flags |= e2.len;
-              win2.skip(L2);
-              state2 += L2 * kStateStep;
-              const float dlt = __fsub_rn(val, __fmul_rn(norm2, e2.val));
-              sq = fma((double)dlt, (double)dlt, sq);
-            }
           }
         }
         bad = bad || (flags & 0x80u);
         s_state[k * kDecThreads + tid] = state;
-        if (DIFF) s_state2[k * kDecThreads + tid] = state2;
       }
       // mean (and the fused state update) of these coordinates
       const size_t e0 = lo + (size_t)first + (size_t)c0;
@@ -499,12 +499,7 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
     }
     for (int k = 0; k < a.K; ++k) {
       bad = bad || ((s_state[k * kDecThreads + tid] >> 18) != 0u);       // every sub-block used exactly its length
-      if (DIFF) bad = bad || ((s_state2[k * kDecThreads + tid] >> 18) != 0u);
     }
-  }
-  if (DIFF) {
-    sq = warp_sum(sq);
-    if (lane == 0 && sq != 0.0) atomicAdd(a.sum_sq, sq);
   }
   if (bad) latch_error(a.st, QGX_ERR_CORRUPT);
 }
@@ -518,11 +513,13 @@ namespace qgx {
 enum { WS_OFF64 = 0, WS_FLAGS = 1, WS_LUT = 2, WS_SLOT0 = 3 /* stream, bits, offsets, total: 3..6 and 7..10 */,
        WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18 };
 
-qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct, bool diff);
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct);
 
-// the whole exchange; diff_slot >= 0 also accumulates sum_k ||vhat(slot) - vhat(diff_slot)||^2 into sum_sq
+// The whole exchange.  sym_mode 1 keeps this exchange's symbols and norms in the workspace; sym_mode 2
+// adds sum_k ||Q(V_k) kept by the other slot - Q(V_k) of this exchange||^2 to *sum_sq (each worker's
+// own two quantized vectors, which the loss-less code reproduces exactly on the receiving side).
 qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
-                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int diff_slot, double* sum_sq) {
+                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int sym_mode, double* sum_sq) {
   if (!c || !cfg || !mean_out || K < 1 || K > 65535 || d < 1 || slot < 0 || slot > 1) return QGX_ERR_INVALID_ARG;
   const int bucket = cfg->bucket;
   if (bucket < kQuad || bucket > QGX_MAX_BUCKET || bucket % kQuad != 0) return QGX_ERR_INVALID_ARG;
@@ -545,7 +542,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   uint32_t* offs = (uint32_t*)ws_get(c, base + 2, sizeof(uint32_t) * (size_t)K * nb);
   unsigned long long* tot = (unsigned long long*)ws_get(c, base + 3, sizeof(uint64_t) * (size_t)K);
   unsigned long long* status = (unsigned long long*)ws_get(c, WS_STATUS, sizeof(uint64_t) * ((size_t)K * nb + 2));
-  float* norms = (float*)ws_get(c, WS_NORMS, sizeof(float) * (size_t)K * nb);
+  float* norms = (float*)ws_get(c, slot == 0 ? WS_NORMS : WS_NORMS2, sizeof(float) * (size_t)K * nb);
   DecEntry* lut = (DecEntry*)ws_get(c, WS_DLUT, sizeof(DecEntry) * (size_t)(2 * kDecLutMax));
   if (!stream || !bbits || !offs || !tot || !status || !norms || !lut) return QGX_ERR_CUDA;
   c->slot_cap_words[slot] = cap;
@@ -561,6 +558,16 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   ea.vec_ok = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(src.v) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
   ea.stream = stream; ea.cap_words = cap; ea.bucket_bits = bbits; ea.offsets = offs; ea.total_bits = tot; ea.norms = norms;
   ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(status + (size_t)K * nb); ea.st = c->dstatus;
+  ea.sym_out = nullptr; ea.sym_prev = nullptr; ea.norms_prev = nullptr; ea.sum_sq = sum_sq;
+  if (sym_mode == 1) {
+    ea.sym_out = (uint8_t*)ws_get(c, WS_SYM, (size_t)K * d + 16);
+    if (!ea.sym_out) return QGX_ERR_CUDA;
+    c->sym_slot = slot; c->sym_K = K; c->sym_d = d;
+  } else if (sym_mode == 2) {
+    if (!sum_sq || c->sym_slot != 1 - slot || c->sym_K != K || c->sym_d != d || c->slot_nb[1 - slot] != nb) return QGX_ERR_INVALID_ARG;
+    ea.sym_prev = (const uint8_t*)c->ws[WS_SYM];
+    ea.norms_prev = (const float*)c->ws[slot == 0 ? WS_NORMS2 : WS_NORMS];
+  }
   const PhiloxKey key = make_philox_key(cfg->seed);
   QuantTable qt;
   make_quant_table(cfg->levels, cfg->nlev, &qt);
@@ -570,20 +577,26 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const size_t img_words = (((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4;
   const size_t smem = sizeof(uint32_t) * img_words;
   int per_sm = 1;
-#define QGX_LAUNCH_E(V, GG)                                                                                    \
-  do {                                                                                                         \
-    cudaFuncSetAttribute(k_exchange_encode<V, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG>, threads, smem);           \
-    if (per_sm < 1) per_sm = 1;                                                                                \
-    const unsigned long long want = (unsigned long long)nb * (unsigned long long)K;                            \
-    const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);   \
-    k_exchange_encode<V, GG><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                          \
+#define QGX_LAUNCH_E(V, GG, SS)                                                                                  \
+  do {                                                                                                           \
+    cudaFuncSetAttribute(k_exchange_encode<V, GG, SS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG, SS>, threads, smem);         \
+    if (per_sm < 1) per_sm = 1;                                                                                  \
+    const unsigned long long want = (unsigned long long)nb * (unsigned long long)K;                              \
+    const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);     \
+    k_exchange_encode<V, GG, SS><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                        \
+  } while (0)
+#define QGX_LAUNCH_ES(V, GG)                               \
+  do {                                                     \
+    if (sym_mode == 1) QGX_LAUNCH_E(V, GG, 1);             \
+    else if (sym_mode == 2) QGX_LAUNCH_E(V, GG, 2);        \
+    else QGX_LAUNCH_E(V, GG, 0);                           \
   } while (0)
 #define QGX_LAUNCH_EG(V)                                   \
   do {                                                     \
-    if (ct.G == 32) QGX_LAUNCH_E(V, 32);                   \
-    else if (ct.G == 64) QGX_LAUNCH_E(V, 64);              \
-    else QGX_LAUNCH_E(V, 128);                             \
+    if (ct.G == 32) QGX_LAUNCH_ES(V, 32);                  \
+    else if (ct.G == 64) QGX_LAUNCH_ES(V, 64);             \
+    else QGX_LAUNCH_ES(V, 128);                            \
   } while (0)
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_ENCODE);
@@ -595,6 +608,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
     }
   }
 #undef QGX_LAUNCH_EG
+#undef QGX_LAUNCH_ES
 #undef QGX_LAUNCH_E
   count_launch(c);
   if (cudaGetLastError() != cudaSuccess) return QGX_ERR_CUDA;
@@ -622,53 +636,37 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
 
   DecodeArgs da;
   da.stream = stream; da.cap_words = cap; da.bucket_bits = bbits; da.offsets = offs;
-  da.stream2 = nullptr; da.cap_words2 = 0; da.bucket_bits2 = nullptr; da.offsets2 = nullptr; da.sum_sq = sum_sq;
-  bool diff = false;
-  if (diff_slot >= 0) {
-    if (diff_slot > 1 || diff_slot == slot || c->slot_K[diff_slot] != K || c->slot_nb[diff_slot] != nb || !sum_sq) return QGX_ERR_INVALID_ARG;
-    const int b2 = WS_SLOT0 + 4 * diff_slot;
-    da.stream2 = (const uint32_t*)c->ws[b2 + 0]; da.cap_words2 = c->slot_cap_words[diff_slot];
-    da.bucket_bits2 = (const uint32_t*)c->ws[b2 + 1]; da.offsets2 = (const uint32_t*)c->ws[b2 + 2];
-    diff = true;
-  }
   da.d = d; da.bucket = bucket; da.K = K; da.nb = nb; da.lut = lut; da.mean = mean_out;
   da.update = upd ? upd->mode : 0; da.xin = upd ? upd->xin : nullptr; da.xout = upd ? upd->xout : nullptr;
   da.scalars = upd ? upd->scalars : nullptr; da.st = c->dstatus;
-  return launch_decode_average(c, da, ct, diff);
+  return launch_decode_average(c, da, ct);
 }
 
 template <int G>
-static qgx_status launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, bool diff) {
+static qgx_status launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct) {
   const size_t total_sub = da.nb * ((size_t)da.bucket / G);
-  const size_t per_set = (sizeof(uint32_t) + sizeof(float)) * (size_t)da.K * kDecThreads;
-  const size_t smem = sizeof(DecEntry) * ((size_t)2 << ct.maxlen) + per_set * (diff ? 2 : 1);
+  const size_t smem = sizeof(DecEntry) * ((size_t)2 << ct.maxlen) + (sizeof(uint32_t) + sizeof(float)) * (size_t)da.K * kDecThreads;
   if (smem > 200 * 1024) return QGX_ERR_INVALID_ARG;   // too many workers for the per-thread positions
   int per_sm = 1;
-  if (diff) {
-    cudaFuncSetAttribute(k_exchange_decode<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, true>, kDecThreads, smem);
-  } else {
-    cudaFuncSetAttribute(k_exchange_decode<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, false>, kDecThreads, smem);
-  }
+  cudaFuncSetAttribute(k_exchange_decode<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G>, kDecThreads, smem);
   if (per_sm < 1) per_sm = 1;
   const size_t want = (total_sub + kDecThreads - 1) / kDecThreads;
   const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
-    if (diff) k_exchange_decode<G, true><<<grid, kDecThreads, smem, c->stream>>>(da, ct);
-    else k_exchange_decode<G, false><<<grid, kDecThreads, smem, c->stream>>>(da, ct);
+    k_exchange_decode<G><<<grid, kDecThreads, smem, c->stream>>>(da, ct);
   }
   count_launch(c);
   return cuda_status(cudaGetLastError());
 }
 
-qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, bool diff) {
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct) {
   if (!ct.has_header || da.bucket % ct.G != 0) return QGX_ERR_INVALID_ARG;
   switch (ct.G) {
-    case 32: return launch_decode_g<32>(c, da, ct, diff);
-    case 64: return launch_decode_g<64>(c, da, ct, diff);
-    case 128: return launch_decode_g<128>(c, da, ct, diff);
+    case 32: return launch_decode_g<32>(c, da, ct);
+    case 64: return launch_decode_g<64>(c, da, ct);
+    case 128: return launch_decode_g<128>(c, da, ct);
     default: return QGX_ERR_INVALID_ARG;
   }
 }
@@ -683,7 +681,7 @@ qgx_status qgx_exchange(qgx_ctx* c, const float* v, int K, size_t d, const qgx_q
                         int slot, float* mean_out, uint64_t* total_bits) {
   if (!v) return QGX_ERR_INVALID_ARG;
   DualSource src{v, nullptr};
-  return exchange_impl(c, src, K, d, cfg, exchange_id, slot, mean_out, total_bits, nullptr, -1, nullptr);
+  return exchange_impl(c, src, K, d, cfg, exchange_id, slot, mean_out, total_bits, nullptr, 0, nullptr);
 }
 
 qgx_status qgx_exchange_streams(qgx_ctx* c, int slot, const uint32_t** stream, size_t* cap_words,
