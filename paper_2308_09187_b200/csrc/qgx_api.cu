@@ -63,14 +63,15 @@ static int tau_of(const float* lev, int nlev, float u) {
 void make_quant_table(const float* lev, int nlev, QuantTable* out) {
   std::memset(out, 0, sizeof(*out));
   out->nlev = nlev;
-  for (int j = 0; j < 2 * QGX_MAX_LEVELS; ++j) out->upper[j] = (j <= nlev - 2) ? lev[j] : 3.0f;
+  for (int t = 0; t < QGX_MAX_LEVELS; ++t)
+    out->upper[t] = make_float2(t + 1 <= nlev - 2 ? lev[t + 1] : 3.0f, t + 2 <= nlev - 2 ? lev[t + 2] : 3.0f);
   for (int t = 0; t <= nlev - 2; ++t) {
     const float width = lev[t + 1] - lev[t];                       // the fp32 difference the exact routine divides by
     const double scale = 8388608.0 / (double)width;
-    const float margin = (float)(4.0 * (double)lev[t + 1] / (double)width + 8.0) * 1.0001f;
-    out->interval[t] = make_float4(lev[t], (float)scale, margin, 8388608.0f - margin);
+    const float margin = (float)(4.0 * (double)lev[t + 1] / (double)width + 10.0) * 1.0001f;
+    out->interval[t] = make_float4(lev[t], (float)scale, margin, 0.0f);
   }
-  for (int t = nlev - 1; t < QGX_MAX_LEVELS; ++t) out->interval[t] = make_float4(0.f, 0.f, 3.0e38f, -3.0e38f);   // never "safe"
+  for (int t = nlev - 1; t < QGX_MAX_LEVELS; ++t) out->interval[t] = make_float4(0.f, 0.f, 3.0e38f, 0.0f);   // never "safe"
   int steps = 0;
   for (int b = 0; b < kKeyBins; ++b) {
     // bin b holds patterns [(b + kKeyMin) << 17, (b + 1 + kKeyMin) << 17); bin 0 also everything below

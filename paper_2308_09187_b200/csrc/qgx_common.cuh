@@ -64,8 +64,8 @@ constexpr int kKeyBins = (0x3F800000 >> kKeyShift) - kKeyMin + 1;   // up to u =
 struct QuantTable {
   int nlev;
   int steps;                             // compare steps after the table look-up
-  float4 interval[QGX_MAX_LEVELS];       // {l_tau, 2^23 / (l_{tau+1} - l_tau), margin, 2^23 - margin}
-  float upper[2 * QGX_MAX_LEVELS];       // upper[j] = l_j for j <= nlev - 2, then a value above 1
+  float4 interval[QGX_MAX_LEVELS];       // {l_tau, 2^23 / (l_{tau+1} - l_tau), margin, unused}
+  float2 upper[QGX_MAX_LEVELS];          // upper[t] = {l_{t+1}, l_{t+2}} while those are interior levels, else a value above 1
   uint8_t start[kKeyBins + 3];
 };
 
@@ -146,7 +146,7 @@ static __device__ __noinline__ int quantize_level_slow(float absv, float norm, c
 // u' = RN(|v| rn) differs from the exact u = RN(|v| / norm) by at most 2^-22 u.  tau is found from a
 // table on the float pattern of u' plus two comparisons (tables that would need more send every
 // coordinate to the exact routine); T = (u' - l_tau) 2^23 / width differs from xi 2^23 by less than
-// margin = 4 l_{tau+1} / width + 8.  The 24-bit variate m rounds up iff m < xi 2^24; with m' = m >> 1
+// margin = 4 l_{tau+1} / width + 10.  The 24-bit variate m rounds up iff m < xi 2^24; with m' = m >> 1
 // taken as a float through the 2^23 trick, the sign of T - m' decides whenever |T - m'| > margin and T
 // is further than margin from both ends of the interval (so that u' and u lie in the same interval).
 // Returns the level index and sets *unsafe when the exact routine has to decide instead.
@@ -154,13 +154,15 @@ __device__ __forceinline__ int quantize_fast(float absv, float rn, const QuantTa
   const float u = fminf(__fmul_rn(absv, rn), 1.0f);
   const int key = max((int)(__float_as_uint(u) >> kKeyShift), kKeyMin) - kKeyMin;
   const int tau0 = q->start[key];
-  const int tau = tau0 + ((q->upper[tau0 + 1] <= u) ? 1 : 0) + ((q->upper[tau0 + 2] <= u) ? 1 : 0);
+  const float2 up = q->upper[tau0];
+  const int tau = tau0 + ((up.x <= u) ? 1 : 0) + ((up.y <= u) ? 1 : 0);
   const float4 iv = q->interval[tau];
-  const float T = __fmul_rn(__fsub_rn(u, iv.x), iv.y);
-  const float mhalf = __fsub_rn(__uint_as_float(0x4B000000u | (word >> 9)), 8388608.0f);   // (m >> 1), exact
-  const float diff = __fsub_rn(T, mhalf);
+  // T + 2^23: the addition rounds T to an integer (error 1/2, inside the margin)
+  const float Tb = fmaf(u - iv.x, iv.y, 8388608.0f);
+  const float mb = __uint_as_float(0x4B000000u | (word >> 9));                    // 2^23 + (m >> 1), exact
+  const float diff = Tb - mb;
   // a zero coordinate is level 0 whatever the variate (T = 0, diff <= 0), so it needs no second look
-  *unsafe = (absv != 0.0f) && !(fabsf(diff) > iv.z && T > iv.z && T < iv.w);
+  *unsafe = (absv != 0.0f) && !(fabsf(diff) > iv.z && fabsf(Tb - 12582912.0f) < 4194304.0f - iv.z);
   return tau + (diff > 0.0f ? 1 : 0);
 }
 
