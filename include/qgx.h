@@ -39,7 +39,8 @@ typedef enum {
   QGX_ERR_CORRUPT = 4,      /* a stream that no encoder could have produced */
   QGX_ERR_NONFINITE = 5,    /* a bucket norm is NaN or infinite */
   QGX_ERR_TIMEOUT = 6,      /* a bounded device-side wait ran out */
-  QGX_ERR_CUDA = 7          /* the CUDA runtime reported an error */
+  QGX_ERR_CUDA = 7,         /* the CUDA runtime reported an error */
+  QGX_ERR_TOO_LARGE = 8     /* the problem exceeds the fixed scratch of qgx_encode_noalloc */
 } qgx_status;
 
 enum { QGX_NORM_L2 = 0, QGX_NORM_LINF = 1 };
@@ -174,6 +175,27 @@ qgx_status qgx_quantize(qgx_ctx *ctx, const float *v, int K, size_t d, int bucke
 qgx_status qgx_encode(qgx_ctx *ctx, const float *norms, const uint8_t *sym, int K, size_t d,
                       int bucket, const qgx_codebook *cb /*[host]*/, uint32_t *stream,
                       size_t cap_words, uint32_t *bucket_bits, uint64_t *total_bits);
+
+/* qgx_encode for callers that must not allocate device memory.  (The paper has no counterpart: this is
+ * a packaging variant of the call above, not another method.)  Who needs it: code that runs where
+ * cudaMalloc is off limits -- a communication hook or an inner loop that is being recorded into a CUDA
+ * stream capture, a process whose memory is handed out up front by a pool or a scheduler, or a library
+ * embedded in another runtime that forbids allocations after start-up.  qgx_encode keeps the buckets'
+ * word offsets and per-worker overflow flags in a workspace that it grows with cudaMalloc; this entry
+ * point keeps them in a fixed array inside the library image instead (about 516 KB, present on every GPU
+ * that loads the library until the process ends) and calls no cudaMalloc, cudaFree or other allocating
+ * routine.  Arguments, stream layout, outputs and device-side errors are those of qgx_encode; the results
+ * are identical.
+ *  - Limits: K <= 1024 and K * nb <= 65536 buckets; beyond that the call returns QGX_ERR_TOO_LARGE and
+ *    launches nothing.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ *    device current); make that first call before any stream capture begins.
+ *  - All calls on a device share the one array and find in it what the previous call left; the call
+ *    overwrites everything it reads.  Two calls that overlap on the GPU (different streams or contexts)
+ *    race on it: run them one after the other. */
+qgx_status qgx_encode_noalloc(qgx_ctx *ctx, const float *norms, const uint8_t *sym, int K, size_t d,
+                              int bucket, const qgx_codebook *cb /*[host]*/, uint32_t *stream,
+                              size_t cap_words, uint32_t *bucket_bits, uint64_t *total_bits);
 
 /* DEQ o CODE: the exact inverse of qgx_encode, driven by bucket_bits.  Every read is bounded by
  * the bucket's length; a codeword that runs past it, an unassigned bit pattern, a sub-block whose

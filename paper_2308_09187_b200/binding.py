@@ -14,7 +14,7 @@ from . import build as _build
 
 QGX_OK = 0
 QGX_ERR_INVALID_ARG, QGX_ERR_BAD_LEVELS, QGX_ERR_CAPACITY, QGX_ERR_CORRUPT = 1, 2, 3, 4
-QGX_ERR_NONFINITE, QGX_ERR_TIMEOUT, QGX_ERR_CUDA = 5, 6, 7
+QGX_ERR_NONFINITE, QGX_ERR_TIMEOUT, QGX_ERR_CUDA, QGX_ERR_TOO_LARGE = 5, 6, 7, 8
 QGX_NORM_L2, QGX_NORM_LINF = 0, 1
 QGX_CODE_FIXED, QGX_CODE_HUFFMAN = 0, 1
 QGX_OP_DENSE_AFFINE, QGX_OP_BILINEAR, QGX_OP_DIAGONAL = 0, 1, 2
@@ -29,6 +29,7 @@ EXPORTS = [
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
     "qgx_eg_init", "qgx_eg_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
+    "qgx_encode_noalloc",
 ]
 QGX_KERNEL_ENCODE, QGX_KERNEL_DECODE, QGX_KERNEL_HISTOGRAM, QGX_KERNEL_OPERATOR, QGX_KERNEL_FINISH = range(5)
 
@@ -255,6 +256,16 @@ def qgx_encode(ctx, norms, sym, bucket, cb, cap_words=None, stream=None, bucket_
         total_bits = torch.empty((K,), dtype=torch.int64, device=sym.device)
     _chk(lib().qgx_encode(ctx.h, _ptr(norms), _ptr(sym), K, C.c_size_t(d), bucket, C.byref(cb), _ptr(stream),
                           C.c_size_t(cap_words), _ptr(bucket_bits), _ptr(total_bits)), "qgx_encode")
+    return stream, bucket_bits, total_bits
+
+
+def qgx_encode_noalloc(ctx, norms, sym, bucket, cb, stream, bucket_bits, total_bits):
+    """qgx_encode without any device allocation: for callers that cannot call cudaMalloc (code inside a
+    stream capture, processes whose memory is handed out once at start-up).  Every buffer, outputs
+    included, is the caller's; this wrapper allocates nothing either.  Limits: K <= 1024, K * nb <= 65536."""
+    K, d = sym.shape
+    _chk(lib().qgx_encode_noalloc(ctx.h, _ptr(norms), _ptr(sym), K, C.c_size_t(d), bucket, C.byref(cb), _ptr(stream),
+                                  C.c_size_t(stream.shape[1]), _ptr(bucket_bits), _ptr(total_bits)), "qgx_encode_noalloc")
     return stream, bucket_bits, total_bits
 
 

@@ -177,6 +177,7 @@ const char* qgx_status_str(qgx_status s) {
     case QGX_ERR_NONFINITE: return "non-finite bucket norm";
     case QGX_ERR_TIMEOUT: return "device-side wait ran out";
     case QGX_ERR_CUDA: return "CUDA runtime error";
+    case QGX_ERR_TOO_LARGE: return "problem larger than the fixed scratch of the no-allocation entry point";
   }
   return "unknown status";
 }

@@ -3,9 +3,18 @@
 #include "qgx_bucket.cuh"
 #include "qgx_codec.cuh"
 
+#include <mutex>
 #include <vector>
 
 namespace qgx {
+
+// Scratch of qgx_encode_noalloc: bucket word offsets (u64 per bucket) followed by one overflow flag per
+// worker.  It lives in the library image, so every GPU that loads the library carries these bytes
+// until the process exits.
+constexpr size_t kNoAllocMaxBuckets = 65536;            // K * nb
+constexpr size_t kNoAllocMaxWorkers = 1024;             // K
+constexpr size_t kNoAllocBytes = kNoAllocMaxBuckets * sizeof(uint64_t) + kNoAllocMaxWorkers * sizeof(uint32_t);
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
 void build_dec_lut_host(const CodeTable& ct, uint16_t* lut) {
   const int n = 1 << ct.maxlen;
@@ -334,6 +343,70 @@ qgx_status qgx_decode(qgx_ctx* c, const uint32_t* stream, size_t cap_words, cons
   k_decode<<<grid, threads, smem, c->stream>>>(stream, cap_words, bucket_bits, off, flags, d, bucket, ct, lut, vec_ok, norms,
                                                sym, c->dstatus);
   count_launch(c, 2);
+  return cuda_status(cudaGetLastError());
+}
+
+
+// Device address of g_noalloc_scratch on the current device.  In host code the array's name only stands
+// in for the symbol; the address a kernel can use has to be asked for, once per device.
+static qgx_status noalloc_scratch_address(int device, unsigned char** out) {
+  static std::mutex mu;
+  static unsigned char* addr[64] = {nullptr};
+  if (device < 0 || device >= 64) return QGX_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(mu);
+  if (addr[device] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return QGX_ERR_CUDA;
+    }
+    addr[device] = static_cast<unsigned char*>(p);
+  }
+  *out = addr[device];
+  return QGX_OK;
+}
+
+qgx_status qgx_encode_noalloc(qgx_ctx* c, const float* norms, const uint8_t* sym, int K, size_t d, int bucket,
+                              const qgx_codebook* cb, uint32_t* stream, size_t cap_words, uint32_t* bucket_bits,
+                              uint64_t* total_bits) {
+  if (!codec_args_ok(c, K, d, bucket) || !norms || !sym || !stream || !bucket_bits || !total_bits) return QGX_ERR_INVALID_ARG;
+  const size_t nb = (d + (size_t)bucket - 1) / (size_t)bucket;
+  if ((size_t)K > kNoAllocMaxWorkers || (size_t)K * nb > kNoAllocMaxBuckets) return QGX_ERR_TOO_LARGE;
+  CodeTable ct;
+  qgx_status rc = make_code_table(cb, bucket, &ct);
+  if (rc != QGX_OK) return rc;
+  if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
+  unsigned char* scratch = nullptr;
+  rc = noalloc_scratch_address(c->device, &scratch);
+  if (rc != QGX_OK) return rc;
+  uint64_t* off = reinterpret_cast<uint64_t*>(scratch);
+  uint32_t* flags = reinterpret_cast<uint32_t*>(scratch + kNoAllocMaxBuckets * sizeof(uint64_t));
+  // Nothing in the scratch has to start at zero: the scan kernel writes every offset and every flag
+  // that the scatter kernel reads.  The flags are cleared all the same, so that a stale "overflow"
+  // of an earlier call can never be seen.
+  if (cudaMemsetAsync(flags, 0, sizeof(uint32_t) * (size_t)K, c->stream) != cudaSuccess) return QGX_ERR_CUDA;
+  const bool vec_ok = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(sym) & 3u) == 0);
+  const int v4 = bucket_v4(bucket);
+  const int threads = bucket_threads(bucket, v4);
+  const dim3 grid((unsigned)nb, (unsigned)K);
+  k_bucket_bits<<<grid, threads, 0, c->stream>>>(sym, d, bucket, ct, vec_ok, bucket_bits, c->dstatus);
+  k_scan_offsets<<<K, 256, 0, c->stream>>>(bucket_bits, nb, cap_words, off, total_bits, flags, QGX_ERR_CAPACITY, c->dstatus);
+  const size_t img_words = (((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4;
+  const size_t smem = sizeof(uint32_t) * (img_words + (size_t)(bucket / ct.G) + 2);
+#define QGX_LAUNCH_S(V)                                                                                         \
+  do {                                                                                                          \
+    cudaFuncSetAttribute(k_bit_scatter<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);             \
+    k_bit_scatter<V><<<grid, threads, smem, c->stream>>>(norms, sym, d, bucket, ct, vec_ok, stream, cap_words,  \
+                                                         bucket_bits, off, flags);                              \
+  } while (0)
+  switch (v4) {
+    case 1: QGX_LAUNCH_S(1); break;
+    case 2: QGX_LAUNCH_S(2); break;
+    case 4: QGX_LAUNCH_S(4); break;
+    default: QGX_LAUNCH_S(8); break;
+  }
+#undef QGX_LAUNCH_S
+  count_launch(c, 3);
   return cuda_status(cudaGetLastError());
 }
 
