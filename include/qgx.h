@@ -217,6 +217,19 @@ qgx_status qgx_average(qgx_ctx *ctx, const float *norms, const uint8_t *sym, int
  * the two exchanges of one iteration can both be kept). */
 qgx_status qgx_exchange(qgx_ctx *ctx, const float *v, int K, size_t d, const qgx_quant_cfg *cfg /*[host]*/,
                         uint32_t exchange_id, int slot, float *mean_out, uint64_t *total_bits);
+/* Layer-wise exchange: v [dev] float[K][d] holds nseg tensors back to back (segment s = coordinates
+ * [offset, offset + length) of every worker, offsets multiples of 4, the segments tiling [0, d) in order);
+ * every segment is exchanged with its own table and code (segs[s].cfg), buckets never cross a segment, and
+ * coordinate offset + i of worker k uses the generator counter of coordinate offset + i.  mean_out [dev]
+ * float[d]; total_bits [dev] uint64[K] (may be NULL) receives the stream bits summed over segments.  The
+ * streams of one segment are overwritten by the next (slot 0 of the workspace). */
+typedef struct {
+  size_t offset;
+  size_t length;
+  const qgx_quant_cfg *cfg;   /* [host] */
+} qgx_segment;
+qgx_status qgx_exchange_segments(qgx_ctx *ctx, const float *v, int K, size_t d, const qgx_segment *segs /*[host]*/,
+                                 int nseg, uint32_t exchange_id, float *mean_out, uint64_t *total_bits);
 /* Where the last qgx_exchange on `slot` left its streams: all [dev], valid until the next call
  * that uses the slot.  Any output pointer may be NULL. */
 qgx_status qgx_exchange_streams(qgx_ctx *ctx, int slot, const uint32_t **stream, size_t *cap_words,

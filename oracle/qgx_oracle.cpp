@@ -242,9 +242,12 @@ int qgxo_bucket_norms(const float* v, int K, uint64_t d, int bucket, int norm_ty
 }
 
 // ------------------------------- quantize ------------------------------------------
-// sym[k][i] from v[k][i], the bucket norms and the Philox word of (seed, k, xid, i).
-int qgxo_quantize(const float* v, int K, uint64_t d, int bucket, const float* lev, int nlev,
-                  const float* norms, uint64_t seed, uint32_t xid, uint8_t* sym) {
+// sym[k][i] from v[k][i], the bucket norms and the Philox word of (seed, k, xid, coord_base + i).
+// coord_base is where this vector starts inside a longer layer-wise dual vector (0 for a vector on its own):
+// each tensor is quantized on its own (its own buckets, norms and levels), only the variates are indexed
+// by the position in the whole vector.
+int qgxo_quantize_at(const float* v, int K, uint64_t d, int bucket, const float* lev, int nlev,
+                     const float* norms, uint64_t seed, uint32_t xid, uint64_t coord_base, uint8_t* sym) {
   if (K < 1 || bucket < 1) return INVALID_ARG;
   if (!levels_ok(lev, nlev)) return BAD_LEVELS;
   const uint64_t nb = n_buckets(d, bucket);
@@ -252,9 +255,14 @@ int qgxo_quantize(const float* v, int K, uint64_t d, int bucket, const float* le
     for (uint64_t i = 0; i < d; ++i) {
       const float norm = norms[(uint64_t)k * nb + i / (uint64_t)bucket];
       sym[(uint64_t)k * d + i] =
-          quantize_element(v[(uint64_t)k * d + i], norm, lev, nlev, element_word(seed, (uint32_t)k, xid, i));
+          quantize_element(v[(uint64_t)k * d + i], norm, lev, nlev, element_word(seed, (uint32_t)k, xid, coord_base + i));
     }
   return OK;
+}
+
+int qgxo_quantize(const float* v, int K, uint64_t d, int bucket, const float* lev, int nlev,
+                  const float* norms, uint64_t seed, uint32_t xid, uint8_t* sym) {
+  return qgxo_quantize_at(v, K, d, bucket, lev, nlev, norms, seed, xid, 0, sym);
 }
 
 // Same, with the random words supplied by the caller (words[k][i]); used to enumerate outcomes.

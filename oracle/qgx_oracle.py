@@ -138,14 +138,15 @@ def bucket_norms(v, bucket, norm_type=L2, allow_nonfinite=False):
     return norms
 
 
-def quantize(v, bucket, levels, norms, seed, xid):
+def quantize(v, bucket, levels, norms, seed, xid, coord_base=0):
+    """coord_base: index of v's first coordinate inside a longer layer-wise vector (variates only)."""
     v = _f32(v)
     lv = _f32(levels)
     norms = _f32(norms)
     K, d = v.shape
     sym = np.zeros((K, d), dtype=np.uint8)
-    _chk(lib().qgxo_quantize(_p(v), K, C.c_uint64(d), bucket, _p(lv), len(lv), _p(norms),
-                             C.c_uint64(seed), C.c_uint32(xid), _p(sym)), "quantize")
+    _chk(lib().qgxo_quantize_at(_p(v), K, C.c_uint64(d), bucket, _p(lv), len(lv), _p(norms),
+                                C.c_uint64(seed), C.c_uint32(xid), C.c_uint64(coord_base), _p(sym)), "quantize")
     return sym
 
 

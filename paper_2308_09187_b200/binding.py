@@ -29,7 +29,7 @@ EXPORTS = [
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
     "qgx_eg_init", "qgx_eg_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
-    "qgx_encode_noalloc",
+    "qgx_encode_noalloc", "qgx_exchange_segments",
 ]
 QGX_KERNEL_ENCODE, QGX_KERNEL_DECODE, QGX_KERNEL_HISTOGRAM, QGX_KERNEL_OPERATOR, QGX_KERNEL_FINISH = range(5)
 
@@ -298,6 +298,27 @@ def qgx_exchange(ctx, v, cfg, exchange_id, slot=0, mean_out=None, total_bits=Non
         total_bits = torch.empty((K,), dtype=torch.int64, device=v.device)
     _chk(lib().qgx_exchange(ctx.h, _ptr(v), K, C.c_size_t(d), C.byref(cfg), C.c_uint32(exchange_id), slot,
                             _ptr(mean_out), _ptr(total_bits)), "qgx_exchange")
+    return mean_out, total_bits
+
+
+class qgx_segment(C.Structure):
+    _fields_ = [("offset", C.c_size_t), ("length", C.c_size_t), ("cfg", C.POINTER(qgx_quant_cfg))]
+
+
+def qgx_exchange_segments(ctx, v, sizes, cfgs, exchange_id, mean_out=None, total_bits=None):
+    """sizes[s] coordinates per tensor (laid back to back in v[K, sum(sizes)]), cfgs[s] its qgx_quant_cfg."""
+    K, d = v.shape
+    if mean_out is None:
+        mean_out = torch.empty((d,), dtype=torch.float32, device=v.device)
+    if total_bits is None:
+        total_bits = torch.empty((K,), dtype=torch.int64, device=v.device)
+    segs = (qgx_segment * len(sizes))()
+    at = 0
+    for s, (n, cfg) in enumerate(zip(sizes, cfgs)):
+        segs[s].offset, segs[s].length, segs[s].cfg = at, n, C.pointer(cfg)
+        at += n
+    _chk(lib().qgx_exchange_segments(ctx.h, _ptr(v), K, C.c_size_t(d), segs, len(sizes), C.c_uint32(exchange_id),
+                                     _ptr(mean_out), _ptr(total_bits)), "qgx_exchange_segments")
     return mean_out, total_bits
 
 

@@ -27,11 +27,13 @@ inline int bucket_v4(int bucket) {
 struct DualSource {
   const float* v;        // [K][d] plain vectors, or the noise U; may be null when a is given
   const float* a;        // [d] operator value A(x) shared by all workers; null for plain vectors
+  size_t ld;             // distance between workers' rows of v in floats; 0 means d
 };
 
 __device__ __forceinline__ float dual_value(const DualSource& s, size_t k, size_t d, size_t i) {
-  if (s.a == nullptr) return s.v[k * d + i];
-  return s.v ? __fadd_rn(s.a[i], s.v[k * d + i]) : s.a[i];
+  const size_t ld = s.ld ? s.ld : d;
+  if (s.a == nullptr) return s.v[k * ld + i];
+  return s.v ? __fadd_rn(s.a[i], s.v[k * ld + i]) : s.a[i];
 }
 
 template <int V4>
@@ -44,17 +46,18 @@ struct BucketRegs {
 template <int V4>
 __device__ __forceinline__ void load_bucket(BucketRegs<V4>& r, const DualSource& s, size_t k, size_t d,
                                             size_t lo, int len, bool vec_ok) {
+  const size_t ld = s.ld ? s.ld : d;
 #pragma unroll
   for (int j = 0; j < V4; ++j) {
     const int e = (j * (int)blockDim.x + (int)threadIdx.x) * kQuad;
     float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
     if (e + kQuad <= len && vec_ok) {
       if (s.a == nullptr) {
-        x = __ldcs(reinterpret_cast<const float4*>(s.v + k * d + lo + e));
+        x = __ldcs(reinterpret_cast<const float4*>(s.v + k * ld + lo + e));
       } else {
         const float4 a = __ldg(reinterpret_cast<const float4*>(s.a + lo + e));
         if (s.v) {
-          const float4 u = __ldcs(reinterpret_cast<const float4*>(s.v + k * d + lo + e));
+          const float4 u = __ldcs(reinterpret_cast<const float4*>(s.v + k * ld + lo + e));
           x = make_float4(__fadd_rn(a.x, u.x), __fadd_rn(a.y, u.y), __fadd_rn(a.z, u.z), __fadd_rn(a.w, u.w));
         } else {
           x = a;

@@ -7,7 +7,8 @@ namespace qgx {
 
 // declared in qgx_exchange.cu / qgx_levels.cu
 qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
-                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int sym_mode, double* sum_sq);
+                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int sym_mode, double* sum_sq,
+                         uint64_t coord_base);
 qgx_status refit_from_source(qgx_ctx* c, DualSource src, int K, size_t d, qgx_quant_cfg* cfg, int refit, double* hist,
                              double* hist_host);
 enum { WS_OPVAL = 15, WS_MEAN = 16, WS_HIST = 17 };
@@ -154,7 +155,7 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
 
   qgx_status rc = apply_operator_impl(c, op, st->X, a);                      // A(X_t)
   if (rc != QGX_OK) return rc;
-  DualSource src{noise_t, a};                                                // V_{k,t} = A(X_t) + U_{k,t}
+  DualSource src{noise_t, a, 0};                                                // V_{k,t} = A(X_t) + U_{k,t}
   if (refit != QGX_REFIT_NONE) {
     double* hist = (double*)ws_get(c, WS_HIST, sizeof(double) * (size_t)std::max(cfg->nbins, 1));
     if (!hist) return QGX_ERR_CUDA;
@@ -163,13 +164,13 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
   }
   const uint32_t xid = 2u * (uint32_t)st->t;
   ExchangeUpdate half{1, st->X, st->Xhalf, st->scalars};                      // X_{t+1/2} = X_t - gamma_t * mean
-  rc = exchange_impl(c, src, K, d, cfg, xid, 0, mean, bits, &half, 1, nullptr);
+  rc = exchange_impl(c, src, K, d, cfg, xid, 0, mean, bits, &half, 1, nullptr, 0);
   if (rc != QGX_OK) return rc;
   rc = apply_operator_impl(c, op, st->Xhalf, a);                              // A(X_{t+1/2})
   if (rc != QGX_OK) return rc;
-  DualSource src2{noise_half, a};
+  DualSource src2{noise_half, a, 0};
   ExchangeUpdate dual{2, st->Y, st->Y, st->scalars};                          // Y_{t+1} = Y_t - mean
-  rc = exchange_impl(c, src2, K, d, cfg, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 2, st->scalars);
+  rc = exchange_impl(c, src2, K, d, cfg, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 2, st->scalars, 0);
   if (rc != QGX_OK) return rc;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);

@@ -65,6 +65,7 @@ struct EncodeArgs {
   size_t nb;
   int norm_type;
   uint32_t xid;
+  uint64_t quad_base;           // (index of the vector's first coordinate in the generator's counter space) / 4
   bool vec_ok;
   uint32_t* stream;
   size_t cap_words;
@@ -189,7 +190,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
       const int nvalid = max(0, min(kQuad, len - q * kQuad));
       uint32_t sym4 = 0;
       if (nvalid > 0 && finite && norm != 0.0f) {
-        const uint64_t ctr = (uint64_t)(lo >> 2) + (uint64_t)q;
+        const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + (uint64_t)q;
         const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
         sym4 = quad_symbols(r.x[j], quantize_quad(r.x[j], w, rn, norm, &s_q, s_lev, nlev));
       }
@@ -511,7 +512,12 @@ namespace qgx {
 
 // workspace slots of a context
 enum { WS_OFF64 = 0, WS_FLAGS = 1, WS_LUT = 2, WS_SLOT0 = 3 /* stream, bits, offsets, total: 3..6 and 7..10 */,
-       WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18 };
+       WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18, WS_SEGBITS = 19 };
+
+__global__ void k_add_u64(uint64_t* acc, const uint64_t* x, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) acc[i] += x[i];
+}
 
 qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct);
 
@@ -519,7 +525,9 @@ qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeT
 // adds sum_k ||Q(V_k) kept by the other slot - Q(V_k) of this exchange||^2 to *sum_sq (each worker's
 // own two quantized vectors, which the loss-less code reproduces exactly on the receiving side).
 qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
-                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int sym_mode, double* sum_sq) {
+                         float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int sym_mode, double* sum_sq,
+                         uint64_t coord_base) {
+  if (coord_base % kQuad != 0) return QGX_ERR_INVALID_ARG;
   if (!c || !cfg || !mean_out || K < 1 || K > 65535 || d < 1 || slot < 0 || slot > 1) return QGX_ERR_INVALID_ARG;
   const int bucket = cfg->bucket;
   if (bucket < kQuad || bucket > QGX_MAX_BUCKET || bucket % kQuad != 0) return QGX_ERR_INVALID_ARG;
@@ -554,8 +562,8 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
     return QGX_ERR_CUDA;
 
   EncodeArgs ea;
-  ea.src = src; ea.d = d; ea.bucket = bucket; ea.K = K; ea.nb = nb; ea.norm_type = cfg->norm_type; ea.xid = xid;
-  ea.vec_ok = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(src.v) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
+  ea.src = src; ea.d = d; ea.bucket = bucket; ea.K = K; ea.nb = nb; ea.norm_type = cfg->norm_type; ea.xid = xid; ea.quad_base = coord_base / kQuad;
+  ea.vec_ok = (d % kQuad == 0) && (src.ld % kQuad == 0) && ((reinterpret_cast<uintptr_t>(src.v) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
   ea.stream = stream; ea.cap_words = cap; ea.bucket_bits = bbits; ea.offsets = offs; ea.total_bits = tot; ea.norms = norms;
   ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(status + (size_t)K * nb); ea.st = c->dstatus;
   ea.sym_out = nullptr; ea.sym_prev = nullptr; ea.norms_prev = nullptr; ea.sum_sq = sum_sq;
@@ -680,8 +688,38 @@ extern "C" {
 qgx_status qgx_exchange(qgx_ctx* c, const float* v, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t exchange_id,
                         int slot, float* mean_out, uint64_t* total_bits) {
   if (!v) return QGX_ERR_INVALID_ARG;
-  DualSource src{v, nullptr};
-  return exchange_impl(c, src, K, d, cfg, exchange_id, slot, mean_out, total_bits, nullptr, 0, nullptr);
+  DualSource src{v, nullptr, 0};
+  return exchange_impl(c, src, K, d, cfg, exchange_id, slot, mean_out, total_bits, nullptr, 0, nullptr, 0);
+}
+
+qgx_status qgx_exchange_segments(qgx_ctx* c, const float* v, int K, size_t d, const qgx_segment* segs, int nseg,
+                                 uint32_t exchange_id, float* mean_out, uint64_t* total_bits) {
+  if (!c || !v || !segs || nseg < 1 || !mean_out || K < 1) return QGX_ERR_INVALID_ARG;
+  // the segments must tile [0, d) in order, each starting on a multiple of 4 coordinates
+  size_t at = 0;
+  for (int s = 0; s < nseg; ++s) {
+    if (segs[s].offset != at || segs[s].length < 1 || segs[s].offset % kQuad != 0 || !segs[s].cfg) return QGX_ERR_INVALID_ARG;
+    at += segs[s].length;
+  }
+  if (at != d) return QGX_ERR_INVALID_ARG;
+  if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
+  uint64_t* seg_bits = nullptr;
+  if (total_bits) {
+    seg_bits = (uint64_t*)ws_get(c, WS_SEGBITS, sizeof(uint64_t) * (size_t)K);
+    if (!seg_bits) return QGX_ERR_CUDA;
+    if (cudaMemsetAsync(total_bits, 0, sizeof(uint64_t) * (size_t)K, c->stream) != cudaSuccess) return QGX_ERR_CUDA;
+  }
+  for (int s = 0; s < nseg; ++s) {
+    DualSource src{v + segs[s].offset, nullptr, d};
+    qgx_status rc = exchange_impl(c, src, K, segs[s].length, segs[s].cfg, exchange_id, 0, mean_out + segs[s].offset, seg_bits,
+                                  nullptr, 0, nullptr, segs[s].offset);
+    if (rc != QGX_OK) return rc;
+    if (total_bits) {
+      k_add_u64<<<(K + 255) / 256, 256, 0, c->stream>>>(total_bits, seg_bits, K);
+      count_launch(c);
+    }
+  }
+  return cuda_status(cudaGetLastError());
 }
 
 qgx_status qgx_exchange_streams(qgx_ctx* c, int slot, const uint32_t** stream, size_t* cap_words,

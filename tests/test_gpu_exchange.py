@@ -116,3 +116,40 @@ def test_fused_capacity_and_nonfinite(q):
     bad = qgx.make_quant_cfg(lev, bucket, qgx.qgx_build_codebook_fixed(9, 96), 5)      # 96 is not a fused sub-block size
     with pytest.raises(qgx.QgxError):
         qgx.qgx_exchange(ctx, v, bad, 0, slot=0)
+
+
+def test_layerwise_segments_c3_shape(q):
+    """c3 at reduced size: tensors of different sizes (one a partial bucket), heavy tails, per-tensor scales,
+    per-tensor fitted tables and Huffman codes, K = 16, bucket 4096."""
+    qgx, ctx = q
+    sizes = [1728, 36864, 73728, 1728, 147456]
+    lw = gen.c3_layerwise(K=16, sizes=sizes, device="cuda")
+    K, d = lw.v.shape
+    vh = lw.v.cpu().numpy()
+    cfgs, at = [], 0
+    for n in sizes:
+        cfg = qgx.make_quant_cfg(np.linspace(0, 1, lw.nlev), lw.bucket, qgx.qgx_build_codebook_fixed(lw.nlev, 128), lw.seed,
+                                 code_type=qgx.QGX_CODE_HUFFMAN)
+        qgx.qgx_update_levels(ctx, lw.v[:, at:at + n].contiguous(), cfg, qgx.QGX_REFIT_FIRST)
+        cfgs.append(cfg)
+        at += n
+    mean, total = qgx.qgx_exchange_segments(ctx, lw.v, sizes, cfgs, 9)
+    qgx.qgx_sync_status(ctx)
+    mean_h = mean.cpu().numpy()
+    bits_ref = np.zeros(K, dtype=np.uint64)
+    at = 0
+    for n, cfg in zip(sizes, cfgs):
+        part = np.ascontiguousarray(vh[:, at:at + n])
+        lev = np.array(cfg.level_list(), dtype=np.float32)
+        cbo = o.codebook_from(cfg.cb.lengths(), cfg.cb.codes(), subblock=128)
+        norms = o.bucket_norms(part, lw.bucket)
+        sym = o.quantize(part, lw.bucket, lev, norms, lw.seed, 9, coord_base=at)
+        _, _, tb = o.encode(norms, sym, lw.bucket, cbo)
+        bits_ref += tb
+        ref = o.average(norms, sym, lw.bucket, lev)
+        scale = float(norms.max())
+        assert np.max(np.abs(mean_h[at:at + n] - ref)) <= 1e-5 * scale
+        assert np.count_nonzero(mean_h[at:at + n] != ref) <= max(1, int(1e-6 * K * n) * K)
+        at += n
+    assert np.array_equal(total.cpu().numpy().astype(np.uint64), bits_ref) or \
+        np.max(np.abs(total.cpu().numpy().astype(np.int64) - bits_ref.astype(np.int64))) <= 16

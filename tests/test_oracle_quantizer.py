@@ -235,3 +235,15 @@ def test_dequantize_and_average_by_hand():
     lev9 = np.linspace(0, 1, 9, dtype=np.float32)
     m = o.average(nv, o.quantize(v, 16, lev9, nv, seed=4, xid=0), 16, lev9)
     assert np.max(np.abs(m - v[0])) < 0.06 * float(nv[0, 0])
+
+
+def test_coordinate_base_only_shifts_the_variates():
+    # a tensor inside a layer-wise vector: same buckets, norms and levels; variates of coordinates base + i
+    rng = np.random.default_rng(31)
+    v = rng.standard_normal((2, 300)).astype(np.float32)
+    lev = np.linspace(0, 1, 9, dtype=np.float32)
+    whole = o.quantize(v, 100, lev, o.bucket_norms(v, 100), seed=8, xid=2)
+    part = v[:, 100:300].copy()
+    at = o.quantize(part, 100, lev, o.bucket_norms(part, 100), seed=8, xid=2, coord_base=100)
+    assert np.array_equal(at, whole[:, 100:300])
+    assert not np.array_equal(o.quantize(part, 100, lev, o.bucket_norms(part, 100), seed=8, xid=2), at)
