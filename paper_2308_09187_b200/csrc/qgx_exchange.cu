@@ -322,6 +322,7 @@ struct DecodeArgs {
   const float* xin;
   float* xout;
   const double* scalars;        // scalars[1] = gamma_t
+  bool vec_out;                 // d % 4 == 0 and mean, xin, xout 16-byte aligned: 128-bit stores
   DevStatus* st;
 };
 
@@ -333,20 +334,21 @@ constexpr uint32_t kStateStep = 1u - (1u << 18);   // adding L * step moves the 
 // of the fused path lie in the context's workspace, which extends past every bucket, so a read a
 // few words beyond a (corrupt) sub-block stays inside allocated memory.
 struct Window {
-  const uint32_t* next;
+  const uint32_t* next;   // address of `ahead`
   uint32_t lo, hi;
+  uint32_t ahead;         // the word after the window, fetched one refill early
   int avail;
-  __device__ __forceinline__ void open(const uint32_t* words, uint32_t bitpos) {
-    const uint32_t* p = words + (bitpos >> 5);
-    const uint32_t sh = bitpos & 31u;
-    const uint32_t w0 = p[0], w1 = p[1];
+  // p = address of the word that holds the first bit, w0..w2 = p[0..2], sh = first bit within w0
+  __device__ __forceinline__ void open(const uint32_t* p, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t sh) {
     lo = __funnelshift_r(w0, w1, sh);
     hi = w1 >> sh;
     avail = 64 - (int)sh;                               // the window ends on a word boundary
+    ahead = w2;
     next = p + 2;
   }
   __device__ __forceinline__ void refill() {            // needs avail <= 32
-    const uint32_t w = *next++;
+    const uint32_t w = ahead;
+    ahead = *++next;                                    // not needed before the next refill
     lo |= __funnelshift_lc(0u, w, (uint32_t)avail);     // w << avail, nothing when avail == 32
     hi |= __funnelshift_lc(w, 0u, (uint32_t)avail);     // the bits of w that do not fit the low word
     avail += 32;
@@ -461,12 +463,22 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
       float acc[kDecChunk];
 #pragma unroll
       for (int i = 0; i < kDecChunk; ++i) acc[i] = 0.0f;
+      // worker k + 1's position, norm and first words are fetched while worker k is decoded
+      uint32_t n_state = s_state[tid];
+      float n_norm = s_norm[tid];
+      const uint32_t* n_p = a.stream + a.offsets[b] + ((n_state & 0x3ffffu) >> 5);
+      uint32_t n_w0 = n_p[0], n_w1 = n_p[1], n_w2 = n_p[2];
       for (int k = 0; k < a.K; ++k) {
-        const size_t kb = (size_t)k * a.nb + b;
-        const float norm = s_norm[k * kDecThreads + tid];
-        uint32_t state = s_state[k * kDecThreads + tid];
+        uint32_t state = n_state;
+        const float norm = n_norm;
         Window win;
-        win.open(a.stream + (size_t)k * a.cap_words + a.offsets[kb], state & 0x3ffffu);
+        win.open(n_p, n_w0, n_w1, n_w2, state & 31u);
+        if (k + 1 < a.K) {
+          n_state = s_state[(k + 1) * kDecThreads + tid];
+          n_norm = s_norm[(k + 1) * kDecThreads + tid];
+          n_p = a.stream + (size_t)(k + 1) * a.cap_words + a.offsets[(size_t)(k + 1) * a.nb + b] + ((n_state & 0x3ffffu) >> 5);
+          n_w0 = n_p[0]; n_w1 = n_p[1]; n_w2 = n_p[2];
+        }
         uint32_t flags = 0;
 #pragma unroll
         for (int i = 0; i < kDecChunk; ++i) {
@@ -488,13 +500,29 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
       }
       // mean (and the fused state update) of these coordinates
       const size_t e0 = lo + (size_t)first + (size_t)c0;
+      if (n == kDecChunk && a.vec_out) {
 #pragma unroll
-      for (int i = 0; i < kDecChunk; ++i) {
-        if (i < n) {
-          const float m = __fdiv_rn(acc[i], Kf);
-          a.mean[e0 + i] = m;
-          if (a.update == 1) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], __fmul_rn(gam, m));
-          if (a.update == 2) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], m);
+        for (int i = 0; i < kDecChunk; i += 4) {
+          const float4 m = make_float4(__fdiv_rn(acc[i], Kf), __fdiv_rn(acc[i + 1], Kf), __fdiv_rn(acc[i + 2], Kf), __fdiv_rn(acc[i + 3], Kf));
+          *reinterpret_cast<float4*>(a.mean + e0 + i) = m;
+          if (a.update != 0) {
+            const float4 x = *reinterpret_cast<const float4*>(a.xin + e0 + i);
+            const float g = a.update == 1 ? gam : 1.0f;
+            // update 2 subtracts the mean itself: g = 1 and the product below is exact
+            *reinterpret_cast<float4*>(a.xout + e0 + i) =
+                make_float4(__fsub_rn(x.x, __fmul_rn(g, m.x)), __fsub_rn(x.y, __fmul_rn(g, m.y)),
+                            __fsub_rn(x.z, __fmul_rn(g, m.z)), __fsub_rn(x.w, __fmul_rn(g, m.w)));
+          }
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < kDecChunk; ++i) {
+          if (i < n) {
+            const float m = __fdiv_rn(acc[i], Kf);
+            a.mean[e0 + i] = m;
+            if (a.update == 1) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], __fmul_rn(gam, m));
+            if (a.update == 2) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], m);
+          }
         }
       }
     }
@@ -647,6 +675,8 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   da.d = d; da.bucket = bucket; da.K = K; da.nb = nb; da.lut = lut; da.mean = mean_out;
   da.update = upd ? upd->mode : 0; da.xin = upd ? upd->xin : nullptr; da.xout = upd ? upd->xout : nullptr;
   da.scalars = upd ? upd->scalars : nullptr; da.st = c->dstatus;
+  da.vec_out = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(mean_out) & 15u) == 0) &&
+               ((reinterpret_cast<uintptr_t>(da.xin) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(da.xout) & 15u) == 0);
   return launch_decode_average(c, da, ct);
 }
 
