@@ -3,7 +3,7 @@
 
 One "step" is one extra-gradient iteration of Algorithm 1 on the scale workload: K = 32 simulated
 workers, d = 2^26 fp32 coordinates each, Gaussian-mixture oracle noise (0.9 N(0,1) + 0.1 N(0,100)),
-diagonal operator V(x) = D x, bucket 16384, 17 adaptive levels, Huffman code, sub-blocks of 128
+diagonal operator V(x) = D x, bucket 16384, 17 adaptive levels, Huffman code, sub-blocks of 64
 coordinates.  A step runs both exchanges (quantize -> encode -> decode -> average), the operator,
 the half/dual/primal updates, the adaptive step size, and -- every `--refit-every` steps -- the
 histogram and level refit.
@@ -356,7 +356,7 @@ def main():
     ap.add_argument("--workers", type=int, default=32, help="K, simulated workers")
     ap.add_argument("--d", type=int, default=1 << 26)
     ap.add_argument("--bucket", type=int, default=16384)
-    ap.add_argument("--subblock", type=int, default=128)
+    ap.add_argument("--subblock", type=int, default=64)
     ap.add_argument("--refit-every", type=int, default=10)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-buckets", type=int, default=16, help="buckets per worker in the timed oracle sample")

@@ -327,8 +327,6 @@ struct DecodeArgs {
 };
 
 constexpr int kDecThreads = 128;
-constexpr int kDecChunk = 32;           // coordinates whose running sums a thread keeps in registers
-constexpr uint32_t kStateStep = 1u - (1u << 18);   // adding L * step moves the position up and the bits left down by L
 
 // Bits not yet consumed of one sub-block: a 64-bit window refilled 32 bits at a time.  The streams
 // of the fused path lie in the context's workspace, which extends past every bucket, so a read a
@@ -406,16 +404,39 @@ __device__ __forceinline__ bool locate_subblock(const uint32_t* stream, size_t c
   return ok && (!exists || (hdr_bits + st + len <= nbits && nbits < (1u << 18) && len < (1u << 14)));
 }
 
-// One thread per sub-block.  The thread walks its sub-block of every worker's stream 32 coordinates
-// at a time, keeping the 32 running sums in registers and each worker's bit position in shared memory.
+// One thread per sub-block, workers in the outer loop: the thread keeps all G running sums of its
+// sub-block in registers (fixed k order, so the mean is bit-identical to a sequential sum) and reads each
+// worker's sub-block once, front to back, so that every fetched sector is used up at once.  The next
+// worker's sub-block is located while the current one is decoded.
+struct SubBlockAt {
+  const uint32_t* p;      // word that holds the first bit
+  uint32_t w0, w1, w2;    // p[0..2]
+  uint32_t sh;            // first bit within w0
+  uint32_t want;          // bits of the sub-block
+  float norm;
+  bool ok;
+};
+
+__device__ __forceinline__ SubBlockAt find_subblock(const DecodeArgs& a, int k, size_t b, uint32_t hdr_bits, uint32_t s,
+                                                    bool exists, bool uniform, int lane) {
+  SubBlockAt r;
+  const uint32_t* w;
+  uint32_t st;
+  r.ok = locate_subblock(a.stream + (size_t)k * a.cap_words, a.cap_words, a.bucket_bits, a.offsets, (size_t)k * a.nb + b,
+                         hdr_bits, s, exists, uniform, lane, &w, &r.norm, &st, &r.want);
+  if (!r.ok) { st = 0; r.want = 0; r.norm = 0.0f; }
+  r.p = w + (st >> 5);
+  r.sh = st & 31u;
+  r.w0 = r.p[0]; r.w1 = r.p[1]; r.w2 = r.p[2];
+  return r;
+}
+
 template <int G>
-__global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_constant__ DecodeArgs a, const __grid_constant__ CodeTable ct) {
+__global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6)) k_exchange_decode(const __grid_constant__ DecodeArgs a,
+                                                                      const __grid_constant__ CodeTable ct) {
   extern __shared__ __align__(16) unsigned char s_raw[];
   const int lut_n = 2 << ct.maxlen;
   DecEntry* s_lut = reinterpret_cast<DecEntry*>(s_raw);
-  // per worker and thread: bit position in the bucket (low 18 bits) | bits left in the sub-block << 18
-  uint32_t* s_state = reinterpret_cast<uint32_t*>(s_raw + sizeof(DecEntry) * (size_t)lut_n);    // [K][threads]
-  float* s_norm = reinterpret_cast<float*>(s_state + (size_t)a.K * kDecThreads);                // [K][threads]
   {
     const uint2* src = reinterpret_cast<const uint2*>(a.lut);
     uint2* dst = reinterpret_cast<uint2*>(s_lut);
@@ -442,92 +463,76 @@ __global__ void __launch_bounds__(kDecThreads) k_exchange_decode(const __grid_co
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
     if (!__any_sync(0xffffffffu, count > 0)) continue;   // beyond the end of a short last bucket
 
-    // where this sub-block lies in every worker's stream
+    float acc[G];
+#pragma unroll
+    for (int i = 0; i < G; ++i) acc[i] = 0.0f;
+    SubBlockAt nxt = find_subblock(a, 0, b, hdr_bits, s, count > 0, uniform, lane);
     for (int k = 0; k < a.K; ++k) {
-      const size_t kb = (size_t)k * a.nb + b;
-      const uint32_t* w;
-      float nm;
-      uint32_t st, want;
-      const bool ok = locate_subblock(a.stream + (size_t)k * a.cap_words, a.cap_words, a.bucket_bits, a.offsets, kb, hdr_bits, s,
-                                      count > 0, uniform, lane, &w, &nm, &st, &want);
-      bad = bad || !ok;
-      s_state[k * kDecThreads + tid] = ok ? (st | (want << 18)) : 0u;
-      s_norm[k * kDecThreads + tid] = ok ? nm : 0.0f;
+      const SubBlockAt cur = nxt;
+      if (k + 1 < a.K) nxt = find_subblock(a, k + 1, b, hdr_bits, s, count > 0, uniform, lane);
+      bad = bad || !cur.ok;
+      Window win;
+      win.open(cur.p, cur.w0, cur.w1, cur.w2, cur.sh);
+      uint32_t flags = 0, used = 0;
+      if (count == G) {
+#pragma unroll
+        for (int i = 0; i < G; ++i) {
+          if ((i & 1) == 0) {                              // two symbols use at most 26 bits
+            if (win.avail <= 32) win.refill();
+          }
+          const DecEntry e = s_lut[win.lo & mask];
+          const uint32_t L = e.len & 31u;
+          flags |= e.len;
+          win.skip(L);
+          used += L;
+          acc[i] = __fadd_rn(acc[i], __fmul_rn(cur.norm, e.val));
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < G; ++i) {
+          if ((i & 1) == 0) {
+            if (win.avail <= 32) win.refill();
+          }
+          if (i < count) {
+            const DecEntry e = s_lut[win.lo & mask];
+            const uint32_t L = e.len & 31u;
+            flags |= e.len;
+            win.skip(L);
+            used += L;
+            acc[i] = __fadd_rn(acc[i], __fmul_rn(cur.norm, e.val));
+          }
+        }
+      }
+      bad = bad || (flags & 0x80u) || (count > 0 && used != cur.want);   // every sub-block uses exactly its length
     }
     if (count <= 0) continue;
 
     float gam = 1.0f;
     if (a.update == 1) gam = (float)a.scalars[1];
-    for (int c0 = 0; c0 < count; c0 += kDecChunk) {
-      const int n = min(kDecChunk, count - c0);
-      float acc[kDecChunk];
+    const size_t e0 = lo + (size_t)first;
+    if (count == G && a.vec_out) {
 #pragma unroll
-      for (int i = 0; i < kDecChunk; ++i) acc[i] = 0.0f;
-      // worker k + 1's position, norm and first words are fetched while worker k is decoded
-      uint32_t n_state = s_state[tid];
-      float n_norm = s_norm[tid];
-      const uint32_t* n_p = a.stream + a.offsets[b] + ((n_state & 0x3ffffu) >> 5);
-      uint32_t n_w0 = n_p[0], n_w1 = n_p[1], n_w2 = n_p[2];
-      for (int k = 0; k < a.K; ++k) {
-        uint32_t state = n_state;
-        const float norm = n_norm;
-        Window win;
-        win.open(n_p, n_w0, n_w1, n_w2, state & 31u);
-        if (k + 1 < a.K) {
-          n_state = s_state[(k + 1) * kDecThreads + tid];
-          n_norm = s_norm[(k + 1) * kDecThreads + tid];
-          n_p = a.stream + (size_t)(k + 1) * a.cap_words + a.offsets[(size_t)(k + 1) * a.nb + b] + ((n_state & 0x3ffffu) >> 5);
-          n_w0 = n_p[0]; n_w1 = n_p[1]; n_w2 = n_p[2];
-        }
-        uint32_t flags = 0;
-#pragma unroll
-        for (int i = 0; i < kDecChunk; ++i) {
-          if ((i & 1) == 0) {                              // two symbols use at most 26 bits
-            if (win.avail <= 32) win.refill();
-          }
-          if (i < n) {
-            const DecEntry e = s_lut[win.lo & mask];
-            const uint32_t L = e.len & 31u;
-            flags |= e.len;
-            win.skip(L);
-            state += L * kStateStep;                       // position up, bits left down
-            const float val = __fmul_rn(norm, e.val);
-            acc[i] = __fadd_rn(acc[i], val);
-          }
-        }
-        bad = bad || (flags & 0x80u);
-        s_state[k * kDecThreads + tid] = state;
-      }
-      // mean (and the fused state update) of these coordinates
-      const size_t e0 = lo + (size_t)first + (size_t)c0;
-      if (n == kDecChunk && a.vec_out) {
-#pragma unroll
-        for (int i = 0; i < kDecChunk; i += 4) {
-          const float4 m = make_float4(__fdiv_rn(acc[i], Kf), __fdiv_rn(acc[i + 1], Kf), __fdiv_rn(acc[i + 2], Kf), __fdiv_rn(acc[i + 3], Kf));
-          *reinterpret_cast<float4*>(a.mean + e0 + i) = m;
-          if (a.update != 0) {
-            const float4 x = *reinterpret_cast<const float4*>(a.xin + e0 + i);
-            const float g = a.update == 1 ? gam : 1.0f;
-            // update 2 subtracts the mean itself: g = 1 and the product below is exact
-            *reinterpret_cast<float4*>(a.xout + e0 + i) =
-                make_float4(__fsub_rn(x.x, __fmul_rn(g, m.x)), __fsub_rn(x.y, __fmul_rn(g, m.y)),
-                            __fsub_rn(x.z, __fmul_rn(g, m.z)), __fsub_rn(x.w, __fmul_rn(g, m.w)));
-          }
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < kDecChunk; ++i) {
-          if (i < n) {
-            const float m = __fdiv_rn(acc[i], Kf);
-            a.mean[e0 + i] = m;
-            if (a.update == 1) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], __fmul_rn(gam, m));
-            if (a.update == 2) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], m);
-          }
+      for (int i = 0; i < G; i += 4) {
+        const float4 m = make_float4(__fdiv_rn(acc[i], Kf), __fdiv_rn(acc[i + 1], Kf), __fdiv_rn(acc[i + 2], Kf), __fdiv_rn(acc[i + 3], Kf));
+        *reinterpret_cast<float4*>(a.mean + e0 + i) = m;
+        if (a.update != 0) {
+          const float4 x = *reinterpret_cast<const float4*>(a.xin + e0 + i);
+          const float g = a.update == 1 ? gam : 1.0f;      // update 2 subtracts the mean itself (1 * m is exact)
+          *reinterpret_cast<float4*>(a.xout + e0 + i) =
+              make_float4(__fsub_rn(x.x, __fmul_rn(g, m.x)), __fsub_rn(x.y, __fmul_rn(g, m.y)),
+                          __fsub_rn(x.z, __fmul_rn(g, m.z)), __fsub_rn(x.w, __fmul_rn(g, m.w)));
         }
       }
-    }
-    for (int k = 0; k < a.K; ++k) {
-      bad = bad || ((s_state[k * kDecThreads + tid] >> 18) != 0u);       // every sub-block used exactly its length
+    } else {
+#pragma unroll
+      for (int i = 0; i < G; ++i) {
+        if (i < count) {
+          const float m = __fdiv_rn(acc[i], Kf);
+          a.mean[e0 + i] = m;
+          if (a.update == 1) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], __fmul_rn(gam, m));
+          if (a.update == 2) a.xout[e0 + i] = __fsub_rn(a.xin[e0 + i], m);
+        }
+      }
     }
   }
   if (bad) latch_error(a.st, QGX_ERR_CORRUPT);
@@ -683,17 +688,16 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
 template <int G>
 static qgx_status launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct) {
   const size_t total_sub = da.nb * ((size_t)da.bucket / G);
-  const size_t smem = sizeof(DecEntry) * ((size_t)2 << ct.maxlen) + (sizeof(uint32_t) + sizeof(float)) * (size_t)da.K * kDecThreads;
-  if (smem > 200 * 1024) return QGX_ERR_INVALID_ARG;   // too many workers for the per-thread positions
-  int per_sm = 1;
-  cudaFuncSetAttribute(k_exchange_decode<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G>, kDecThreads, smem);
-  if (per_sm < 1) per_sm = 1;
+  const size_t lut_bytes = sizeof(DecEntry) * ((size_t)2 << ct.maxlen);
   const size_t want = (total_sub + kDecThreads - 1) / kDecThreads;
-  const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
+  int per_sm = 1;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
-    k_exchange_decode<G><<<grid, kDecThreads, smem, c->stream>>>(da, ct);
+    cudaFuncSetAttribute(k_exchange_decode<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lut_bytes);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G>, kDecThreads, lut_bytes);
+    if (per_sm < 1) per_sm = 1;
+    const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
+    k_exchange_decode<G><<<grid, kDecThreads, lut_bytes, c->stream>>>(da, ct);
   }
   count_launch(c);
   return cuda_status(cudaGetLastError());
