@@ -119,31 +119,67 @@ __device__ __forceinline__ float bucket_norm_all(const BucketRegs<V4>& r, int no
   return bad ? __int_as_float(0x7fc00000) : m;
 }
 
+// Loads bucket [lo, lo + len) of worker k, warp-major: warp w holds quads [w * V4 * 32, (w + 1) * V4 * 32),
+// its j-th load covering 32 consecutive quads (512 contiguous bytes), lane l the l-th of them.
+template <int V4>
+__device__ __forceinline__ void load_bucket_warp_major(BucketRegs<V4>& r, const DualSource& s, size_t k, size_t d,
+                                                       size_t lo, int len, bool vec_ok) {
+  const size_t ld = s.ld ? s.ld : d;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int j = 0; j < V4; ++j) {
+    const int e = ((warp * V4 + j) * 32 + lane) * kQuad;
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (e + kQuad <= len && vec_ok) {
+      if (s.a == nullptr) {
+        x = __ldcs(reinterpret_cast<const float4*>(s.v + k * ld + lo + e));
+      } else {
+        const float4 av = __ldg(reinterpret_cast<const float4*>(s.a + lo + e));
+        if (s.v) {
+          const float4 u = __ldcs(reinterpret_cast<const float4*>(s.v + k * ld + lo + e));
+          x = make_float4(__fadd_rn(av.x, u.x), __fadd_rn(av.y, u.y), __fadd_rn(av.z, u.z), __fadd_rn(av.w, u.w));
+        } else {
+          x = av;
+        }
+      }
+    } else {
+      if (e + 0 < len) x.x = dual_value(s, k, d, lo + e + 0);
+      if (e + 1 < len) x.y = dual_value(s, k, d, lo + e + 1);
+      if (e + 2 < len) x.z = dual_value(s, k, d, lo + e + 2);
+      if (e + 3 < len) x.w = dual_value(s, k, d, lo + e + 3);
+    }
+    r.x[j] = x;
+  }
+}
+
 // One persistent CTA per SM slot; each ticket is one bucket (k = ticket % K, b = ticket / K).
-//   load + zero image | barrier | norm, quantize, pack, header fields, warp scans | barrier |
-//   chunk prefixes, bit scatter, look-back (warp 0) | barrier | copy out | barrier
+//   loads, zero the image | barrier | norm, Philox, rounding, packing, sub-block lengths, warp scans |
+//   barrier | warp offsets, bit scatter, look-back (warp 0) | barrier | copy out
+// The bucket image is double buffered, so the copy-out of one bucket needs no barrier before the next
+// bucket starts.  Warp w owns the 128 * V4 coordinates [w * 128 * V4, ...) of the bucket.
 // SYM: 0 plain, 1 also keeps the symbols, 2 also compares with the kept symbols of the other exchange
 template <int V4, int G, int SYM>
 __global__ void __launch_bounds__(V4 == 8 ? 512 : (V4 == 4 ? 512 : 256), V4 == 8 ? 2 : 1)
 k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
                   const __grid_constant__ QuantTable qt) {
-  extern __shared__ uint32_t s_img[];
+  extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ QuantTable s_q;
   __shared__ EncLut s_lut;
   __shared__ uint32_t s_pair[kPairLutSize];
   __shared__ float s_lev[QGX_MAX_LEVELS];
   __shared__ double s_red[2][32];
-  __shared__ uint32_t s_chunk[2][8 * 16];
+  __shared__ uint32_t s_wtot[2][32];
   __shared__ unsigned int s_ticket[2];
-  __shared__ unsigned long long s_prefix;
-  __shared__ int s_skip;
+  __shared__ unsigned long long s_prefix[2];
+  __shared__ int s_skip[2];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  const int img_words = (int)((((uint32_t)a.bucket * (uint32_t)(ct.maxlen + 1) + 16u * (uint32_t)(a.bucket / G + 1) + kNormBits + 31u) >> 5) + 4);
+  // words of one image, a multiple of 4 so that both images are 16-byte aligned
+  const int img_words = (int)((((((uint32_t)a.bucket * (uint32_t)(ct.maxlen + 1) + 16u * (uint32_t)(a.bucket / G + 1) + kNormBits + 31u) >> 5) + 4) + 3u) & ~3u);
   const unsigned long long total = (unsigned long long)a.nb * (unsigned long long)a.K;
   constexpr int kSegLanes = G / kQuad;                  // lanes per sub-block within a warp's 128 coordinates
-  constexpr int kSegs = 32 / kSegLanes;                 // sub-blocks per chunk
+  constexpr int kSegs = 32 / kSegLanes;                 // sub-blocks per chunk of 128 coordinates
 
   fill_enc_lut(&s_lut, ct);
   {
@@ -153,12 +189,14 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   }
   if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 1.0f;
   if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
+  for (int i = threadIdx.x; i < 2 * img_words; i += blockDim.x) s_dyn[i] = 0;
   __syncthreads();
   fill_pair_lut(s_pair, &s_lut);
   __syncthreads();
   const int steps = s_q.steps;
   const int nlev = lt.nlev;
   double sq = 0.0;
+  uint32_t used_words[2] = {0u, 0u};                    // words of each image that the last bucket in it dirtied
 
   for (int par = 0;; par ^= 1) {
     const unsigned long long t = s_ticket[par];
@@ -166,10 +204,16 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     const size_t b = (size_t)(t / (unsigned long long)a.K), k = (size_t)(t % (unsigned long long)a.K);
     const size_t lo = b * (size_t)a.bucket;
     const int len = (int)min((size_t)a.bucket, a.d - lo);
+    uint32_t* s_img = s_dyn + par * img_words;
 
     BucketRegs<V4> r;
-    load_bucket<V4>(r, a.src, k, a.d, lo, len, a.vec_ok);
-    for (int i = threadIdx.x; i < img_words; i += blockDim.x) s_img[i] = 0;
+    load_bucket_warp_major<V4>(r, a.src, k, a.d, lo, len, a.vec_ok);
+    {
+      // this image was last read by the copy-out two buckets ago; two barriers have passed since
+      uint4* z = reinterpret_cast<uint4*>(s_img);
+      const int n4 = (int)((used_words[par] + 3u + 3u) >> 2);
+      for (int i = threadIdx.x; i < n4; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
     const float norm = bucket_norm_all<V4>(r, a.norm_type, s_red[par]);      // barrier inside: the image is zero
     const bool finite = (norm - norm) == 0.0f;
     const float rn = fast_reciprocal(norm, steps);
@@ -181,15 +225,17 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     const uint32_t nsub = (uint32_t)((len + G - 1) / G);
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
     const float norm_prev = SYM == 2 ? a.norms_prev[k * a.nb + b] : 0.0f;
+    const bool whole = (len == a.bucket) && a.vec_ok;     // no ragged end: no per-quad checks
+    const bool live = finite && norm != 0.0f;             // otherwise every coordinate is level 0
 
     uint64_t qbits[V4];
-    uint32_t qn[V4], qexcl[V4];
+    uint32_t qn[V4], qoff[V4];
 #pragma unroll
     for (int j = 0; j < V4; ++j) {
-      const int q = j * (int)blockDim.x + (int)threadIdx.x;
-      const int nvalid = max(0, min(kQuad, len - q * kQuad));
+      const int q = (warp * V4 + j) * 32 + lane;
+      const int nvalid = whole ? kQuad : max(0, min(kQuad, len - q * kQuad));
       uint32_t sym4 = 0;
-      if (nvalid > 0 && finite && norm != 0.0f) {
+      if (live && nvalid > 0) {
         const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + (uint64_t)q;
         const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
         sym4 = quad_symbols(r.x[j], quantize_quad(r.x[j], w, rn, norm, &s_q, s_lev, nlev));
@@ -220,56 +266,50 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
         pack_quad(sym4, nvalid, &s_lut, &qbits[j], &qn[j]);      // the ragged end of a bucket
       }
     }
-    // warp scans of the bit counts, two quads per 32-bit word (a chunk holds at most 32 * 52 bits)
+    // warp scans of the bit counts, two chunks per 32-bit word (a chunk holds at most 32 * 52 bits);
+    // qoff[j] becomes the quad's bit offset inside the warp's part of the payload
+    uint32_t warp_bits = 0;
 #pragma unroll
     for (int j = 0; j < V4; j += 2) {
       const uint32_t both = qn[j] | ((j + 1 < V4 ? qn[j + 1] : 0u) << 16);
       const uint32_t incl = warp_incl_scan(both, lane);
       const uint32_t before = __shfl_up_sync(0xffffffffu, incl, kSegLanes);
       const uint32_t seg = incl - (lane >= kSegLanes ? before : 0u);   // per field: no borrow, the scans are monotone
+      const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (j + h < V4) {
           const uint32_t mine = (incl >> (16 * h)) & 0xffffu;
-          qexcl[j + h] = mine - qn[j + h];
-          // sub-block lengths: the last lane of each sub-block knows its total
+          qoff[j + h] = warp_bits + mine - qn[j + h];
+          warp_bits += (tot >> (16 * h)) & 0xffffu;
+          // sub-block lengths: the last lane of each sub-block knows its total; the 16-bit fields are
+          // halfword aligned, a plain store
           if ((lane + 1) % kSegLanes == 0) {
-            const int sb = ((j + h) * nwarps + warp) * kSegs + lane / kSegLanes;
-            // the 16-bit length fields are halfword aligned: a plain store
-            if (sb * G < len) reinterpret_cast<uint16_t*>(s_img)[2 + sb] = (uint16_t)((seg >> (16 * h)) & 0xffffu);
+            const int sb = (warp * V4 + j + h) * kSegs + lane / kSegLanes;
+            if (whole || sb * G < len) reinterpret_cast<uint16_t*>(s_img)[2 + sb] = (uint16_t)((seg >> (16 * h)) & 0xffffu);
           }
-          if (lane == 31) s_chunk[par][(j + h) * nwarps + warp] = mine;
         }
       }
     }
+    if (lane == 0) s_wtot[par][warp] = warp_bits;
     __syncthreads();
-    // exclusive prefix of the chunk totals, computed by every warp for itself
-    const int nchunks = V4 * nwarps;                     // <= 128
-    uint32_t pre[4];
-    uint32_t carry = 0;
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-      const int i = g * 32 + lane;
-      const uint32_t x = i < nchunks ? s_chunk[par][i] : 0u;
-      const uint32_t incl = warp_incl_scan(x, lane);
-      pre[g] = carry + incl - x;
-      carry += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    const uint32_t nbits = hdr_bits + carry;
+    // where this warp's part starts: exclusive prefix of the warps' totals
+    const uint32_t wt = lane < nwarps ? s_wtot[par][lane] : 0u;
+    const uint32_t wincl = warp_incl_scan(wt, lane);
+    const uint32_t wbase = __shfl_sync(0xffffffffu, wincl - wt, warp);
+    const uint32_t payload = __shfl_sync(0xffffffffu, wincl, 31);
+    const uint32_t nbits = hdr_bits + payload;
     const uint32_t nwords = (nbits + 31) >> 5;
+    used_words[par] = nwords;
     unsigned long long* row = a.status + k * a.nb;
     if (threadIdx.x == 0) {
       st_status(row + b, kStAggregate | (unsigned long long)nwords);
       a.bucket_bits[k * a.nb + b] = nbits;
       atomicAdd(a.total_bits + k, (unsigned long long)nbits);
     }
+    const uint32_t base = hdr_bits + wbase;
 #pragma unroll
-    for (int j = 0; j < V4; ++j) {
-      const int c = j * nwarps + warp;
-      const uint32_t sel = (c >> 5) == 0 ? pre[0] : ((c >> 5) == 1 ? pre[1] : ((c >> 5) == 2 ? pre[2] : pre[3]));
-      const uint32_t p = __shfl_sync(0xffffffffu, sel, c & 31) + qexcl[j];
-      put_bits(s_img, hdr_bits + p, qbits[j], qn[j]);
-    }
+    for (int j = 0; j < V4; ++j) put_bits(s_img, base + qoff[j], qbits[j], qn[j]);
     if (warp == 0) {
       bool timed_out = false;
       const unsigned long long excl = lookback_prefix(row, (long long)b, lane, &timed_out);
@@ -279,17 +319,18 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
         if (timed_out) { latch_error(a.st, QGX_ERR_TIMEOUT); skip = 1; }
         if (excl + nwords > (unsigned long long)a.cap_words) { latch_error(a.st, QGX_ERR_CAPACITY); skip = 1; }
         a.offsets[k * a.nb + b] = (uint32_t)min(excl, (unsigned long long)0xffffffffu);
-        s_prefix = excl;
-        s_skip = skip;
+        s_prefix[par] = excl;
+        s_skip[par] = skip;
         s_ticket[par ^ 1] = atomicAdd(a.ticket, 1u);
       }
     }
     __syncthreads();
-    if (!s_skip) {
-      uint32_t* dst = a.stream + k * a.cap_words + s_prefix;
+    if (!s_skip[par]) {
+      uint32_t* dst = a.stream + k * a.cap_words + s_prefix[par];
       for (uint32_t i = threadIdx.x; i < nwords; i += blockDim.x) dst[i] = s_img[i];
     }
-    __syncthreads();
+    // no barrier here: the next bucket works in the other image, and this one is next written after
+    // two more barriers
   }
   if (SYM == 2) {
     sq = warp_sum(sq);
@@ -615,8 +656,8 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   if (!ct.has_header || bucket % ct.G != 0 || (ct.G != 32 && ct.G != 64 && ct.G != 128)) return QGX_ERR_INVALID_ARG;
   const int v4 = bucket_v4(bucket);
   const int threads = bucket_threads(bucket, v4);
-  const size_t img_words = (((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4;
-  const size_t smem = sizeof(uint32_t) * img_words;
+  const size_t img_words = (((((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4) + 3) & ~(size_t)3;
+  const size_t smem = sizeof(uint32_t) * 2 * img_words;   // two images: see k_exchange_encode
   int per_sm = 1;
 #define QGX_LAUNCH_E(V, GG, SS)                                                                                  \
   do {                                                                                                           \
