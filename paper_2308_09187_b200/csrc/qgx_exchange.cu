@@ -75,13 +75,6 @@ struct EncodeArgs {
   float* norms;                 // [K][nb] (kept for the caller; the streams carry them too)
   unsigned long long* status;   // [K][nb], zeroed before the launch
   unsigned int* ticket;         // zeroed before the launch
-  // optional: keep this exchange's symbols (1 byte per coordinate) ...
-  uint8_t* sym_out;             // [K][d] or null
-  // ... and compare with the symbols and norms kept by an earlier exchange:
-  // *sum_sq += sum_k ||Q(V_k) of that exchange - Q(V_k) of this one||^2 (fp32 differences, fp64 sum)
-  const uint8_t* sym_prev;      // [K][d] or null
-  const float* norms_prev;      // [K][nb]
-  double* sum_sq;
   DevStatus* st;
 };
 
@@ -157,8 +150,7 @@ __device__ __forceinline__ void load_bucket_warp_major(BucketRegs<V4>& r, const 
 //   barrier | warp offsets, bit scatter, look-back (warp 0) | barrier | copy out
 // The bucket image is double buffered, so the copy-out of one bucket needs no barrier before the next
 // bucket starts.  Warp w owns the 128 * V4 coordinates [w * 128 * V4, ...) of the bucket.
-// SYM: 0 plain, 1 also keeps the symbols, 2 also compares with the kept symbols of the other exchange
-template <int V4, int G, int SYM>
+template <int V4, int G>
 __global__ void __launch_bounds__(V4 == 8 ? 512 : (V4 == 4 ? 512 : 256), V4 == 8 ? 2 : 1)
 k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
@@ -195,7 +187,6 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   __syncthreads();
   const int steps = s_q.steps;
   const int nlev = lt.nlev;
-  double sq = 0.0;
   uint32_t used_words[2] = {0u, 0u};                    // words of each image that the last bucket in it dirtied
 
   for (int par = 0;; par ^= 1) {
@@ -224,7 +215,6 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     const uint32_t nsub = (uint32_t)((len + G - 1) / G);
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
-    const float norm_prev = SYM == 2 ? a.norms_prev[k * a.nb + b] : 0.0f;
     const bool whole = (len == a.bucket) && a.vec_ok;     // no ragged end: no per-quad checks
     const bool live = finite && norm != 0.0f;             // otherwise every coordinate is level 0
 
@@ -239,26 +229,6 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
         const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + (uint64_t)q;
         const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
         sym4 = quad_symbols(r.x[j], quantize_quad(r.x[j], w, rn, norm, &s_q, s_lev, nlev));
-      }
-      if (SYM == 1 && nvalid > 0) {
-        uint8_t* o = a.sym_out + k * a.d + lo + (size_t)q * kQuad;
-        if (nvalid == kQuad && a.vec_ok) *reinterpret_cast<uint32_t*>(o) = sym4;
-        else for (int c = 0; c < nvalid; ++c) o[c] = (uint8_t)(sym4 >> (8 * c));
-      }
-      if (SYM == 2 && nvalid > 0) {
-        const uint8_t* o = a.sym_prev + k * a.d + lo + (size_t)q * kQuad;
-        uint32_t prev4 = 0;
-        if (nvalid == kQuad && a.vec_ok) prev4 = __ldcs(reinterpret_cast<const uint32_t*>(o));
-        else for (int c = 0; c < nvalid; ++c) prev4 |= (uint32_t)o[c] << (8 * c);
-#pragma unroll
-        for (int c = 0; c < kQuad; ++c) {
-          if (c < nvalid) {
-            const float d1 = dequantize_symbol((prev4 >> (8 * c)) & 0xffu, norm_prev, s_lev);
-            const float d2 = dequantize_symbol((sym4 >> (8 * c)) & 0xffu, finite ? norm : 0.0f, s_lev);
-            const float dlt = __fsub_rn(d1, d2);
-            sq = fma((double)dlt, (double)dlt, sq);
-          }
-        }
       }
       if (nvalid == kQuad) {
         pack_quad_pairs(sym4, s_pair, &qbits[j], &qn[j]);
@@ -332,10 +302,6 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     // no barrier here: the next bucket works in the other image, and this one is next written after
     // two more barriers
   }
-  if (SYM == 2) {
-    sq = warp_sum(sq);
-    if (lane == 0 && sq != 0.0) atomicAdd(a.sum_sq, sq);
-  }
 }
 
 // ---- decode + average ------------------------------------------------------------------------
@@ -364,6 +330,14 @@ struct DecodeArgs {
   float* xout;
   const double* scalars;        // scalars[1] = gamma_t
   bool vec_out;                 // d % 4 == 0 and mean, xin, xout 16-byte aligned: 128-bit stores
+  // optional: keep the decoded symbols (1 byte per coordinate and worker) ...
+  uint8_t* sym_out;             // [K][d] or null
+  // ... or compare with the symbols and norms kept by the other exchange of the iteration:
+  // *sum_sq += sum_k ||vhat_k of that exchange - vhat_k of this one||^2 (fp32 differences, fp64 sum)
+  const uint8_t* sym_prev;      // [K][d] or null
+  const float* norms_prev;      // [K][nb]
+  double* sum_sq;
+  bool vec_sym;                 // d % 4 == 0: four symbol bytes move as one word
   DevStatus* st;
 };
 
@@ -455,6 +429,7 @@ struct SubBlockAt {
   uint32_t sh;            // first bit within w0
   uint32_t want;          // bits of the sub-block
   float norm;
+  float norm_prev;        // norm of the same bucket in the other exchange (when comparing)
   bool ok;
 };
 
@@ -469,13 +444,17 @@ __device__ __forceinline__ SubBlockAt find_subblock(const DecodeArgs& a, int k, 
   r.p = w + (st >> 5);
   r.sh = st & 31u;
   r.w0 = r.p[0]; r.w1 = r.p[1]; r.w2 = r.p[2];
+  r.norm_prev = a.norms_prev ? a.norms_prev[(size_t)k * a.nb + b] : 0.0f;
   return r;
 }
 
-template <int G>
+// SYM: 0 plain, 1 also keeps the decoded symbols, 2 also compares with the symbols kept by the other exchange
+template <int G, int SYM>
 __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6)) k_exchange_decode(const __grid_constant__ DecodeArgs a,
-                                                                      const __grid_constant__ CodeTable ct) {
+                                                                      const __grid_constant__ CodeTable ct,
+                                                                      const __grid_constant__ LevelTable lt) {
   extern __shared__ __align__(16) unsigned char s_raw[];
+  __shared__ float s_lev[QGX_MAX_LEVELS];
   const int lut_n = 2 << ct.maxlen;
   DecEntry* s_lut = reinterpret_cast<DecEntry*>(s_raw);
   {
@@ -483,6 +462,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
     uint2* dst = reinterpret_cast<uint2*>(s_lut);
     for (int i = threadIdx.x; i < lut_n; i += blockDim.x) dst[i] = src[i];
   }
+  if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 0.0f;
   __syncthreads();
   const uint32_t mask = (uint32_t)lut_n - 1u;
   const int lane = threadIdx.x & 31, tid = threadIdx.x;
@@ -491,6 +471,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
   const bool uniform = (spb % 32 == 0);
   const float Kf = (float)a.K;
   bool bad = false;
+  double sq = 0.0;
 
   for (size_t gs = (size_t)blockIdx.x * blockDim.x + tid; gs - lane < total_sub; gs += (size_t)gridDim.x * blockDim.x) {
     const bool live = gs < total_sub;
@@ -503,6 +484,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
     const uint32_t nsub = (uint32_t)((len + G - 1) / G);
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
     if (!__any_sync(0xffffffffu, count > 0)) continue;   // beyond the end of a short last bucket
+    const size_t e0 = lo + (size_t)first;
 
     float acc[G];
 #pragma unroll
@@ -515,18 +497,29 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
       Window win;
       win.open(cur.p, cur.w0, cur.w1, cur.w2, cur.sh);
       uint32_t flags = 0, used = 0;
-      if (count == G) {
+      if (count == G && a.vec_sym) {
+        uint32_t pack = 0, prev4 = 0;
 #pragma unroll
         for (int i = 0; i < G; ++i) {
           if ((i & 1) == 0) {                              // two symbols use at most 26 bits
             if (win.avail <= 32) win.refill();
           }
+          if (SYM == 2 && (i & 3) == 0) prev4 = __ldcs(reinterpret_cast<const uint32_t*>(a.sym_prev + (size_t)k * a.d + e0 + i));
           const DecEntry e = s_lut[win.lo & mask];
           const uint32_t L = e.len & 31u;
           flags |= e.len;
           win.skip(L);
           used += L;
-          acc[i] = __fadd_rn(acc[i], __fmul_rn(cur.norm, e.val));
+          const float val = __fmul_rn(cur.norm, e.val);
+          acc[i] = __fadd_rn(acc[i], val);
+          if (SYM == 1) {
+            pack |= ((e.len >> 8) & 0xffu) << (8 * (i & 3));
+            if ((i & 3) == 3) { *reinterpret_cast<uint32_t*>(a.sym_out + (size_t)k * a.d + e0 + i - 3) = pack; pack = 0; }
+          }
+          if (SYM == 2) {
+            const float dlt = __fsub_rn(dequantize_symbol((prev4 >> (8 * (i & 3))) & 0xffu, cur.norm_prev, s_lev), val);
+            sq = fma((double)dlt, (double)dlt, sq);
+          }
         }
       } else {
 #pragma unroll
@@ -540,7 +533,13 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
             flags |= e.len;
             win.skip(L);
             used += L;
-            acc[i] = __fadd_rn(acc[i], __fmul_rn(cur.norm, e.val));
+            const float val = __fmul_rn(cur.norm, e.val);
+            acc[i] = __fadd_rn(acc[i], val);
+            if (SYM == 1) a.sym_out[(size_t)k * a.d + e0 + i] = (uint8_t)((e.len >> 8) & 0xffu);
+            if (SYM == 2) {
+              const float dlt = __fsub_rn(dequantize_symbol(a.sym_prev[(size_t)k * a.d + e0 + i], cur.norm_prev, s_lev), val);
+              sq = fma((double)dlt, (double)dlt, sq);
+            }
           }
         }
       }
@@ -550,7 +549,6 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
 
     float gam = 1.0f;
     if (a.update == 1) gam = (float)a.scalars[1];
-    const size_t e0 = lo + (size_t)first;
     if (count == G && a.vec_out) {
 #pragma unroll
       for (int i = 0; i < G; i += 4) {
@@ -576,6 +574,10 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
       }
     }
   }
+  if (SYM == 2) {
+    sq = warp_sum(sq);
+    if (lane == 0 && sq != 0.0) atomicAdd(a.sum_sq, sq);
+  }
   if (bad) latch_error(a.st, QGX_ERR_CORRUPT);
 }
 
@@ -593,11 +595,10 @@ __global__ void k_add_u64(uint64_t* acc, const uint64_t* x, int n) {
   if (i < n) acc[i] += x[i];
 }
 
-qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct);
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct, const LevelTable& lt, int sym_mode);
 
-// The whole exchange.  sym_mode 1 keeps this exchange's symbols and norms in the workspace; sym_mode 2
-// adds sum_k ||Q(V_k) kept by the other slot - Q(V_k) of this exchange||^2 to *sum_sq (each worker's
-// own two quantized vectors, which the loss-less code reproduces exactly on the receiving side).
+// The whole exchange.  sym_mode 1 keeps the decoded symbols (and the norms) in the workspace; sym_mode 2
+// adds sum_k ||vhat_k kept by the other slot - vhat_k decoded in this exchange||^2 to *sum_sq.
 qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
                          float* mean_out, uint64_t* total_bits_out, const ExchangeUpdate* upd, int sym_mode, double* sum_sq,
                          uint64_t coord_base) {
@@ -640,15 +641,17 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   ea.vec_ok = (d % kQuad == 0) && (src.ld % kQuad == 0) && ((reinterpret_cast<uintptr_t>(src.v) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
   ea.stream = stream; ea.cap_words = cap; ea.bucket_bits = bbits; ea.offsets = offs; ea.total_bits = tot; ea.norms = norms;
   ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(status + (size_t)K * nb); ea.st = c->dstatus;
-  ea.sym_out = nullptr; ea.sym_prev = nullptr; ea.norms_prev = nullptr; ea.sum_sq = sum_sq;
+  uint8_t* sym_out = nullptr;
+  const uint8_t* sym_prev = nullptr;
+  const float* norms_prev = nullptr;
   if (sym_mode == 1) {
-    ea.sym_out = (uint8_t*)ws_get(c, WS_SYM, (size_t)K * d + 16);
-    if (!ea.sym_out) return QGX_ERR_CUDA;
+    sym_out = (uint8_t*)ws_get(c, WS_SYM, (size_t)K * d + 16);
+    if (!sym_out) return QGX_ERR_CUDA;
     c->sym_slot = slot; c->sym_K = K; c->sym_d = d;
   } else if (sym_mode == 2) {
     if (!sum_sq || c->sym_slot != 1 - slot || c->sym_K != K || c->sym_d != d || c->slot_nb[1 - slot] != nb) return QGX_ERR_INVALID_ARG;
-    ea.sym_prev = (const uint8_t*)c->ws[WS_SYM];
-    ea.norms_prev = (const float*)c->ws[slot == 0 ? WS_NORMS2 : WS_NORMS];
+    sym_prev = (const uint8_t*)c->ws[WS_SYM];
+    norms_prev = (const float*)c->ws[slot == 0 ? WS_NORMS2 : WS_NORMS];
   }
   const PhiloxKey key = make_philox_key(cfg->seed);
   QuantTable qt;
@@ -659,26 +662,20 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const size_t img_words = (((((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4) + 3) & ~(size_t)3;
   const size_t smem = sizeof(uint32_t) * 2 * img_words;   // two images: see k_exchange_encode
   int per_sm = 1;
-#define QGX_LAUNCH_E(V, GG, SS)                                                                                  \
-  do {                                                                                                           \
-    cudaFuncSetAttribute(k_exchange_encode<V, GG, SS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG, SS>, threads, smem);         \
-    if (per_sm < 1) per_sm = 1;                                                                                  \
-    const unsigned long long want = (unsigned long long)nb * (unsigned long long)K;                              \
-    const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);     \
-    k_exchange_encode<V, GG, SS><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                        \
-  } while (0)
-#define QGX_LAUNCH_ES(V, GG)                               \
-  do {                                                     \
-    if (sym_mode == 1) QGX_LAUNCH_E(V, GG, 1);             \
-    else if (sym_mode == 2) QGX_LAUNCH_E(V, GG, 2);        \
-    else QGX_LAUNCH_E(V, GG, 0);                           \
+#define QGX_LAUNCH_E(V, GG)                                                                                    \
+  do {                                                                                                         \
+    cudaFuncSetAttribute(k_exchange_encode<V, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG>, threads, smem);           \
+    if (per_sm < 1) per_sm = 1;                                                                                \
+    const unsigned long long want = (unsigned long long)nb * (unsigned long long)K;                            \
+    const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);   \
+    k_exchange_encode<V, GG><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                          \
   } while (0)
 #define QGX_LAUNCH_EG(V)                                   \
   do {                                                     \
-    if (ct.G == 32) QGX_LAUNCH_ES(V, 32);                  \
-    else if (ct.G == 64) QGX_LAUNCH_ES(V, 64);             \
-    else QGX_LAUNCH_ES(V, 128);                            \
+    if (ct.G == 32) QGX_LAUNCH_E(V, 32);                   \
+    else if (ct.G == 64) QGX_LAUNCH_E(V, 64);              \
+    else QGX_LAUNCH_E(V, 128);                             \
   } while (0)
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_ENCODE);
@@ -690,7 +687,6 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
     }
   }
 #undef QGX_LAUNCH_EG
-#undef QGX_LAUNCH_ES
 #undef QGX_LAUNCH_E
   count_launch(c);
   if (cudaGetLastError() != cudaSuccess) return QGX_ERR_CUDA;
@@ -707,10 +703,10 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
       const uint16_t e = by_code[i & (((size_t)1 << ct.maxlen) - 1)];
       const uint32_t L = e >> 8, idx = e & 0xffu;
       if (L == 0) { h_lut[i].val = 0.0f; h_lut[i].len = 1u | 0x80u; continue; }
-      if (idx == 0) { h_lut[i].val = 0.0f; h_lut[i].len = L; continue; }
+      if (idx == 0) { h_lut[i].val = 0.0f; h_lut[i].len = L; continue; }       // symbol byte 0
       const bool neg = (i >> L) & 1u;
       h_lut[i].val = neg ? -cfg->levels[idx] : cfg->levels[idx];
-      h_lut[i].len = L + 1u;
+      h_lut[i].len = (L + 1u) | ((idx | (neg ? 0x80u : 0u)) << 8);       // bits 8..15: the symbol byte
     }
     if (cudaMemcpyAsync(lut, h_lut.data(), h_lut.size() * sizeof(DecEntry), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
       return QGX_ERR_CUDA;
@@ -718,38 +714,47 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
 
   DecodeArgs da;
   da.stream = stream; da.cap_words = cap; da.bucket_bits = bbits; da.offsets = offs;
+  da.sym_out = sym_out; da.sym_prev = sym_prev; da.norms_prev = norms_prev; da.sum_sq = sum_sq;
+  da.vec_sym = (d % kQuad == 0);
   da.d = d; da.bucket = bucket; da.K = K; da.nb = nb; da.lut = lut; da.mean = mean_out;
   da.update = upd ? upd->mode : 0; da.xin = upd ? upd->xin : nullptr; da.xout = upd ? upd->xout : nullptr;
   da.scalars = upd ? upd->scalars : nullptr; da.st = c->dstatus;
   da.vec_out = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(mean_out) & 15u) == 0) &&
                ((reinterpret_cast<uintptr_t>(da.xin) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(da.xout) & 15u) == 0);
-  return launch_decode_average(c, da, ct);
+  return launch_decode_average(c, da, ct, lt, sym_mode);
 }
 
-template <int G>
-static qgx_status launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct) {
+template <int G, int SYM>
+static qgx_status launch_decode_gs(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt) {
   const size_t total_sub = da.nb * ((size_t)da.bucket / G);
   const size_t lut_bytes = sizeof(DecEntry) * ((size_t)2 << ct.maxlen);
   const size_t want = (total_sub + kDecThreads - 1) / kDecThreads;
   int per_sm = 1;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
-    cudaFuncSetAttribute(k_exchange_decode<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lut_bytes);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G>, kDecThreads, lut_bytes);
+    cudaFuncSetAttribute(k_exchange_decode<G, SYM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lut_bytes);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, SYM>, kDecThreads, lut_bytes);
     if (per_sm < 1) per_sm = 1;
     const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
-    k_exchange_decode<G><<<grid, kDecThreads, lut_bytes, c->stream>>>(da, ct);
+    k_exchange_decode<G, SYM><<<grid, kDecThreads, lut_bytes, c->stream>>>(da, ct, lt);
   }
   count_launch(c);
   return cuda_status(cudaGetLastError());
 }
 
-qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct) {
+template <int G>
+static qgx_status launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt, int sym_mode) {
+  if (sym_mode == 1) return launch_decode_gs<G, 1>(c, da, ct, lt);
+  if (sym_mode == 2) return launch_decode_gs<G, 2>(c, da, ct, lt);
+  return launch_decode_gs<G, 0>(c, da, ct, lt);
+}
+
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt, int sym_mode) {
   if (!ct.has_header || da.bucket % ct.G != 0) return QGX_ERR_INVALID_ARG;
   switch (ct.G) {
-    case 32: return launch_decode_g<32>(c, da, ct);
-    case 64: return launch_decode_g<64>(c, da, ct);
-    case 128: return launch_decode_g<128>(c, da, ct);
+    case 32: return launch_decode_g<32>(c, da, ct, lt, sym_mode);
+    case 64: return launch_decode_g<64>(c, da, ct, lt, sym_mode);
+    case 128: return launch_decode_g<128>(c, da, ct, lt, sym_mode);
     default: return QGX_ERR_INVALID_ARG;
   }
 }
