@@ -89,6 +89,53 @@ void make_quant_table(const float* lev, int nlev, QuantTable* out) {
   out->steps = steps;
 }
 
+// Tables of round_fast.  The margin bounds, in units of 1 / S of an interval, everything by which the
+// kernel's S (F - r) can differ from the exact routine's decision variable: u2 against the correctly
+// rounded quotient and the rounding of b and of the knot (together under 2 * 2^-22 (l_{tau+1} + 2^-16) / width,
+// with the narrower of the two intervals around a level), the rounding of a, three fused multiply-adds of
+// results below 2^24, the slope-change term, and the exact routine's own roundings of xi plus the variate's
+// dropped last bit (3.02 S / 2^24).
+void make_round_table(const float* lev, int nlev, RoundTable* out) {
+  std::memset(out, 0, sizeof(*out));
+  out->nlev = nlev;
+  const double S = nlev <= 17 ? 524288.0 : 262144.0;
+  const double c0 = (double)kRoundShift;
+  double b[QGX_MAX_LEVELS] = {0}, width[QGX_MAX_LEVELS] = {0};
+  for (int t = 0; t <= nlev - 2; ++t) {
+    width[t] = (double)(float)(lev[t + 1] - lev[t]);             // the fp32 difference the exact routine divides by
+    b[t] = S / width[t];
+    out->b[t] = (float)b[t];
+    out->a[t] = (float)(S * t - b[t] * ((double)lev[t] + c0) + 1.5 * S);
+  }
+  for (int j = 0; j < QGX_MAX_LEVELS; ++j) {
+    const bool interior = j >= 1 && j <= nlev - 2;
+    out->knot[j] = interior ? (float)((double)lev[j] + c0) : 4.0f;
+    out->db[j] = interior ? (float)(b[j] - b[j - 1]) : 0.0f;
+  }
+  double margin = 0.0;
+  for (int t = 0; t <= nlev - 2; ++t) {
+    const double wmin = std::min(width[t], t + 1 <= nlev - 2 ? width[t + 1] : width[t]);
+    const double a_ulp = (double)std::nextafter(std::fabs(out->a[t]), INFINITY) - (double)std::fabs(out->a[t]);
+    const double e = 2.0 * S * 0x1p-22 * ((double)lev[t + 1] + c0) / wmin + a_ulp + 1.5 + 1.0 + 3.02 * S / 16777216.0;
+    margin = std::max(margin, e);
+  }
+  margin = (margin + 2.0) * 1.01;
+  bool usable = std::isfinite(margin) && margin < S / 4.0;
+  for (int i = 0; i < kKeyBins && usable; ++i) {
+    const uint32_t lo_bits = (uint32_t)(i + kKeyMin) << kKeyShift, hi_bits = ((uint32_t)(i + 1 + kKeyMin) << kKeyShift) - 1u;
+    float lo, hi;
+    std::memcpy(&lo, &lo_bits, 4);
+    std::memcpy(&hi, &hi_bits, 4);
+    int inside = 0;
+    for (int j = 1; j <= nlev - 2; ++j) inside += (out->knot[j] > lo && out->knot[j] <= hi) ? 1 : 0;
+    if (inside > 1) usable = false;
+  }
+  out->usable = usable ? 1 : 0;
+  out->thr = usable ? (float)(S / 2.0 - margin) : -1.0f;
+  out->neg_qscale = (float)(-S / 8388608.0);
+  out->magic = (float)(1.5 * 8388608.0 * S);
+}
+
 void* ws_get(qgx_ctx* c, int which, size_t bytes) {
   if (bytes == 0) bytes = 16;
   if (c->ws_bytes[which] >= bytes) return c->ws[which];

@@ -192,6 +192,101 @@ __device__ __forceinline__ uint32_t quad_symbols(const float4 x, uint32_t idx4) 
   return idx4 | (s & nz);
 }
 
+// ---- rounding through the level map -----------------------------------------------------------
+// F(u) = tau + (u - l_tau) / (l_{tau+1} - l_tau) is continuous and piecewise linear, and Definition 1
+// rounds u to level floor(F(u) - r) + 1 (r the uniform variate) unless F(u) - r is an integer.  The
+// kernels evaluate S F(u) with S = 2^19 (2^18 above 17 levels) from a table over the float pattern
+// of u2 = |v| RN(1 / norm) + 2^-16 (64 bins per octave, every bin holding at most one level: the lower
+// piece plus a slope change past that level), subtract S r, and read the level index off the mantissa
+// after adding 1.5 * 2^23 * S.  Whenever S (F - r) comes closer than `margin` to a multiple of S the
+// exact routine decides instead; the margin (see make_round_table) covers the difference between u2 and
+// the exact quotient, the table's roundings and the three fused multiply-adds.
+constexpr float kRoundShift = 1.52587890625e-05f;       // 2^-16: keeps u2 inside the table
+struct RoundTable {
+  int nlev;
+  int usable;                            // 0: some bin holds two levels, or the margin is too wide
+  float thr;                             // S / 2 - margin
+  float neg_qscale;                      // -S / 2^23
+  float magic;                           // 1.5 * 2^23 * S
+  float a[QGX_MAX_LEVELS];               // per interval: S tau - b (l_tau + 2^-16) + 1.5 S
+  float b[QGX_MAX_LEVELS];               //               S / (l_{tau+1} - l_tau)
+  float knot[QGX_MAX_LEVELS];            // l_j + 2^-16 for interior levels j, else a value never reached
+  float db[QGX_MAX_LEVELS];              // b[j] - b[j - 1]
+};
+
+// one entry per bin: {a, b, knot, db} of the interval of the bin's lowest value
+__device__ __forceinline__ void fill_bin_table(float4* bin, const RoundTable& rt) {
+  for (int i = threadIdx.x; i < kKeyBins; i += blockDim.x) {
+    const float lo = __uint_as_float((uint32_t)(i + kKeyMin) << kKeyShift);
+    const float hi = __uint_as_float(((uint32_t)(i + 1 + kKeyMin) << kKeyShift) - 1u);
+    int t0 = 0;
+    for (int j = 1; j <= rt.nlev - 2; ++j) t0 = (rt.knot[j] <= lo) ? j : t0;
+    const bool straddle = (t0 + 1 <= rt.nlev - 2) && (rt.knot[t0 + 1] <= hi);
+    bin[i] = make_float4(rt.a[t0], rt.b[t0], straddle ? rt.knot[t0 + 1] : 4.0f, straddle ? rt.db[t0 + 1] : 0.0f);
+  }
+}
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+
+struct RoundConsts {
+  float rn;                              // RN(1 / norm)
+  float thr;                             // negative: every coordinate goes to the exact routine
+  float neg_qscale, magic;
+};
+
+__device__ __forceinline__ RoundConsts round_consts(const RoundTable& rt, float norm) {
+  const bool ok = rt.usable && norm > 7.9e-31f && norm < 1.2e30f;
+  RoundConsts c;
+  c.rn = ok ? __frcp_rn(norm) : 0.0f;
+  c.thr = ok ? rt.thr : -1.0f;
+  c.neg_qscale = rt.neg_qscale;
+  c.magic = rt.magic;
+  return c;
+}
+
+// pattern of the float whose low mantissa bits are the level index; *unsafe: ask the exact routine
+__device__ __forceinline__ uint32_t round_fast(float absv, const RoundConsts& c, const float4* bin, uint32_t word, bool* unsafe) {
+  const float u2 = fmaf(absv, c.rn, kRoundShift);
+  const float4 e = bin[(int)(__float_as_uint(u2) >> kKeyShift) - kKeyMin];
+  float X = fmaf(u2, e.y, e.x);
+  X = fmaf(__saturatef(__fsub_rn(u2, e.z)), e.w, X);
+  const float mb = __uint_as_float(0x4B000000u | (word >> 9));                    // 2^23 + (m >> 1), exact
+  const float D = fmaf(mb, c.neg_qscale, X);                                       // S (F - r) + S / 2
+  const float Z = __fadd_rn(D, c.magic);
+  const float rho = __fsub_rn(D, __fsub_rn(Z, c.magic));                            // D minus the nearest multiple of S
+  *unsafe = fabsf(rho) > c.thr;
+  return __float_as_uint(Z);
+}
+
+// The four coordinates of a quad as 6-bit codes, one per byte: level index, bit 5 the sign of a
+// nonzero level.
+__device__ __forceinline__ uint32_t quantize_quad_codes(const float4 x, const uint4 w, const RoundConsts& c, float norm,
+                                                        const float4* bin, const float* lev, int nlev) {
+  bool u0, u1, u2, u3;
+  const uint32_t z0 = round_fast(fabsf(x.x), c, bin, w.x, &u0);
+  const uint32_t z1 = round_fast(fabsf(x.y), c, bin, w.y, &u1);
+  const uint32_t z2 = round_fast(fabsf(x.z), c, bin, w.z, &u2);
+  const uint32_t z3 = round_fast(fabsf(x.w), c, bin, w.w, &u3);
+  uint32_t idx4 = prmt(prmt(z0, z1, 0x0040u), prmt(z2, z3, 0x0040u), 0x5410u);    // the low bytes
+  if (u0 | u1 | u2 | u3) {
+    uint32_t i0 = idx4 & 0xffu, i1 = (idx4 >> 8) & 0xffu, i2 = (idx4 >> 16) & 0xffu, i3 = idx4 >> 24;
+    if (u0) i0 = (uint32_t)quantize_level_slow(fabsf(x.x), norm, lev, nlev, w.x);
+    if (u1) i1 = (uint32_t)quantize_level_slow(fabsf(x.y), norm, lev, nlev, w.y);
+    if (u2) i2 = (uint32_t)quantize_level_slow(fabsf(x.z), norm, lev, nlev, w.z);
+    if (u3) i3 = (uint32_t)quantize_level_slow(fabsf(x.w), norm, lev, nlev, w.w);
+    idx4 = i0 | (i1 << 8) | (i2 << 16) | (i3 << 24);
+  }
+  // sign bytes (0x00 / 0xff) of the four floats, kept at bit 5 where the level is not zero
+  const uint32_t s4 = prmt(prmt(__float_as_uint(x.x), __float_as_uint(x.y), 0x00fbu),
+                           prmt(__float_as_uint(x.z), __float_as_uint(x.w), 0x00fbu), 0x5410u);
+  const uint32_t nz = (idx4 + 0x1f1f1f1fu) & 0x20202020u;                          // level indices are < 0x20
+  return idx4 | (s4 & nz);
+}
+
 // reciprocal of a bucket norm for quantize_fast; 0 sends every coordinate to the exact routine
 // (u' = 0 is never further than the margin from the lower end of its interval)
 __device__ __forceinline__ float fast_reciprocal(float norm, int steps) {
@@ -240,6 +335,7 @@ struct ExchangeUpdate {
 qgx_status check_levels_host(const float* lev, int nlev);
 qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out);
 void make_quant_table(const float* lev, int nlev, QuantTable* out);
+void make_round_table(const float* lev, int nlev, RoundTable* out);
 void* ws_get(qgx_ctx* c, int which, size_t bytes);          // nullptr on failure
 qgx_status cuda_status(cudaError_t e);
 inline void count_launch(qgx_ctx* c, int n = 1) { c->launches += (uint64_t)n; }

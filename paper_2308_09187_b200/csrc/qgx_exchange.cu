@@ -154,9 +154,9 @@ template <int V4, int G>
 __global__ void __launch_bounds__(V4 == 8 ? 512 : (V4 == 4 ? 512 : 256), V4 == 8 ? 2 : 1)
 k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
-                  const __grid_constant__ QuantTable qt) {
+                  const __grid_constant__ RoundTable rt) {
   extern __shared__ __align__(16) uint32_t s_dyn[];
-  __shared__ QuantTable s_q;
+  __shared__ float4 s_bin[kKeyBins];
   __shared__ EncLut s_lut;
   __shared__ uint32_t s_pair[kPairLutSize];
   __shared__ float s_lev[QGX_MAX_LEVELS];
@@ -174,18 +174,13 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   constexpr int kSegs = 32 / kSegLanes;                 // sub-blocks per chunk of 128 coordinates
 
   fill_enc_lut(&s_lut, ct);
-  {
-    const uint32_t* src = reinterpret_cast<const uint32_t*>(&qt);
-    uint32_t* dst = reinterpret_cast<uint32_t*>(&s_q);
-    for (int i = threadIdx.x; i < (int)(sizeof(QuantTable) / 4); i += blockDim.x) dst[i] = src[i];
-  }
+  fill_bin_table(s_bin, rt);
   if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 1.0f;
   if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
   for (int i = threadIdx.x; i < 2 * img_words; i += blockDim.x) s_dyn[i] = 0;
   __syncthreads();
   fill_pair_lut(s_pair, &s_lut);
   __syncthreads();
-  const int steps = s_q.steps;
   const int nlev = lt.nlev;
   uint32_t used_words[2] = {0u, 0u};                    // words of each image that the last bucket in it dirtied
 
@@ -207,7 +202,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     const float norm = bucket_norm_all<V4>(r, a.norm_type, s_red[par]);      // barrier inside: the image is zero
     const bool finite = (norm - norm) == 0.0f;
-    const float rn = fast_reciprocal(norm, steps);
+    const RoundConsts rc = round_consts(rt, norm);
     if (threadIdx.x == 0) {
       a.norms[k * a.nb + b] = norm;
       if (!finite) latch_error(a.st, QGX_ERR_NONFINITE);
@@ -224,16 +219,16 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     for (int j = 0; j < V4; ++j) {
       const int q = (warp * V4 + j) * 32 + lane;
       const int nvalid = whole ? kQuad : max(0, min(kQuad, len - q * kQuad));
-      uint32_t sym4 = 0;
+      uint32_t code4 = 0;
       if (live && nvalid > 0) {
         const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + (uint64_t)q;
         const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
-        sym4 = quad_symbols(r.x[j], quantize_quad(r.x[j], w, rn, norm, &s_q, s_lev, nlev));
+        code4 = quantize_quad_codes(r.x[j], w, rc, norm, s_bin, s_lev, nlev);
       }
       if (nvalid == kQuad) {
-        pack_quad_pairs(sym4, s_pair, &qbits[j], &qn[j]);
-      } else {
-        pack_quad(sym4, nvalid, &s_lut, &qbits[j], &qn[j]);      // the ragged end of a bucket
+        pack_quad_codes(code4, s_pair, &qbits[j], &qn[j]);
+      } else {                                                   // the ragged end of a bucket
+        pack_quad((code4 & 0x1f1f1f1fu) | ((code4 & 0x20202020u) << 2), nvalid, &s_lut, &qbits[j], &qn[j]);
       }
     }
     // warp scans of the bit counts, two chunks per 32-bit word (a chunk holds at most 32 * 52 bits);
@@ -654,8 +649,8 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
     norms_prev = (const float*)c->ws[slot == 0 ? WS_NORMS2 : WS_NORMS];
   }
   const PhiloxKey key = make_philox_key(cfg->seed);
-  QuantTable qt;
-  make_quant_table(cfg->levels, cfg->nlev, &qt);
+  RoundTable qt;
+  make_round_table(cfg->levels, cfg->nlev, &qt);
   if (!ct.has_header || bucket % ct.G != 0 || (ct.G != 32 && ct.G != 64 && ct.G != 128)) return QGX_ERR_INVALID_ARG;
   const int v4 = bucket_v4(bucket);
   const int threads = bucket_threads(bucket, v4);
