@@ -53,42 +53,6 @@ qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out) {
   return QGX_OK;
 }
 
-// tau(u) by definition: the largest j <= nlev - 2 with l_j <= u
-static int tau_of(const float* lev, int nlev, float u) {
-  int tau = 0;
-  for (int j = 1; j <= nlev - 2; ++j)
-    if (lev[j] <= u) tau = j;
-  return tau;
-}
-
-void make_quant_table(const float* lev, int nlev, QuantTable* out) {
-  std::memset(out, 0, sizeof(*out));
-  out->nlev = nlev;
-  for (int t = 0; t < QGX_MAX_LEVELS; ++t)
-    out->upper[t] = make_float2(t + 1 <= nlev - 2 ? lev[t + 1] : 3.0f, t + 2 <= nlev - 2 ? lev[t + 2] : 3.0f);
-  for (int t = 0; t <= nlev - 2; ++t) {
-    const float width = lev[t + 1] - lev[t];                       // the fp32 difference the exact routine divides by
-    const double scale = 8388608.0 / (double)width;
-    const float margin = (float)(4.0 * (double)lev[t + 1] / (double)width + 10.0) * 1.0001f;
-    out->interval[t] = make_float4(lev[t], (float)scale, margin, 0.0f);
-  }
-  for (int t = nlev - 1; t < QGX_MAX_LEVELS; ++t) out->interval[t] = make_float4(0.f, 0.f, 3.0e38f, 0.0f);   // never "safe"
-  int steps = 0;
-  for (int b = 0; b < kKeyBins; ++b) {
-    // bin b holds patterns [(b + kKeyMin) << 17, (b + 1 + kKeyMin) << 17); bin 0 also everything below
-    uint32_t lo_bits = (uint32_t)(b + kKeyMin) << kKeyShift, hi_bits = ((uint32_t)(b + 1 + kKeyMin) << kKeyShift) - 1u;
-    float lo, hi;
-    std::memcpy(&lo, &lo_bits, 4);
-    std::memcpy(&hi, &hi_bits, 4);
-    if (b == 0) lo = 0.0f;
-    if (hi > 1.0f) hi = 1.0f;
-    const int t_lo = tau_of(lev, nlev, lo), t_hi = tau_of(lev, nlev, hi);
-    out->start[b] = (uint8_t)t_lo;
-    steps = std::max(steps, t_hi - t_lo);
-  }
-  out->steps = steps;
-}
-
 // Tables of round_fast.  The margin bounds, in units of 1 / S of an interval, everything by which the
 // kernel's S (F - r) can differ from the exact routine's decision variable: u2 against the correctly
 // rounded quotient and the rounding of b and of the knot (together under 2 * 2^-22 (l_{tau+1} + 2^-16) / width,

@@ -54,9 +54,7 @@ __device__ __forceinline__ void fill_pair_lut(uint32_t* pair, const EncLut* lut)
   }
 }
 
-// stream bits of a full quad of symbols (bytes: level | sign << 7) through the pair table
-__device__ __forceinline__ void pack_quad_pairs(uint32_t sym4, const uint32_t* pair, uint64_t* bits, uint32_t* nbits);
-// the same from 6-bit codes (level | sign << 5), one per byte
+// stream bits of a full quad of 6-bit codes (level | sign << 5, one per byte) through the pair table
 __device__ __forceinline__ void pack_quad_codes(uint32_t t, const uint32_t* pair, uint64_t* bits, uint32_t* nbits) {
   const uint32_t e01 = pair[(t & 0x3fu) | ((t >> 2) & 0xfc0u)];
   const uint32_t e23 = pair[((t >> 16) & 0x3fu) | ((t >> 18) & 0xfc0u)];
@@ -66,17 +64,6 @@ __device__ __forceinline__ void pack_quad_codes(uint32_t t, const uint32_t* pair
   *bits = ((uint64_t)hi << 32) | lo;
   *nbits = n01 + n23;
 }
-__device__ __forceinline__ void pack_quad_pairs(uint32_t sym4, const uint32_t* pair, uint64_t* bits, uint32_t* nbits) {
-  const uint32_t t = (sym4 & 0x1f1f1f1fu) | ((sym4 >> 2) & 0x20202020u);        // 6-bit code in every byte
-  const uint32_t e01 = pair[(t & 0x3fu) | ((t >> 2) & 0xfc0u)];
-  const uint32_t e23 = pair[((t >> 16) & 0x3fu) | ((t >> 18) & 0xfc0u)];
-  const uint32_t b01 = e01 & 0x3ffffffu, n01 = e01 >> 26, b23 = e23 & 0x3ffffffu, n23 = e23 >> 26;
-  const uint32_t lo = b01 | (b23 << n01);
-  const uint32_t hi = __funnelshift_l(b23, 0u, n01);
-  *bits = ((uint64_t)hi << 32) | lo;
-  *nbits = n01 + n23;
-}
-
 // OR `nbits` (<= 52) bits into the bucket image at bit position pos (shared memory, zeroed before).
 // Two words are always touched; a third only when the bits reach it.
 __device__ __forceinline__ void put_bits(uint32_t* img, uint32_t pos, uint64_t bits, uint32_t nbits) {

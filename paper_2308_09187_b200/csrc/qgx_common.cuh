@@ -55,20 +55,10 @@ struct LevelTable {
   float lev[QGX_MAX_LEVELS];
 };
 
-// Tables of the fast rounding path (see quantize_fast): a 1025-entry map from the top bits of the
-// float pattern of u to a lower bound of tau(u), and per interval the level, 2^23 / width, the
-// rounding margin and 2^23 - margin.
+// bins of the rounding table over the float pattern of the normalized coordinate (see round_fast)
 constexpr int kKeyShift = 17;                       // 64 bins per octave of u
 constexpr int kKeyMin = 0x37800000 >> kKeyShift;    // pattern of 2^-16: everything below shares bin 0
 constexpr int kKeyBins = (0x3F800000 >> kKeyShift) - kKeyMin + 1;   // up to u = 1.0: 1025 bins
-struct QuantTable {
-  int nlev;
-  int steps;                             // compare steps after the table look-up
-  float4 interval[QGX_MAX_LEVELS];       // {l_tau, 2^23 / (l_{tau+1} - l_tau), margin, unused}
-  float2 upper[QGX_MAX_LEVELS];          // upper[t] = {l_{t+1}, l_{t+2}} while those are interior levels, else a value above 1
-  uint8_t start[kKeyBins + 3];
-};
-
 struct CodeTable {
   int nlev;
   int maxlen;
@@ -140,56 +130,6 @@ __device__ __forceinline__ int quantize_level(float absv, float norm, const floa
 // The exact routine as one out-of-line copy (it runs for about 1e-5 of the coordinates).
 static __device__ __noinline__ int quantize_level_slow(float absv, float norm, const float* lev, int nlev, uint32_t word) {
   return quantize_level(absv, norm, lev, nlev, word);
-}
-
-// Same decision as quantize_level, without divisions in the common case.  With rn = RN(1/norm),
-// u' = RN(|v| rn) differs from the exact u = RN(|v| / norm) by at most 2^-22 u.  tau is found from a
-// table on the float pattern of u' plus two comparisons (tables that would need more send every
-// coordinate to the exact routine); T = (u' - l_tau) 2^23 / width differs from xi 2^23 by less than
-// margin = 4 l_{tau+1} / width + 10.  The 24-bit variate m rounds up iff m < xi 2^24; with m' = m >> 1
-// taken as a float through the 2^23 trick, the sign of T - m' decides whenever |T - m'| > margin and T
-// is further than margin from both ends of the interval (so that u' and u lie in the same interval).
-// Returns the level index and sets *unsafe when the exact routine has to decide instead.
-__device__ __forceinline__ int quantize_fast(float absv, float rn, const QuantTable* q, uint32_t word, bool* unsafe) {
-  const float u = fminf(__fmul_rn(absv, rn), 1.0f);
-  const int key = max((int)(__float_as_uint(u) >> kKeyShift), kKeyMin) - kKeyMin;
-  const int tau0 = q->start[key];
-  const float2 up = q->upper[tau0];
-  const int tau = tau0 + ((up.x <= u) ? 1 : 0) + ((up.y <= u) ? 1 : 0);
-  const float4 iv = q->interval[tau];
-  // T + 2^23: the addition rounds T to an integer (error 1/2, inside the margin)
-  const float Tb = fmaf(u - iv.x, iv.y, 8388608.0f);
-  const float mb = __uint_as_float(0x4B000000u | (word >> 9));                    // 2^23 + (m >> 1), exact
-  const float diff = Tb - mb;
-  // a zero coordinate is level 0 whatever the variate (T = 0, diff <= 0), so it needs no second look
-  *unsafe = (absv != 0.0f) && !(fabsf(diff) > iv.z && fabsf(Tb - 12582912.0f) < 4194304.0f - iv.z);
-  return tau + (diff > 0.0f ? 1 : 0);
-}
-
-// Level indices of the four coordinates of a quad, packed one per byte (no sign).
-__device__ __forceinline__ uint32_t quantize_quad(const float4 x, const uint4 w, float rn, float norm, const QuantTable* q,
-                                                  const float* lev, int nlev) {
-  bool u0, u1, u2, u3;
-  int i0 = quantize_fast(fabsf(x.x), rn, q, w.x, &u0);
-  int i1 = quantize_fast(fabsf(x.y), rn, q, w.y, &u1);
-  int i2 = quantize_fast(fabsf(x.z), rn, q, w.z, &u2);
-  int i3 = quantize_fast(fabsf(x.w), rn, q, w.w, &u3);
-  if (u0 | u1 | u2 | u3) {
-    if (u0) i0 = quantize_level_slow(fabsf(x.x), norm, lev, nlev, w.x);
-    if (u1) i1 = quantize_level_slow(fabsf(x.y), norm, lev, nlev, w.y);
-    if (u2) i2 = quantize_level_slow(fabsf(x.z), norm, lev, nlev, w.z);
-    if (u3) i3 = quantize_level_slow(fabsf(x.w), norm, lev, nlev, w.w);
-  }
-  return (uint32_t)i0 | ((uint32_t)i1 << 8) | ((uint32_t)i2 << 16) | ((uint32_t)i3 << 24);
-}
-
-// sign bits of the four coordinates, at bits 7, 15, 23, 31, dropped where the level index is zero
-__device__ __forceinline__ uint32_t quad_symbols(const float4 x, uint32_t idx4) {
-  const uint32_t s = ((__float_as_uint(x.x) >> 31) << 7) | ((__float_as_uint(x.y) >> 31) << 15) |
-                     ((__float_as_uint(x.z) >> 31) << 23) | ((__float_as_uint(x.w) >> 31) << 31);
-  // a byte of idx4 is nonzero iff (byte + 0x7f) has bit 7 set (level indices are < 0x80)
-  const uint32_t nz = (idx4 + 0x7f7f7f7fu) & 0x80808080u;
-  return idx4 | (s & nz);
 }
 
 // ---- rounding through the level map -----------------------------------------------------------
@@ -287,12 +227,6 @@ __device__ __forceinline__ uint32_t quantize_quad_codes(const float4 x, const ui
   return idx4 | (s4 & nz);
 }
 
-// reciprocal of a bucket norm for quantize_fast; 0 sends every coordinate to the exact routine
-// (u' = 0 is never further than the margin from the lower end of its interval)
-__device__ __forceinline__ float fast_reciprocal(float norm, int steps) {
-  return (norm > 7.9e-31f && norm < 1.2e30f && steps <= 2) ? __frcp_rn(norm) : 0.0f;
-}
-
 __device__ __forceinline__ uint32_t symbol_of(float v, int idx) {
   const uint32_t neg = (__float_as_uint(v) >> 31) & (idx != 0 ? 1u : 0u);
   return (uint32_t)idx | (neg << 7);
@@ -334,7 +268,6 @@ struct ExchangeUpdate {
 // host side
 qgx_status check_levels_host(const float* lev, int nlev);
 qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out);
-void make_quant_table(const float* lev, int nlev, QuantTable* out);
 void make_round_table(const float* lev, int nlev, RoundTable* out);
 void* ws_get(qgx_ctx* c, int which, size_t bytes);          // nullptr on failure
 qgx_status cuda_status(cudaError_t e);

@@ -7,16 +7,12 @@ namespace qgx {
 // the rounding pass, so v is read from HBM exactly once.
 template <int V4>
 __global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int bucket, const __grid_constant__ LevelTable lt,
-                                                   const __grid_constant__ PhiloxKey key, const __grid_constant__ QuantTable qt,
+                                                   const __grid_constant__ PhiloxKey key, const __grid_constant__ RoundTable rt,
                                                    uint32_t xid, int norm_type, int norms_supplied, bool vec_ok,
                                                    float* __restrict__ norms, uint8_t* __restrict__ sym, DevStatus* st) {
   __shared__ float s_lev[QGX_MAX_LEVELS];
-  __shared__ QuantTable s_q;
-  {
-    const uint32_t* qsrc = reinterpret_cast<const uint32_t*>(&qt);
-    uint32_t* qdst = reinterpret_cast<uint32_t*>(&s_q);
-    for (int i = threadIdx.x; i < (int)(sizeof(QuantTable) / 4); i += blockDim.x) qdst[i] = qsrc[i];
-  }
+  __shared__ float4 s_bin[kKeyBins];
+  fill_bin_table(s_bin, rt);
   __shared__ double s_red[34];
   const size_t b = blockIdx.x, k = blockIdx.y;
   const size_t nb = gridDim.x;
@@ -36,7 +32,7 @@ __global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int 
   }
   const bool finite = (norm - norm) == 0.0f;
   if (!finite && threadIdx.x == 0) latch_error(st, QGX_ERR_NONFINITE);
-  const float rn = fast_reciprocal(norm, s_q.steps);
+  const RoundConsts rc = round_consts(rt, norm);
 
   uint8_t* out = sym + k * d + lo;
   const bool sym_vec = vec_ok;            // d % 4 == 0 and bucket % 4 == 0: every quad is 4-byte aligned
@@ -50,7 +46,8 @@ __global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int 
       const uint64_t ctr = (uint64_t)(lo >> 2) + (uint64_t)q;      // (coordinate index) / 4
       const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, xid, key);
       const float4 x = r.x[j];
-      packed = quad_symbols(x, quantize_quad(x, w, rn, norm, &s_q, s_lev, lt.nlev));
+      const uint32_t code4 = quantize_quad_codes(x, w, rc, norm, s_bin, s_lev, lt.nlev);
+      packed = (code4 & 0x1f1f1f1fu) | ((code4 & 0x20202020u) << 2);      // symbol bytes: level | sign << 7
     }
     if (e + kQuad <= len && sym_vec) {
       *reinterpret_cast<uint32_t*>(out + e) = packed;
@@ -109,8 +106,8 @@ qgx_status launch_quantize(qgx_ctx* c, DualSource src, int K, size_t d, int buck
   const bool vec_ok = (d % kQuad == 0) && all_aligned16({src.v, src.a}) &&
                       ((reinterpret_cast<uintptr_t>(sym) & 3u) == 0);
   const PhiloxKey key = make_philox_key(seed);
-  QuantTable qt;
-  make_quant_table(lt.lev, lt.nlev, &qt);
+  RoundTable qt;
+  make_round_table(lt.lev, lt.nlev, &qt);
   const int v4 = bucket_v4(bucket);
   const dim3 grid((unsigned)nb, (unsigned)K);
   const int threads = bucket_threads(bucket, v4);

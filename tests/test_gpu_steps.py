@@ -89,6 +89,49 @@ def test_quantize_encode_decode_average(q, K, d, bucket, nlev, sub):
     assert np.array_equal(out.cpu().numpy(), o.average(n_gpu, s_ref, bucket, lev))
 
 
+LEVEL_SETS = {
+    "uniform17": np.linspace(0, 1, 17),
+    "uniform32": np.linspace(0, 1, 32),
+    "exponential": np.r_[0.0, 2.0 ** np.arange(-15, 1)],
+    "below_2^-16": np.r_[0.0, 3e-6, 1.1e-5, 4e-4, 2e-2, 1.0],
+    "two_levels_in_one_bin": np.r_[0.0, 0.01, 0.5, 0.5005, 0.501, 1.0],      # every coordinate takes the exact routine
+    "narrow_interval": np.r_[0.0, 0.05, 0.25, 0.2500004, 0.7, 1.0],
+    "two": np.r_[0.0, 1.0],
+}
+
+
+@pytest.mark.parametrize("name", sorted(LEVEL_SETS))
+def test_rounding_agrees_with_definition_1_on_awkward_levels(q, name):
+    """Symbols bit for bit on level sets that stress the kernel's rounding tables, with coordinates
+    placed on the levels, next to them, at zero and at |v| = norm."""
+    qgx, ctx = q
+    lev = LEVEL_SETS[name].astype(np.float32)
+    K, d, bucket = 2, 1 << 18, 4096
+    v = gen.gaussian((K, d), seed=77, device="cuda").cpu().numpy()
+    rng = np.random.default_rng(5)
+    v[0, :d // 2] = (rng.random(d // 2) ** 4).astype(np.float32) * np.sign(v[0, :d // 2]) * 60.0      # spread over all octaves
+    nb = d // bucket
+    # second worker: buckets whose coordinates sit on multiples of the levels
+    for b in range(0, nb, 2):
+        seg = v[1, b * bucket:(b + 1) * bucket]
+        seg[:] = 0.0
+        seg[0] = 100.0                                  # dominates the norm: u = l_j reproduced closely below
+        j = rng.integers(0, len(lev), bucket - 1)
+        off = rng.integers(-2, 3, bucket - 1)
+        val = lev[j] * np.float32(100.0)
+        for _ in range(2):
+            val = np.where(off > 0, np.nextafter(val, np.float32(np.inf)), np.where(off < 0, np.nextafter(val, np.float32(0)), val))
+        seg[1:] = val * np.where(rng.random(bucket - 1) < 0.5, -1, 1)
+    v[1, bucket:2 * bucket] = 0.0
+    v[1, bucket + 5] = -3.0                             # a bucket with one nonzero coordinate: u = 1
+    vd = torch.from_numpy(v).cuda()
+    for norm_type in (qgx.QGX_NORM_L2, qgx.QGX_NORM_LINF):
+        norms, sym = qgx.qgx_quantize(ctx, vd, bucket, lev, norm_type, 99, 4)
+        qgx.qgx_sync_status(ctx)
+        n_gpu = norms.cpu().numpy()
+        assert np.array_equal(sym.cpu().numpy(), o.quantize(v, bucket, lev, n_gpu, 99, 4))
+
+
 def test_linf_norm_and_heavy_tails(q):
     qgx, ctx = q
     K, d, bucket = 2, 9000, 4096
