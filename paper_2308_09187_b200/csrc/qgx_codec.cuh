@@ -74,6 +74,25 @@ __device__ __forceinline__ void put_bits(uint32_t* img, uint32_t pos, uint64_t b
   if (sh + nbits > 64u) atomicOr(&img[w + 2], __funnelshift_l(bhi, 0u, sh));
 }
 
+// Two adjacent runs (a first, then b; each <= 52 bits) as one value of up to 104 bits.  Two words are
+// always touched, further ones only when the bits reach them.
+__device__ __forceinline__ void put_bits2(uint32_t* img, uint32_t pos, uint64_t a, uint32_t na, uint64_t b, uint32_t nb) {
+  const uint64_t lo = a | (b << na);
+  const uint64_t hi = (b >> 1) >> (63u - na);           // the bits of b past bit 63 (none when na == 0)
+  const uint32_t n = na + nb;
+  const uint32_t w = pos >> 5, sh = pos & 31u;
+  const uint32_t m0 = (uint32_t)lo, m1 = (uint32_t)(lo >> 32), m2 = (uint32_t)hi, m3 = (uint32_t)(hi >> 32);
+  atomicOr(&img[w], m0 << sh);
+  atomicOr(&img[w + 1], __funnelshift_l(m0, m1, sh));
+  if (sh + n > 64u) {
+    atomicOr(&img[w + 2], __funnelshift_l(m1, m2, sh));
+    if (sh + n > 96u) {
+      atomicOr(&img[w + 3], __funnelshift_l(m2, m3, sh));
+      if (sh + n > 128u) atomicOr(&img[w + 4], __funnelshift_l(m3, 0u, sh));
+    }
+  }
+}
+
 // Decoder table: index = next `maxlen` stream bits, entry = level | codeword length << 8 (0 = no
 // codeword starts with these bits).
 constexpr int kDecLutMax = 1 << QGX_MAX_CODE_LEN;

@@ -113,6 +113,25 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
   return make_uint4(c0, c1, c2, c3);
 }
 
+// two blocks that share the last two counter words, round by round (the round keys are fetched once)
+__device__ __forceinline__ void philox4x32_10_x2(uint64_t ctr_a, uint64_t ctr_b, uint32_t c2, uint32_t c3, const PhiloxKey& key,
+                                                 uint4* out_a, uint4* out_b) {
+  uint32_t a0 = (uint32_t)ctr_a, a1 = (uint32_t)(ctr_a >> 32), a2 = c2, a3 = c3;
+  uint32_t b0 = (uint32_t)ctr_b, b1 = (uint32_t)(ctr_b >> 32), b2 = c2, b3 = c3;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t k0 = key.k0[r], k1 = key.k1[r];
+    const uint64_t pa0 = (uint64_t)0xD2511F53u * (uint64_t)a0, pa1 = (uint64_t)0xCD9E8D57u * (uint64_t)a2;
+    const uint64_t pb0 = (uint64_t)0xD2511F53u * (uint64_t)b0, pb1 = (uint64_t)0xCD9E8D57u * (uint64_t)b2;
+    const uint32_t na0 = (uint32_t)(pa1 >> 32) ^ a1 ^ k0, na2 = (uint32_t)(pa0 >> 32) ^ a3 ^ k1;
+    const uint32_t nb0 = (uint32_t)(pb1 >> 32) ^ b1 ^ k0, nb2 = (uint32_t)(pb0 >> 32) ^ b3 ^ k1;
+    a0 = na0; a1 = (uint32_t)pa1; a2 = na2; a3 = (uint32_t)pa0;
+    b0 = nb0; b1 = (uint32_t)pb1; b2 = nb2; b3 = (uint32_t)pb0;
+  }
+  *out_a = make_uint4(a0, a1, a2, a3);
+  *out_b = make_uint4(b0, b1, b2, b3);
+}
+
 // ---- Definition 1 for one normalized coordinate, every operation one IEEE rounding ----------
 // returns the level index; lev points to the table in shared memory
 __device__ __forceinline__ int quantize_level(float absv, float norm, const float* lev, int nlev, uint32_t word) {

@@ -112,16 +112,16 @@ __device__ __forceinline__ float bucket_norm_all(const BucketRegs<V4>& r, int no
   return bad ? __int_as_float(0x7fc00000) : m;
 }
 
-// Loads bucket [lo, lo + len) of worker k, warp-major: warp w holds quads [w * V4 * 32, (w + 1) * V4 * 32),
-// its j-th load covering 32 consecutive quads (512 contiguous bytes), lane l the l-th of them.
-template <int V4>
-__device__ __forceinline__ void load_bucket_warp_major(BucketRegs<V4>& r, const DualSource& s, size_t k, size_t d,
-                                                       size_t lo, int len, bool vec_ok) {
+// Loads bucket [lo, lo + len) of worker k: warp w holds coordinates [w * 256 * P, (w + 1) * 256 * P), row j of
+// them 32 octets (8 consecutive coordinates: two quads), lane l the l-th octet of the row.
+template <int P>
+__device__ __forceinline__ void load_bucket_octets(BucketRegs<2 * P>& r, const DualSource& s, size_t k, size_t d,
+                                                   size_t lo, int len, bool vec_ok) {
   const size_t ld = s.ld ? s.ld : d;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-  for (int j = 0; j < V4; ++j) {
-    const int e = ((warp * V4 + j) * 32 + lane) * kQuad;
+  for (int j = 0; j < 2 * P; ++j) {
+    const int e = ((((warp * P + (j >> 1)) * 32 + lane) << 1) + (j & 1)) * kQuad;
     float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
     if (e + kQuad <= len && vec_ok) {
       if (s.a == nullptr) {
@@ -149,9 +149,9 @@ __device__ __forceinline__ void load_bucket_warp_major(BucketRegs<V4>& r, const 
 //   loads, zero the image | barrier | norm, Philox, rounding, packing, sub-block lengths, warp scans |
 //   barrier | warp offsets, bit scatter, look-back (warp 0) | barrier | copy out
 // The bucket image is double buffered, so the copy-out of one bucket needs no barrier before the next
-// bucket starts.  Warp w owns the 128 * V4 coordinates [w * 128 * V4, ...) of the bucket.
-template <int V4, int G>
-__global__ void __launch_bounds__(V4 == 8 ? 512 : (V4 == 4 ? 512 : 256), V4 == 8 ? 2 : 1)
+// bucket starts.  A thread works on P octets; warp w owns the 256 * P coordinates [w * 256 * P, ...).
+template <int P, int G>
+__global__ void __launch_bounds__(P == 1 ? 256 : 512, P == 4 ? 2 : 1)
 k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
                   const __grid_constant__ RoundTable rt) {
@@ -170,8 +170,9 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   // words of one image, a multiple of 4 so that both images are 16-byte aligned
   const int img_words = (int)((((((uint32_t)a.bucket * (uint32_t)(ct.maxlen + 1) + 16u * (uint32_t)(a.bucket / G + 1) + kNormBits + 31u) >> 5) + 4) + 3u) & ~3u);
   const unsigned long long total = (unsigned long long)a.nb * (unsigned long long)a.K;
-  constexpr int kSegLanes = G / kQuad;                  // lanes per sub-block within a warp's 128 coordinates
-  constexpr int kSegs = 32 / kSegLanes;                 // sub-blocks per chunk of 128 coordinates
+  constexpr int kOctet = 2 * kQuad;
+  constexpr int kSegLanes = G / kOctet;                 // lanes per sub-block within a row of 256 coordinates
+  constexpr int kSegs = 32 / kSegLanes;                 // sub-blocks per row
 
   fill_enc_lut(&s_lut, ct);
   fill_bin_table(s_bin, rt);
@@ -192,15 +193,15 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     const int len = (int)min((size_t)a.bucket, a.d - lo);
     uint32_t* s_img = s_dyn + par * img_words;
 
-    BucketRegs<V4> r;
-    load_bucket_warp_major<V4>(r, a.src, k, a.d, lo, len, a.vec_ok);
+    BucketRegs<2 * P> r;
+    load_bucket_octets<P>(r, a.src, k, a.d, lo, len, a.vec_ok);
     {
       // this image was last read by the copy-out two buckets ago; two barriers have passed since
       uint4* z = reinterpret_cast<uint4*>(s_img);
       const int n4 = (int)((used_words[par] + 3u + 3u) >> 2);
       for (int i = threadIdx.x; i < n4; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
     }
-    const float norm = bucket_norm_all<V4>(r, a.norm_type, s_red[par]);      // barrier inside: the image is zero
+    const float norm = bucket_norm_all<2 * P>(r, a.norm_type, s_red[par]);   // barrier inside: the image is zero
     const bool finite = (norm - norm) == 0.0f;
     const RoundConsts rc = round_consts(rt, norm);
     if (threadIdx.x == 0) {
@@ -210,47 +211,56 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     const uint32_t nsub = (uint32_t)((len + G - 1) / G);
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
-    const bool whole = (len == a.bucket) && a.vec_ok;     // no ragged end: no per-quad checks
+    const bool whole = (len == a.bucket) && a.vec_ok && (a.bucket % (32 * kOctet * P) == 0);   // every lane holds full octets: no checks
     const bool live = finite && norm != 0.0f;             // otherwise every coordinate is level 0
 
-    uint64_t qbits[V4];
-    uint32_t qn[V4], qoff[V4];
+    uint64_t qbits[2 * P];
+    uint32_t qn[P], qoff[P];                              // qn: bits of the first quad | bits of the second << 8
 #pragma unroll
-    for (int j = 0; j < V4; ++j) {
-      const int q = (warp * V4 + j) * 32 + lane;
-      const int nvalid = whole ? kQuad : max(0, min(kQuad, len - q * kQuad));
-      uint32_t code4 = 0;
-      if (live && nvalid > 0) {
-        const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + (uint64_t)q;
-        const uint4 w = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), (uint32_t)k, a.xid, key);
-        code4 = quantize_quad_codes(r.x[j], w, rc, norm, s_bin, s_lev, nlev);
+    for (int j = 0; j < P; ++j) {
+      const int o = (warp * P + j) * 32 + lane;           // octet of the bucket
+      const int nv0 = whole ? kQuad : max(0, min(kQuad, len - o * kOctet));
+      const int nv1 = whole ? kQuad : max(0, min(kQuad, len - o * kOctet - kQuad));
+      uint32_t code0 = 0, code1 = 0;
+      if (live && nv0 > 0) {
+        const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + 2ull * (uint64_t)o;
+        uint4 w0, w1;
+        philox4x32_10_x2(ctr, ctr + 1ull, (uint32_t)k, a.xid, key, &w0, &w1);
+        code0 = quantize_quad_codes(r.x[2 * j], w0, rc, norm, s_bin, s_lev, nlev);
+        code1 = quantize_quad_codes(r.x[2 * j + 1], w1, rc, norm, s_bin, s_lev, nlev);
       }
-      if (nvalid == kQuad) {
-        pack_quad_codes(code4, s_pair, &qbits[j], &qn[j]);
-      } else {                                                   // the ragged end of a bucket
-        pack_quad((code4 & 0x1f1f1f1fu) | ((code4 & 0x20202020u) << 2), nvalid, &s_lut, &qbits[j], &qn[j]);
+      uint32_t n0, n1;
+      if (nv1 == kQuad) {
+        pack_quad_codes(code0, s_pair, &qbits[2 * j], &n0);
+        pack_quad_codes(code1, s_pair, &qbits[2 * j + 1], &n1);
+      } else {                                              // the ragged end of a bucket
+        pack_quad((code0 & 0x1f1f1f1fu) | ((code0 & 0x20202020u) << 2), nv0, &s_lut, &qbits[2 * j], &n0);
+        pack_quad((code1 & 0x1f1f1f1fu) | ((code1 & 0x20202020u) << 2), nv1, &s_lut, &qbits[2 * j + 1], &n1);
       }
+      qn[j] = n0 | (n1 << 8);
     }
-    // warp scans of the bit counts, two chunks per 32-bit word (a chunk holds at most 32 * 52 bits);
-    // qoff[j] becomes the quad's bit offset inside the warp's part of the payload
+    // warp scans of the bit counts, two rows per 32-bit word (a row holds at most 32 * 104 bits);
+    // qoff[j] becomes the octet's bit offset inside the warp's part of the payload
     uint32_t warp_bits = 0;
 #pragma unroll
-    for (int j = 0; j < V4; j += 2) {
-      const uint32_t both = qn[j] | ((j + 1 < V4 ? qn[j + 1] : 0u) << 16);
+    for (int j = 0; j < P; j += 2) {
+      const uint32_t cnt0 = (qn[j] & 0xffu) + (qn[j] >> 8);
+      const uint32_t cnt1 = j + 1 < P ? (qn[j + 1 < P ? j + 1 : j] & 0xffu) + (qn[j + 1 < P ? j + 1 : j] >> 8) : 0u;
+      const uint32_t both = cnt0 | (cnt1 << 16);
       const uint32_t incl = warp_incl_scan(both, lane);
       const uint32_t before = __shfl_up_sync(0xffffffffu, incl, kSegLanes);
       const uint32_t seg = incl - (lane >= kSegLanes ? before : 0u);   // per field: no borrow, the scans are monotone
       const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
-        if (j + h < V4) {
+        if (j + h < P) {
           const uint32_t mine = (incl >> (16 * h)) & 0xffffu;
-          qoff[j + h] = warp_bits + mine - qn[j + h];
+          qoff[j + h < P ? j + h : j] = warp_bits + mine - (h == 0 ? cnt0 : cnt1);
           warp_bits += (tot >> (16 * h)) & 0xffffu;
           // sub-block lengths: the last lane of each sub-block knows its total; the 16-bit fields are
           // halfword aligned, a plain store
           if ((lane + 1) % kSegLanes == 0) {
-            const int sb = (warp * V4 + j + h) * kSegs + lane / kSegLanes;
+            const int sb = (warp * P + j + h) * kSegs + lane / kSegLanes;
             if (whole || sb * G < len) reinterpret_cast<uint16_t*>(s_img)[2 + sb] = (uint16_t)((seg >> (16 * h)) & 0xffffu);
           }
         }
@@ -274,7 +284,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     const uint32_t base = hdr_bits + wbase;
 #pragma unroll
-    for (int j = 0; j < V4; ++j) put_bits(s_img, base + qoff[j], qbits[j], qn[j]);
+    for (int j = 0; j < P; ++j) put_bits2(s_img, base + qoff[j], qbits[2 * j], qn[j] & 0xffu, qbits[2 * j + 1], qn[j] >> 8);
     if (warp == 0) {
       bool timed_out = false;
       const unsigned long long excl = lookback_prefix(row, (long long)b, lane, &timed_out);
@@ -652,8 +662,9 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   RoundTable qt;
   make_round_table(cfg->levels, cfg->nlev, &qt);
   if (!ct.has_header || bucket % ct.G != 0 || (ct.G != 32 && ct.G != 64 && ct.G != 128)) return QGX_ERR_INVALID_ARG;
-  const int v4 = bucket_v4(bucket);
-  const int threads = bucket_threads(bucket, v4);
+  // octets per thread chosen so that CTAs have at most 256 / 512 / 512 threads
+  const int pp = bucket <= 2048 ? 1 : (bucket <= 8192 ? 2 : 4);
+  const int threads = bucket_threads(bucket, 2 * pp);
   const size_t img_words = (((((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4) + 3) & ~(size_t)3;
   const size_t smem = sizeof(uint32_t) * 2 * img_words;   // two images: see k_exchange_encode
   int per_sm = 1;
@@ -674,11 +685,10 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   } while (0)
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_ENCODE);
-    switch (v4) {
+    switch (pp) {
       case 1: QGX_LAUNCH_EG(1); break;
       case 2: QGX_LAUNCH_EG(2); break;
-      case 4: QGX_LAUNCH_EG(4); break;
-      default: QGX_LAUNCH_EG(8); break;
+      default: QGX_LAUNCH_EG(4); break;
     }
   }
 #undef QGX_LAUNCH_EG
