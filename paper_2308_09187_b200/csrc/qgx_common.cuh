@@ -39,6 +39,7 @@ struct qgx_ctx {
   int sym_slot;
   int sym_K;
   size_t sym_d;
+  size_t sym_ld;                         // bytes per worker in the kept-symbol layout
   // optional per-kernel timing: pairs of events recorded around instrumented launches
   int timing_on;
   int timing_cap;                        // pairs allocated

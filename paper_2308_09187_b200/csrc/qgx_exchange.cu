@@ -336,13 +336,15 @@ struct DecodeArgs {
   const double* scalars;        // scalars[1] = gamma_t
   bool vec_out;                 // d % 4 == 0 and mean, xin, xout 16-byte aligned: 128-bit stores
   // optional: keep the decoded symbols (1 byte per coordinate and worker) ...
-  uint8_t* sym_out;             // [K][d] or null
+  // Symbol bytes are kept transposed, so that a warp's accesses coalesce: worker k, sub-block gs, coordinate i of the
+  // sub-block -> byte k * sym_ld + (gs / 32) * 32 * G + (i / 4) * 128 + (gs % 32) * 4 + i % 4.
+  uint8_t* sym_out;             // [K][sym_ld] or null
   // ... or compare with the symbols and norms kept by the other exchange of the iteration:
   // *sum_sq += sum_k ||vhat_k of that exchange - vhat_k of this one||^2 (fp32 differences, fp64 sum)
-  const uint8_t* sym_prev;      // [K][d] or null
+  const uint8_t* sym_prev;      // [K][sym_ld] or null
+  size_t sym_ld;
   const float* norms_prev;      // [K][nb]
   double* sum_sq;
-  bool vec_sym;                 // d % 4 == 0: four symbol bytes move as one word
   DevStatus* st;
 };
 
@@ -490,6 +492,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
     if (!__any_sync(0xffffffffu, count > 0)) continue;   // beyond the end of a short last bucket
     const size_t e0 = lo + (size_t)first;
+    const size_t sbase = (gs >> 5) * (size_t)(32 * G) + (size_t)(gs & 31) * 4;   // see DecodeArgs::sym_out
 
     float acc[G];
 #pragma unroll
@@ -502,14 +505,14 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
       Window win;
       win.open(cur.p, cur.w0, cur.w1, cur.w2, cur.sh);
       uint32_t flags = 0, used = 0;
-      if (count == G && a.vec_sym) {
+      if (count == G) {
         uint32_t pack = 0, prev4 = 0;
 #pragma unroll
         for (int i = 0; i < G; ++i) {
           if ((i & 1) == 0) {                              // two symbols use at most 26 bits
             if (win.avail <= 32) win.refill();
           }
-          if (SYM == 2 && (i & 3) == 0) prev4 = __ldcs(reinterpret_cast<const uint32_t*>(a.sym_prev + (size_t)k * a.d + e0 + i));
+          if (SYM == 2 && (i & 3) == 0) prev4 = __ldcs(reinterpret_cast<const uint32_t*>(a.sym_prev + (size_t)k * a.sym_ld + sbase + (i >> 2) * 128));
           const DecEntry e = s_lut[win.lo & mask];
           const uint32_t L = e.len & 31u;
           flags |= e.len;
@@ -519,7 +522,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
           acc[i] = __fadd_rn(acc[i], val);
           if (SYM == 1) {
             pack |= ((e.len >> 8) & 0xffu) << (8 * (i & 3));
-            if ((i & 3) == 3) { *reinterpret_cast<uint32_t*>(a.sym_out + (size_t)k * a.d + e0 + i - 3) = pack; pack = 0; }
+            if ((i & 3) == 3) { *reinterpret_cast<uint32_t*>(a.sym_out + (size_t)k * a.sym_ld + sbase + (i >> 2) * 128) = pack; pack = 0; }
           }
           if (SYM == 2) {
             const float dlt = __fsub_rn(dequantize_symbol((prev4 >> (8 * (i & 3))) & 0xffu, cur.norm_prev, s_lev), val);
@@ -540,9 +543,9 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
             used += L;
             const float val = __fmul_rn(cur.norm, e.val);
             acc[i] = __fadd_rn(acc[i], val);
-            if (SYM == 1) a.sym_out[(size_t)k * a.d + e0 + i] = (uint8_t)((e.len >> 8) & 0xffu);
+            if (SYM == 1) a.sym_out[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)] = (uint8_t)((e.len >> 8) & 0xffu);
             if (SYM == 2) {
-              const float dlt = __fsub_rn(dequantize_symbol(a.sym_prev[(size_t)k * a.d + e0 + i], cur.norm_prev, s_lev), val);
+              const float dlt = __fsub_rn(dequantize_symbol(a.sym_prev[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)], cur.norm_prev, s_lev), val);
               sq = fma((double)dlt, (double)dlt, sq);
             }
           }
@@ -648,13 +651,14 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(status + (size_t)K * nb); ea.st = c->dstatus;
   uint8_t* sym_out = nullptr;
   const uint8_t* sym_prev = nullptr;
+  const size_t sym_ld = ((nb * (size_t)(bucket / ct.G) + 31) / 32) * 32 * (size_t)ct.G;   // see DecodeArgs::sym_out
   const float* norms_prev = nullptr;
   if (sym_mode == 1) {
-    sym_out = (uint8_t*)ws_get(c, WS_SYM, (size_t)K * d + 16);
+    sym_out = (uint8_t*)ws_get(c, WS_SYM, (size_t)K * sym_ld + 16);
     if (!sym_out) return QGX_ERR_CUDA;
-    c->sym_slot = slot; c->sym_K = K; c->sym_d = d;
+    c->sym_slot = slot; c->sym_K = K; c->sym_d = d; c->sym_ld = sym_ld;
   } else if (sym_mode == 2) {
-    if (!sum_sq || c->sym_slot != 1 - slot || c->sym_K != K || c->sym_d != d || c->slot_nb[1 - slot] != nb) return QGX_ERR_INVALID_ARG;
+    if (!sum_sq || c->sym_slot != 1 - slot || c->sym_K != K || c->sym_d != d || c->sym_ld != sym_ld || c->slot_nb[1 - slot] != nb) return QGX_ERR_INVALID_ARG;
     sym_prev = (const uint8_t*)c->ws[WS_SYM];
     norms_prev = (const float*)c->ws[slot == 0 ? WS_NORMS2 : WS_NORMS];
   }
@@ -719,8 +723,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
 
   DecodeArgs da;
   da.stream = stream; da.cap_words = cap; da.bucket_bits = bbits; da.offsets = offs;
-  da.sym_out = sym_out; da.sym_prev = sym_prev; da.norms_prev = norms_prev; da.sum_sq = sum_sq;
-  da.vec_sym = (d % kQuad == 0);
+  da.sym_out = sym_out; da.sym_prev = sym_prev; da.sym_ld = sym_ld; da.norms_prev = norms_prev; da.sum_sq = sum_sq;
   da.d = d; da.bucket = bucket; da.K = K; da.nb = nb; da.lut = lut; da.mean = mean_out;
   da.update = upd ? upd->mode : 0; da.xin = upd ? upd->xin : nullptr; da.xout = upd ? upd->xout : nullptr;
   da.scalars = upd ? upd->scalars : nullptr; da.st = c->dstatus;
