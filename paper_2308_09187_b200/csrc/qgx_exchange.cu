@@ -455,6 +455,18 @@ __device__ __forceinline__ SubBlockAt find_subblock(const DecodeArgs& a, int k, 
   return r;
 }
 
+// Copies one row of kept symbol words (kWords words, contiguous, 16-byte aligned) into shared memory without
+// waiting; one commit group per call.
+template <int kWords>
+__device__ __forceinline__ void stage_symbol_row(uint32_t* dst, const uint8_t* src, int lane) {
+#pragma unroll
+  for (int c = lane; c < kWords / 4; c += 32) {
+    const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + 4 * c);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src + 16 * (size_t)c) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
 // SYM: 0 plain, 1 also keeps the decoded symbols, 2 also compares with the symbols kept by the other exchange
 template <int G, int SYM>
 __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6)) k_exchange_decode(const __grid_constant__ DecodeArgs a,
@@ -462,6 +474,9 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
                                                                       const __grid_constant__ LevelTable lt) {
   extern __shared__ __align__(16) unsigned char s_raw[];
   __shared__ float s_lev[QGX_MAX_LEVELS];
+  // SYM == 2: the other exchange's symbol words of the warp's 32 sub-blocks, one worker ahead (asynchronous copies)
+  constexpr int kRowWords = G * 8;                      // 32 sub-blocks x G bytes
+  __shared__ __align__(16) uint32_t s_prev[SYM == 2 ? 2 * (kDecThreads / 32) * kRowWords : 4];
   const int lut_n = 2 << ct.maxlen;
   DecEntry* s_lut = reinterpret_cast<DecEntry*>(s_raw);
   {
@@ -498,8 +513,24 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
 #pragma unroll
     for (int i = 0; i < G; ++i) acc[i] = 0.0f;
     SubBlockAt nxt = find_subblock(a, 0, b, hdr_bits, s, count > 0, uniform, lane);
+    uint32_t* my_rows = s_prev + (SYM == 2 ? (tid >> 5) * 2 * kRowWords : 0);
+    if (SYM == 2) {
+      __syncwarp();                                       // the previous sub-block's rows are no longer read
+      stage_symbol_row<kRowWords>(my_rows, a.sym_prev + (gs >> 5) * (size_t)(32 * G), lane);
+    }
     for (int k = 0; k < a.K; ++k) {
       const SubBlockAt cur = nxt;
+      const uint32_t* prev_row = my_rows + (k & 1) * kRowWords + lane;
+      if (SYM == 2) {
+        __syncwarp();                                     // every lane is done with the row that is overwritten next
+        if (k + 1 < a.K)
+          stage_symbol_row<kRowWords>(my_rows + ((k + 1) & 1) * kRowWords,
+                                      a.sym_prev + (size_t)(k + 1) * a.sym_ld + (gs >> 5) * (size_t)(32 * G), lane);
+        else
+          asm volatile("cp.async.commit_group;" ::: "memory");     // keeps the group count uniform
+        asm volatile("cp.async.wait_group 1;" ::: "memory");      // worker k's row has landed
+        __syncwarp();
+      }
       if (k + 1 < a.K) nxt = find_subblock(a, k + 1, b, hdr_bits, s, count > 0, uniform, lane);
       bad = bad || !cur.ok;
       Window win;
@@ -512,7 +543,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
           if ((i & 1) == 0) {                              // two symbols use at most 26 bits
             if (win.avail <= 32) win.refill();
           }
-          if (SYM == 2 && (i & 3) == 0) prev4 = __ldcs(reinterpret_cast<const uint32_t*>(a.sym_prev + (size_t)k * a.sym_ld + sbase + (i >> 2) * 128));
+          if (SYM == 2 && (i & 3) == 0) prev4 = prev_row[(i >> 2) * 32];
           const DecEntry e = s_lut[win.lo & mask];
           const uint32_t L = e.len & 31u;
           flags |= e.len;
