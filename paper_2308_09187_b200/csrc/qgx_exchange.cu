@@ -358,8 +358,9 @@ struct Window {
   uint32_t lo, hi;
   uint32_t ahead;         // the word after the window, fetched one refill early
   int avail;
-  // p = address of the word that holds the first bit, w0..w2 = p[0..2], sh = first bit within w0
-  __device__ __forceinline__ void open(const uint32_t* p, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t sh) {
+  // p = address of the word that holds the first bit (shared or global memory), sh = first bit within it
+  __device__ __forceinline__ void open(const uint32_t* p, uint32_t sh) {
+    const uint32_t w0 = p[0], w1 = p[1], w2 = p[2];
     lo = __funnelshift_r(w0, w1, sh);
     hi = w1 >> sh;
     avail = 64 - (int)sh;                               // the window ends on a word boundary
@@ -397,7 +398,7 @@ __device__ __forceinline__ uint32_t header_sum_before_warp(const uint32_t* w, ui
 __device__ __forceinline__ bool locate_subblock(const uint32_t* stream, size_t cap_words, const uint32_t* bucket_bits,
                                                 const uint32_t* offsets, size_t kb, uint32_t hdr_bits, uint32_t s,
                                                 bool exists, bool uniform, int lane, const uint32_t** words, float* norm,
-                                                uint32_t* start, uint32_t* want) {
+                                                uint32_t* start, uint32_t* want, uint32_t* row_before, uint32_t* row_bits) {
   const uint32_t nbits = bucket_bits[kb];
   const uint32_t off = offsets[kb];
   const uint32_t* w = stream + off;
@@ -405,13 +406,18 @@ __device__ __forceinline__ bool locate_subblock(const uint32_t* stream, size_t c
   const bool ok = nbits >= hdr_bits && (size_t)off + ((nbits + 31) >> 5) <= cap_words;
   uint32_t st = 0, len = 0;
   float nm = 0.0f;
+  *row_before = 0;
+  *row_bits = 0;
   if (ok) {
     nm = __uint_as_float(w[0]);
     if (uniform) {
       const uint32_t bit = kNormBits + 16u * s;
       len = exists ? ((w[bit >> 5] >> (bit & 31u)) & 0xffffu) : 0u;
       const uint32_t incl = warp_incl_scan(len, lane);
-      st = header_sum_before_warp(w, s - (uint32_t)lane, lane) + incl - len;
+      const uint32_t before = header_sum_before_warp(w, s - (uint32_t)lane, lane);
+      st = before + incl - len;
+      *row_before = before;
+      *row_bits = __shfl_sync(0xffffffffu, incl, 31);
     } else if (exists) {
       for (uint32_t i = 0; i <= s; ++i) {
         const uint32_t bit = kNormBits + 16u * i;
@@ -431,32 +437,54 @@ __device__ __forceinline__ bool locate_subblock(const uint32_t* stream, size_t c
 // worker's sub-block once, front to back, so that every fetched sector is used up at once.  The next
 // worker's sub-block is located while the current one is decoded.
 struct SubBlockAt {
-  const uint32_t* p;      // word that holds the first bit
-  uint32_t w0, w1, w2;    // p[0..2]
-  uint32_t sh;            // first bit within w0
+  const uint32_t* p;      // word that holds the first bit: in the warp's staged row (shared memory) or in the stream
+  uint32_t sh;            // first bit within that word
   uint32_t want;          // bits of the sub-block
   float norm;
   float norm_prev;        // norm of the same bucket in the other exchange (when comparing)
   bool ok;
 };
 
+// Words that a thread may read past the first word of its sub-block: G symbols of at most 13 bits, the
+// partial first word and the two words fetched ahead.
+template <int G>
+struct DecodeReach { static constexpr int kWords = (G * 13) / 32 + 4; };
+
+// Locates sub-block s of bucket (k, b) and starts the asynchronous copy of the warp's row -- the stream words
+// of its 32 consecutive sub-blocks plus what a thread may read past them -- into `row` (shared memory, row_words
+// words).  A thread whose reads would leave the staged words reads the stream itself.  The copies belong to the
+// caller's next commit group.
+template <int G>
 __device__ __forceinline__ SubBlockAt find_subblock(const DecodeArgs& a, int k, size_t b, uint32_t hdr_bits, uint32_t s,
-                                                    bool exists, bool uniform, int lane) {
+                                                    bool exists, bool uniform, int lane, uint32_t* row, int row_words) {
   SubBlockAt r;
   const uint32_t* w;
-  uint32_t st;
+  uint32_t st, row_before, row_bits;
   r.ok = locate_subblock(a.stream + (size_t)k * a.cap_words, a.cap_words, a.bucket_bits, a.offsets, (size_t)k * a.nb + b,
-                         hdr_bits, s, exists, uniform, lane, &w, &r.norm, &st, &r.want);
+                         hdr_bits, s, exists, uniform, lane, &w, &r.norm, &st, &r.want, &row_before, &row_bits);
   if (!r.ok) { st = 0; r.want = 0; r.norm = 0.0f; }
   r.p = w + (st >> 5);
   r.sh = st & 31u;
-  r.w0 = r.p[0]; r.w1 = r.p[1]; r.w2 = r.p[2];
+  // bucket-level validity is the same for all lanes; the lengths are bounded, so the row is at most 2^19 bits
+  const bool stage = uniform && __all_sync(0xffffffffu, r.ok) && row_bits < (1u << 19);
+  if (stage) {
+    const size_t first = (size_t)(w - a.stream) + ((hdr_bits + row_before) >> 5);       // word index in the whole buffer
+    const size_t first_al = first & ~(size_t)3;                                          // 16-byte aligned
+    const size_t last = (size_t)(w - a.stream) + ((hdr_bits + row_before + row_bits + 31u) >> 5) + DecodeReach<G>::kWords;
+    const int nwords = (int)min((size_t)row_words, ((last - first_al) + 3) & ~(size_t)3);   // the buffer ends 64 words after the streams
+    for (int c = lane; c < nwords / 4; c += 32) {
+      const unsigned sa = (unsigned)__cvta_generic_to_shared(row + 4 * c);
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(a.stream + first_al + 4 * (size_t)c) : "memory");
+    }
+    const size_t mine = (size_t)(r.p - a.stream) - first_al;
+    if (mine + DecodeReach<G>::kWords <= (size_t)nwords) r.p = row + mine;
+  }
   r.norm_prev = a.norms_prev ? a.norms_prev[(size_t)k * a.nb + b] : 0.0f;
   return r;
 }
 
 // Copies one row of kept symbol words (kWords words, contiguous, 16-byte aligned) into shared memory without
-// waiting; one commit group per call.
+// waiting; the copies belong to the caller's next commit group.
 template <int kWords>
 __device__ __forceinline__ void stage_symbol_row(uint32_t* dst, const uint8_t* src, int lane) {
 #pragma unroll
@@ -464,8 +492,14 @@ __device__ __forceinline__ void stage_symbol_row(uint32_t* dst, const uint8_t* s
     const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + 4 * c);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src + 16 * (size_t)c) : "memory");
   }
-  asm volatile("cp.async.commit_group;" ::: "memory");
 }
+
+// shared memory of the decode kernel after its table: two stream rows and (SYM == 2) two symbol rows per warp
+template <int G, int SYM>
+struct DecodeSmem {
+  static constexpr int kStreamRow = 9 * G + 64;         // words, a multiple of 4
+  static constexpr size_t kBytes = sizeof(uint32_t) * 2 * (128 / 32) * (size_t)(kStreamRow + (SYM == 2 ? G * 8 : 0));
+};
 
 // SYM: 0 plain, 1 also keeps the decoded symbols, 2 also compares with the symbols kept by the other exchange
 template <int G, int SYM>
@@ -476,9 +510,13 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
   __shared__ float s_lev[QGX_MAX_LEVELS];
   // SYM == 2: the other exchange's symbol words of the warp's 32 sub-blocks, one worker ahead (asynchronous copies)
   constexpr int kRowWords = G * 8;                      // 32 sub-blocks x G bytes
-  __shared__ __align__(16) uint32_t s_prev[SYM == 2 ? 2 * (kDecThreads / 32) * kRowWords : 4];
+  // the stream words of the warp's 32 sub-blocks, one worker ahead (asynchronous copies): room for 8 bits per
+  // symbol and sign on average; longer rows are partly read from the stream itself
+  constexpr int kStreamRow = DecodeSmem<G, SYM>::kStreamRow;
   const int lut_n = 2 << ct.maxlen;
-  DecEntry* s_lut = reinterpret_cast<DecEntry*>(s_raw);
+  DecEntry* s_lut = reinterpret_cast<DecEntry*>(s_raw);                       // dynamic shared memory: table, stream rows, symbol rows
+  uint32_t* s_rows = reinterpret_cast<uint32_t*>(s_raw + sizeof(DecEntry) * (size_t)lut_n);
+  uint32_t* s_prev = s_rows + 2 * (kDecThreads / 32) * kStreamRow;
   {
     const uint2* src = reinterpret_cast<const uint2*>(a.lut);
     uint2* dst = reinterpret_cast<uint2*>(s_lut);
@@ -512,29 +550,28 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
     float acc[G];
 #pragma unroll
     for (int i = 0; i < G; ++i) acc[i] = 0.0f;
-    SubBlockAt nxt = find_subblock(a, 0, b, hdr_bits, s, count > 0, uniform, lane);
     uint32_t* my_rows = s_prev + (SYM == 2 ? (tid >> 5) * 2 * kRowWords : 0);
-    if (SYM == 2) {
-      __syncwarp();                                       // the previous sub-block's rows are no longer read
-      stage_symbol_row<kRowWords>(my_rows, a.sym_prev + (gs >> 5) * (size_t)(32 * G), lane);
-    }
+    uint32_t* my_stream = s_rows + (tid >> 5) * 2 * kStreamRow;
+    __syncwarp();                                         // the previous sub-block's rows are no longer read
+    SubBlockAt nxt = find_subblock<G>(a, 0, b, hdr_bits, s, count > 0, uniform, lane, my_stream, kStreamRow);
+    if (SYM == 2) stage_symbol_row<kRowWords>(my_rows, a.sym_prev + (gs >> 5) * (size_t)(32 * G), lane);
+    asm volatile("cp.async.commit_group;" ::: "memory");
     for (int k = 0; k < a.K; ++k) {
       const SubBlockAt cur = nxt;
       const uint32_t* prev_row = my_rows + (k & 1) * kRowWords + lane;
-      if (SYM == 2) {
-        __syncwarp();                                     // every lane is done with the row that is overwritten next
-        if (k + 1 < a.K)
+      __syncwarp();                                       // every lane is done with the rows that are overwritten next
+      if (k + 1 < a.K) {
+        nxt = find_subblock<G>(a, k + 1, b, hdr_bits, s, count > 0, uniform, lane, my_stream + ((k + 1) & 1) * kStreamRow, kStreamRow);
+        if (SYM == 2)
           stage_symbol_row<kRowWords>(my_rows + ((k + 1) & 1) * kRowWords,
                                       a.sym_prev + (size_t)(k + 1) * a.sym_ld + (gs >> 5) * (size_t)(32 * G), lane);
-        else
-          asm volatile("cp.async.commit_group;" ::: "memory");     // keeps the group count uniform
-        asm volatile("cp.async.wait_group 1;" ::: "memory");      // worker k's row has landed
-        __syncwarp();
       }
-      if (k + 1 < a.K) nxt = find_subblock(a, k + 1, b, hdr_bits, s, count > 0, uniform, lane);
+      asm volatile("cp.async.commit_group;" ::: "memory");       // one group per worker, empty after the last
+      asm volatile("cp.async.wait_group 1;" ::: "memory");       // worker k's rows have landed
+      __syncwarp();
       bad = bad || !cur.ok;
       Window win;
-      win.open(cur.p, cur.w0, cur.w1, cur.w2, cur.sh);
+      win.open(cur.p, cur.sh);
       uint32_t flags = 0, used = 0;
       if (count == G) {
         uint32_t pack = 0, prev4 = 0;
@@ -766,7 +803,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
 template <int G, int SYM>
 static qgx_status launch_decode_gs(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt) {
   const size_t total_sub = da.nb * ((size_t)da.bucket / G);
-  const size_t lut_bytes = sizeof(DecEntry) * ((size_t)2 << ct.maxlen);
+  const size_t lut_bytes = sizeof(DecEntry) * ((size_t)2 << ct.maxlen) + DecodeSmem<G, SYM>::kBytes;   // table, then the rows
   const size_t want = (total_sub + kDecThreads - 1) / kDecThreads;
   int per_sm = 1;
   {
