@@ -35,6 +35,9 @@ METRIC = "Q-GenX quantize->code->decode->average GB/s (% of HBM peak); EG iterat
 WORKLOAD = "c5-scale: K=32, d=2^26, mixture noise, diagonal operator, bucket 16384, 17 adaptive levels"
 
 
+# measured DRAM traffic of k_exchange_encode per coordinate (ncu, current kernel); None once the kernel has changed
+ENCODE_DRAM_BYTES_PER_COORDINATE = 4.891
+
 def exchange_bytes(K, d, nb, stream_words):
     """Algorithmic bytes of one exchange: read V, write + read the streams and their length words, write the mean."""
     S = 4 * int(stream_words) + 4 * K * nb
@@ -197,9 +200,15 @@ def run_ours(args):
     enc_bytes = 4 * K * d + 4 * d + 4 * (sum(words) / 2.0) + 12 * K * nb
     enc_ms = ms_enc / max(n_enc, 1)
     achieved = enc_bytes / (enc_ms * 1e-3) / 1e9 if n_enc else None
+    # DRAM bytes per launch of that kernel: counted by ncu on a smaller case of the same kernel (see
+    # profiles/exchange_kernels_K8_d16M.txt: 656.5 MB read + written for K * d = 2^27 coordinates) and scaled by
+    # the coordinates of a launch, which the traffic is proportional to.  Set to None when the kernel changes.
+    traffic = args.traffic_bytes
+    if traffic is None and ENCODE_DRAM_BYTES_PER_COORDINATE is not None:
+        traffic = ENCODE_DRAM_BYTES_PER_COORDINATE * K * d
     roofline = {"bound": "hbm", "kernel": "k_exchange_encode", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None, "peak_kind": "of " + peak_kind,
-                "traffic": args.traffic_bytes, "ms_per_launch": enc_ms,
+                "traffic": traffic, "ms_per_launch": enc_ms,
                 "kernels_ms_per_step": {"encode": ms_enc / args.steps, "decode": ms_dec / args.steps,
                                         "histogram": ms_his / args.steps, "operator": ms_op / args.steps,
                                         "finish": ms_fin / args.steps}}
