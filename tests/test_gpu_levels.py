@@ -64,3 +64,40 @@ def test_update_levels_matches_oracle_refit(q):
         lev2 = np.array(cfg.level_list(), dtype=np.float32)
         lev_ref2, _ = o.refit(vh, bucket, 1024, lev_ref, cbo, False, code_type)
         assert np.max(np.abs(lev2 - lev_ref2)) < 5e-5
+
+
+def test_linf_normalisation_refit_and_exchange(q):
+    """The max-norm variant end to end: histogram and level fit on u = |v| / max|v|, then a fused exchange
+    with the fitted table.  Max norms are exact, so streams and mean are bit-identical to the oracle's."""
+    qgx, ctx = q
+    K, d, bucket, nlev, sub = 4, 3 * 4096 + 500, 4096, 17, 64
+    v = gen.student_t3((K, d), seed=77, device="cuda") * 0.01
+    vh = v.cpu().numpy()
+    cfg = qgx.make_quant_cfg(np.linspace(0, 1, nlev), bucket, qgx.qgx_build_codebook_fixed(nlev, sub), 9,
+                             norm_type=qgx.QGX_NORM_LINF, code_type=qgx.QGX_CODE_HUFFMAN, nbins=1024)
+    hist = qgx.qgx_update_levels(ctx, v, cfg, qgx.QGX_REFIT_FIRST)
+    cbo = o.codebook_fixed(nlev, sub)
+    lev_ref, hist_ref = o.refit(vh, bucket, 1024, np.linspace(0, 1, nlev, dtype=np.float32), cbo, True, o.CODE_HUFFMAN,
+                                norm_type=o.LINF)
+    assert np.allclose(hist, hist_ref, rtol=1e-6, atol=1e-9 * hist_ref.sum())
+    lev = np.array(cfg.level_list(), dtype=np.float32)
+    assert o.check_levels(lev) == o.OK
+    assert np.max(np.abs(lev - lev_ref)) < 5e-5
+    # the max norm spreads u over [0, 1]: the fitted table uses the upper half of the range too
+    assert lev[-2] > 0.3
+    # exchange with the library's table and code on both sides
+    cbo = o.codebook_from(cfg.cb.lengths(), cfg.cb.codes(), subblock=sub)
+    mean, total = qgx.qgx_exchange(ctx, v, cfg, 12, slot=0)
+    qgx.qgx_sync_status(ctx)
+    m_or, t_or = o.exchange(vh, bucket, lev, cbo, 9, 12, norm_type=o.LINF)
+    assert np.array_equal(total.cpu().numpy().astype(np.uint64), t_or)
+    assert np.array_equal(mean.cpu().numpy(), m_or)
+    nb = o.nbuckets(d, bucket)
+    stream, bbits, _ = qgx.exchange_stream_tensors(ctx, 0, K, nb)
+    n_ref = o.bucket_norms(vh, bucket, o.LINF)
+    st_ref, bb_ref, _ = o.encode(n_ref, o.quantize(vh, bucket, lev, n_ref, 9, 12), bucket, cbo)
+    assert np.array_equal(bbits.cpu().numpy().view(np.uint32), bb_ref)
+    used = ((bb_ref.astype(np.int64) + 31) // 32).sum(axis=1)
+    sh = stream.cpu().numpy().view(np.uint32)
+    for k in range(K):
+        assert np.array_equal(sh[k, :used[k]], st_ref[k, :used[k]])
