@@ -20,6 +20,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <string>
 #include <vector>
 #include <algorithm>
 #include <limits>
@@ -338,6 +339,37 @@ int qgxo_codebook_fixed(int nlev, int subblock, qgxo_codebook* cb) {
   cb->nlev = nlev; cb->subblock = subblock;
   for (int j = 0; j < nlev; ++j) cb->len[j] = (uint8_t)L;
   canonical_codes(cb);
+  return OK;
+}
+
+// Elias' recursive ("omega") code of the positive integer n, as a string of '0'/'1' in sending order
+// (Elias 1975; the universal integer code that App. J names for an unknown symbol distribution):
+// start from the single bit 0; while n > 1, put the binary expansion of n in front and replace n by
+// the number of bits of that expansion minus one.
+static std::string elias_omega(unsigned n) {
+  std::string out = "0";
+  while (n > 1) {
+    std::string bin;
+    for (unsigned m = n; m > 0; m >>= 1) bin.insert(bin.begin(), (m & 1u) ? '1' : '0');
+    out = bin + out;
+    n = (unsigned)bin.size() - 1;
+  }
+  return out;
+}
+
+// level index j is sent as the code of the integer j + 1: smaller levels get shorter codewords
+int qgxo_codebook_elias(int nlev, int subblock, qgxo_codebook* cb) {
+  if (nlev < 2 || nlev > kMaxLevels) return INVALID_ARG;
+  std::memset(cb, 0, sizeof(*cb));
+  cb->nlev = nlev; cb->subblock = subblock;
+  for (int j = 0; j < nlev; ++j) {
+    const std::string w = elias_omega((unsigned)j + 1u);
+    uint32_t code = 0;
+    for (char c : w) code = (code << 1) | (c == '1' ? 1u : 0u);     // first sent bit = most significant
+    cb->len[j] = (uint8_t)w.size();
+    cb->code[j] = code;
+    cb->maxlen = std::max<int>(cb->maxlen, (int)w.size());
+  }
   return OK;
 }
 
@@ -782,7 +814,7 @@ int qgxo_exchange_full(const float* V, int K, uint64_t d, int bucket, int norm_t
 // the norm^2-weighted histogram of all buckets of the K current dual vectors; the levels are
 // refitted (from quantiles on the first fit, from the current levels afterwards) and, for
 // code_type 1, the Huffman code is rebuilt from the symbol weights; code_type 0 keeps the
-// fixed-length code.
+// fixed-length code, code_type 2 Elias' recursive code (neither depends on the weights).
 int qgxo_refit(const float* V, int K, uint64_t d, int bucket, int norm_type, int nbins, int first_fit,
                int code_type, float* lev, int nlev, qgxo_codebook* cb, double* hist_out) {
   std::vector<double> hist(nbins), p(nlev);
@@ -795,6 +827,8 @@ int qgxo_refit(const float* V, int K, uint64_t d, int bucket, int norm_type, int
     st = qgxo_symbol_pmf(hist.data(), nbins, lev, nlev, p.data());
     if (st) return st;
     st = qgxo_codebook_huffman(p.data(), nlev, sub, cb);
+  } else if (code_type == 2) {
+    st = qgxo_codebook_elias(nlev, sub, cb);
   } else {
     st = qgxo_codebook_fixed(nlev, sub, cb);
   }

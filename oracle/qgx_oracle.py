@@ -11,7 +11,7 @@ from . import build as _build
 
 OK, INVALID_ARG, BAD_LEVELS, CAPACITY, CORRUPT, NONFINITE = range(6)
 L2, LINF = 0, 1
-CODE_FIXED, CODE_HUFFMAN = 0, 1
+CODE_FIXED, CODE_HUFFMAN, CODE_ELIAS = 0, 1, 2
 OP_DENSE_AFFINE, OP_BILINEAR, OP_DIAGONAL = 0, 1, 2
 
 
@@ -187,6 +187,12 @@ def average(norms, sym, bucket, levels):
 def codebook_fixed(nlev, subblock=0):
     cb = Codebook()
     _chk(lib().qgxo_codebook_fixed(nlev, subblock, C.byref(cb)), "codebook_fixed")
+    return cb
+
+
+def codebook_elias(nlev, subblock=0):
+    cb = Codebook()
+    _chk(lib().qgxo_codebook_elias(nlev, subblock, C.byref(cb)), "codebook_elias")
     return cb
 
 

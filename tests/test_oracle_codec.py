@@ -51,7 +51,8 @@ def test_round_trip_every_alphabet_size(nlev):
     K, d, bucket = 2, 700, 256                      # buckets of 256, 256, 188
     p = rng.dirichlet(np.ones(nlev) * 0.3)
     for cb in (o.codebook_fixed(nlev, 0), o.codebook_fixed(nlev, 64), o.codebook_huffman(p, 0),
-               o.codebook_huffman(p, 128), o.codebook_huffman(p, 100)):
+               o.codebook_huffman(p, 128), o.codebook_huffman(p, 100), o.codebook_elias(nlev, 0),
+               o.codebook_elias(nlev, 64)):
         sym = _random_symbols(rng, K, d, nlev, p)
         sym[0, :256] = 0                                 # an all-zero bucket
         sym[1, 256:512] = (nlev - 1) | 0x80              # an all-top-level, all-negative bucket
@@ -132,6 +133,33 @@ def test_huffman_is_optimal_and_within_one_bit_of_entropy():
                 H = -np.sum(p[p > 0] * np.log2(p[p > 0]))
                 el = float(np.dot(p, cb.lengths()))
                 assert H - 1e-9 <= el <= H + 1 + 1e-9        # Theorem (Huffman), App. J
+
+
+def test_elias_recursive_code_table_and_properties():
+    """The code Psi for an unknown symbol distribution (App. J): level j is sent as Elias' recursive code of
+    j + 1.  Pinned to the published table of the code, to its length recursion and to the prefix property."""
+    cb = o.codebook_elias(32, 0)
+    words = [format(c, "0%db" % L) for c, L in zip(cb.codes(), cb.lengths())]
+    for n, w in read_golden("elias_omega.txt"):
+        assert words[int(n) - 1] == w
+    # length recursion: len(1) = 1, len(n) = len(floor(log2 n)) + floor(log2 n) + 1
+    def length(n):
+        return 1 if n == 1 else length(n.bit_length() - 1) + n.bit_length()
+    assert [len(w) for w in words] == [length(n) for n in range(1, 33)]
+    assert cb.maxlen == 12 and max(len(w) for w in words) == 12
+    # smaller values never get longer codewords; no codeword is a prefix of another; Kraft sum below one
+    assert all(len(a) <= len(b) for a, b in zip(words, words[1:]))
+    assert not any(a != b and b.startswith(a) for a in words for b in words)
+    assert sum(2.0 ** -len(w) for w in words) < 1.0
+    # every codeword ends the recursion with a 0 and every group before it starts with a 1
+    assert all(w.endswith("0") for w in words) and all(w[0] == "1" for w in words[1:])
+    # a smaller alphabet takes the first codewords
+    cb9 = o.codebook_elias(9, 16)
+    assert cb9.codes() == cb.codes()[:9] and cb9.lengths() == cb.lengths()[:9] and cb9.subblock == 16 and cb9.maxlen == 7
+    # on a distribution that decays with the level it beats the fixed-length code, as the paper says it is meant to
+    p = 0.5 ** np.arange(1, 18)
+    p /= p.sum()
+    assert np.dot(p, o.codebook_elias(17, 0).lengths()) < np.dot(p, o.codebook_fixed(17, 0).lengths())
 
 
 def test_codeword_length_cap():
