@@ -44,7 +44,7 @@ typedef enum {
 } qgx_status;
 
 enum { QGX_NORM_L2 = 0, QGX_NORM_LINF = 1 };
-enum { QGX_CODE_FIXED = 0, QGX_CODE_HUFFMAN = 1 };
+enum { QGX_CODE_FIXED = 0, QGX_CODE_HUFFMAN = 1, QGX_CODE_ELIAS = 2 };
 enum { QGX_OP_DENSE_AFFINE = 0, QGX_OP_BILINEAR = 1, QGX_OP_DIAGONAL = 2 };
 enum { QGX_REFIT_NONE = 0, QGX_REFIT_CONTINUE = 1, QGX_REFIT_FIRST = 2 };
 /* flag of qgx_quantize: `norms` is an input (the caller's norms are used as they are) */
@@ -71,7 +71,7 @@ typedef struct {
   int32_t nlev;
   int32_t bucket;           /* multiple of 4, <= QGX_MAX_BUCKET */
   int32_t norm_type;        /* QGX_NORM_L2 | QGX_NORM_LINF */
-  int32_t code_type;        /* what a refit rebuilds: QGX_CODE_FIXED | QGX_CODE_HUFFMAN */
+  int32_t code_type;        /* what a refit rebuilds: QGX_CODE_FIXED | QGX_CODE_HUFFMAN | QGX_CODE_ELIAS */
   int32_t nbins;            /* histogram bins of the level refit (Sec. 3.3) */
   int32_t pad;
   uint64_t seed;            /* key of the counter-based generator */
@@ -143,6 +143,12 @@ qgx_status qgx_build_codebook_fixed(int nlev, int subblock, qgx_codebook *cb /*[
  * (length, index); if the longest codeword would exceed QGX_MAX_CODE_LEN the weights are
  * flattened by adding 2^(m-16), m = 0, 1, ..., until it fits. */
 qgx_status qgx_build_codebook_huffman(const double *p, int nlev, int subblock, qgx_codebook *cb);
+/* Elias' recursive code (App. J: the choice when the distribution of the levels is unknown but small
+ * levels are known to be frequent): level j is sent as the codeword of the integer j + 1 -- the bit 0
+ * preceded by groups, the last group the binary form of the integer, each earlier group the binary
+ * form of the following group's bit count minus one.  At most 12 bits for 32 levels; independent of
+ * any weights.  cb [host] out. */
+qgx_status qgx_build_codebook_elias(int nlev, int subblock, qgx_codebook *cb);
 /* Level fit of Sec. 3.3 on a histogram hist[nbins] [host] of normalized magnitudes, read as a
  * piecewise-uniform density: coordinate descent on the (QAda) objective, each interior level
  * moved to the root of the objective's derivative with its neighbours fixed; at most 32 sweeps.

@@ -16,7 +16,7 @@ QGX_OK = 0
 QGX_ERR_INVALID_ARG, QGX_ERR_BAD_LEVELS, QGX_ERR_CAPACITY, QGX_ERR_CORRUPT = 1, 2, 3, 4
 QGX_ERR_NONFINITE, QGX_ERR_TIMEOUT, QGX_ERR_CUDA, QGX_ERR_TOO_LARGE = 5, 6, 7, 8
 QGX_NORM_L2, QGX_NORM_LINF = 0, 1
-QGX_CODE_FIXED, QGX_CODE_HUFFMAN = 0, 1
+QGX_CODE_FIXED, QGX_CODE_HUFFMAN, QGX_CODE_ELIAS = 0, 1, 2
 QGX_OP_DENSE_AFFINE, QGX_OP_BILINEAR, QGX_OP_DIAGONAL = 0, 1, 2
 QGX_REFIT_NONE, QGX_REFIT_CONTINUE, QGX_REFIT_FIRST = 0, 1, 2
 QGX_NORMS_SUPPLIED = 1
@@ -24,7 +24,7 @@ QGX_MAX_LEVELS, QGX_MAX_CODE_LEN, QGX_MAX_BUCKET = 32, 12, 16384
 
 EXPORTS = [
     "qgx_create", "qgx_destroy", "qgx_sync_status", "qgx_status_str", "qgx_launch_count",
-    "qgx_check_levels", "qgx_stream_capacity_words", "qgx_build_codebook_fixed",
+    "qgx_check_levels", "qgx_stream_capacity_words", "qgx_build_codebook_fixed", "qgx_build_codebook_elias",
     "qgx_build_codebook_huffman", "qgx_fit_levels", "qgx_symbol_pmf",
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
@@ -178,6 +178,12 @@ def qgx_check_levels(levels):
 
 def qgx_stream_capacity_words(d, bucket, subblock, maxlen):
     return int(lib().qgx_stream_capacity_words(d, bucket, subblock, maxlen))
+
+
+def qgx_build_codebook_elias(nlev, subblock=0):
+    cb = qgx_codebook()
+    _chk(lib().qgx_build_codebook_elias(nlev, subblock, C.byref(cb)), "qgx_build_codebook_elias")
+    return cb
 
 
 def qgx_build_codebook_fixed(nlev, subblock=0):

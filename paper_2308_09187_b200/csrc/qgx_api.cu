@@ -274,6 +274,32 @@ qgx_status qgx_build_codebook_fixed(int nlev, int subblock, qgx_codebook* cb) {
   return QGX_OK;
 }
 
+// Elias' recursive code of j + 1 for level j.  The codeword is the closing 0 preceded by groups; walking
+// backwards from the integer itself, each group is the binary form of the current value and the next value is
+// that group's bit count minus one.  Groups are placed from the low end of the word upwards.
+qgx_status qgx_build_codebook_elias(int nlev, int subblock, qgx_codebook* cb) {
+  if (cb == nullptr || nlev < 2 || nlev > QGX_MAX_LEVELS) return QGX_ERR_INVALID_ARG;
+  std::memset(cb, 0, sizeof(*cb));
+  cb->nlev = nlev;
+  cb->subblock = subblock;
+  for (int j = 0; j < nlev; ++j) {
+    uint32_t word = 0;                    // the closing 0
+    int used = 1;
+    for (uint32_t value = (uint32_t)j + 1u; value > 1u;) {
+      int width = 0;
+      while ((value >> width) != 0u) ++width;
+      word |= value << used;
+      used += width;
+      value = (uint32_t)width - 1u;
+    }
+    if (used > QGX_MAX_CODE_LEN) return QGX_ERR_INVALID_ARG;
+    cb->len[j] = (uint8_t)used;
+    cb->code[j] = word;
+    cb->maxlen = std::max<int>(cb->maxlen, used);
+  }
+  return QGX_OK;
+}
+
 // Huffman lengths: a forest kept as parent links; each round joins the two lightest roots
 // (among equal weights the root that has existed longest first) and every leaf below gains a bit.
 static int huffman_depths(const double* w, int n, int* depth) {

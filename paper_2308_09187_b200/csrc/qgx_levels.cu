@@ -95,6 +95,8 @@ qgx_status refit_from_source(qgx_ctx* c, DualSource src, int K, size_t d, qgx_qu
     rc = qgx_symbol_pmf(h.data(), cfg->nbins, cfg->levels, cfg->nlev, p);
     if (rc != QGX_OK) return rc;
     rc = qgx_build_codebook_huffman(p, cfg->nlev, sub, &cfg->cb);
+  } else if (cfg->code_type == QGX_CODE_ELIAS) {
+    rc = qgx_build_codebook_elias(cfg->nlev, sub, &cfg->cb);
   } else {
     rc = qgx_build_codebook_fixed(cfg->nlev, sub, &cfg->cb);
   }

@@ -153,3 +153,48 @@ def test_layerwise_segments_c3_shape(q):
         at += n
     assert np.array_equal(total.cpu().numpy().astype(np.uint64), bits_ref) or \
         np.max(np.abs(total.cpu().numpy().astype(np.int64) - bits_ref.astype(np.int64))) <= 16
+
+
+@pytest.mark.parametrize("K,d,bucket,nlev,sub", [(3, 2 * 4096 + 777, 4096, 17, 64), (2, 20000, 2048, 32, 128),
+                                                   (4, 3000, 512, 9, 32)])
+def test_elias_recursive_code(q, K, d, bucket, nlev, sub):
+    """The second prefix code of App. J through the same kernels: separate calls, fused exchange and a refit that
+    keeps this code, bit for bit against the oracle."""
+    qgx, ctx = q
+    rng = np.random.default_rng(nlev)
+    v = gen.gaussian_mixture((K, d), seed=3 * d, device="cuda")
+    vh = v.cpu().numpy()
+    lev = _levels(rng, nlev, top=0.4)
+    cb = qgx.qgx_build_codebook_elias(nlev, sub)
+    cbo = o.codebook_elias(nlev, sub)
+    assert cb.codes() == cbo.codes() and cb.lengths() == cbo.lengths()
+    seed, xid = 31, 5
+    norms, sym = qgx.qgx_quantize(ctx, v, bucket, lev, qgx.QGX_NORM_L2, seed, xid)
+    qgx.qgx_sync_status(ctx)
+    n_gpu = norms.cpu().numpy()
+    s_ref = o.quantize(vh, bucket, lev, n_gpu, seed, xid)
+    assert np.array_equal(sym.cpu().numpy(), s_ref)
+    stream, bbits, total = qgx.qgx_encode(ctx, norms, sym, bucket, cb)
+    qgx.qgx_sync_status(ctx)
+    st_ref, bb_ref, tot_ref = o.encode(n_gpu, s_ref, bucket, cbo)
+    assert np.array_equal(bbits.cpu().numpy().view(np.uint32), bb_ref)
+    assert np.array_equal(stream.cpu().numpy().view(np.uint32), st_ref)
+    n2, s2 = qgx.qgx_decode(ctx, stream, bbits, d, bucket, cb)
+    qgx.qgx_sync_status(ctx)
+    assert np.array_equal(s2.cpu().numpy(), s_ref)
+    # fused
+    cfg = qgx.make_quant_cfg(lev, bucket, cb, seed, code_type=qgx.QGX_CODE_ELIAS)
+    mean, tot = qgx.qgx_exchange(ctx, v, cfg, xid, slot=1)
+    qgx.qgx_sync_status(ctx)
+    assert np.array_equal(tot.cpu().numpy().astype(np.uint64), tot_ref)
+    assert np.array_equal(mean.cpu().numpy(), o.average(n_gpu, s_ref, bucket, lev))
+    fs, fb, _ = qgx.exchange_stream_tensors(ctx, 1, K, o.nbuckets(d, bucket))
+    used = _used_words(bb_ref)
+    fsh = fs.cpu().numpy().view(np.uint32)
+    for k in range(K):
+        assert np.array_equal(fsh[k, :used[k]], st_ref[k, :used[k]])
+    # a refit moves the levels and leaves this code in place
+    qgx.qgx_update_levels(ctx, v, cfg, qgx.QGX_REFIT_FIRST)
+    lev_ref, _ = o.refit(vh, bucket, 1024, lev.copy(), cbo, True, o.CODE_ELIAS)
+    assert np.max(np.abs(np.array(cfg.level_list(), dtype=np.float32) - lev_ref)) < 5e-5
+    assert cfg.cb.codes() == cbo.codes() and cfg.cb.lengths() == cbo.lengths() and cfg.cb.subblock == sub

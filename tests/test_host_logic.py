@@ -56,6 +56,8 @@ def test_codebooks_match_oracle(qgx):
     for nlev in range(2, 33):
         a, b = qgx.qgx_build_codebook_fixed(nlev, 64), o.codebook_fixed(nlev, 64)
         assert a.lengths() == b.lengths() and a.codes() == b.codes() and a.maxlen == b.maxlen
+        a, b = qgx.qgx_build_codebook_elias(nlev, 32), o.codebook_elias(nlev, 32)
+        assert a.lengths() == b.lengths() and a.codes() == b.codes() and a.maxlen == b.maxlen and a.subblock == 32
         for _ in range(5):
             p = rng.dirichlet(np.ones(nlev) * rng.uniform(0.05, 2.0))
             a, b = qgx.qgx_build_codebook_huffman(list(p), 0), o.codebook_huffman(p, 0)
