@@ -887,4 +887,60 @@ int qgxo_eg_step(qgxo_eg_state* st, const qgxo_operator* op, const float* noise_
   return OK;
 }
 
+// The two other members of the family named in Sec. 3.1, one oracle call and one exchange per iteration.
+// method 1, quantized dual averaging (Vhat_{k,t} = 0, hence X_{t+1/2} = X_t):
+//   g_{k,t} = Q(A(X_t) + U_{k,t});  Y_{t+1} = Y_t - mean_k g_{k,t};  sum_sq += sum_k ||0 - g_{k,t}||^2
+// method 2, quantized optimistic dual averaging (Vhat_{k,t} = g_{k,t-1/2}, the vectors of the previous iteration,
+// taken as zero in the first iteration):
+//   X_{t+1/2} = X_t - gamma_t * mean_k g_{k,t-1/2};  g_{k,t+1/2} = Q(A(X_{t+1/2}) + U_{k,t+1/2});
+//   Y_{t+1} = Y_t - mean_k g_{k,t+1/2};  sum_sq += sum_k ||g_{k,t-1/2} - g_{k,t+1/2}||^2
+// both: gamma_{t+1} = K / sqrt(1 + sum_sq), X_{t+1} = anchor + gamma_{t+1} Y_{t+1}, Xbar += (X_{t+1/2} - Xbar) / t.
+// A refit (t in U) uses the iteration's only dual vectors.  The exchange id is 2t + 1 (the draw of the second
+// exchange of Algorithm 1).  g_prev [K][d] and mean_prev [d] carry g_{k,t-1/2} and its mean from call to call
+// (method 2; zero before the first call) and are overwritten.
+int qgxo_family_step(qgxo_eg_state* st, int method, const qgxo_operator* op, const float* noise,
+                     int bucket, int norm_type, float* lev, int nlev, qgxo_codebook* cb,
+                     uint64_t seed, int quantizer_off, int refit, int code_type, int nbins,
+                     float* g_prev, float* mean_prev, uint64_t* bits_out) {
+  if (method != 1 && method != 2) return INVALID_ARG;
+  if (method == 2 && (!g_prev || !mean_prev)) return INVALID_ARG;
+  const uint64_t d = st->d; const int K = st->K;
+  std::vector<float> a(d), V((uint64_t)K * d), g((uint64_t)K * d), mean(d);
+  std::vector<uint64_t> tb(K);
+  for (uint64_t i = 0; i < d; ++i) {
+    if (method == 2) { const float step = st->gamma * mean_prev[i]; st->Xhalf[i] = st->X[i] - step; }
+    else st->Xhalf[i] = st->X[i];
+  }
+  int rc = qgxo_apply_operator(op, st->Xhalf, a.data());
+  if (rc) return rc;
+  qgxo_form_dual_vectors(a.data(), noise, K, d, V.data());
+  if (refit && !quantizer_off) {
+    rc = qgxo_refit(V.data(), K, d, bucket, norm_type, nbins, refit == 2, code_type, lev, nlev, cb, nullptr);
+    if (rc) return rc;
+  }
+  rc = qgxo_exchange_full(V.data(), K, d, bucket, norm_type, lev, nlev, cb, seed, 2u * (uint32_t)st->t + 1u,
+                          quantizer_off, g.data(), mean.data(), tb.data());
+  if (rc) return rc;
+  for (uint64_t i = 0; i < d; ++i) st->Y[i] = st->Y[i] - mean[i];
+  double s = 0.0;
+  for (int k = 0; k < K; ++k)
+    for (uint64_t i = 0; i < d; ++i) {
+      const float before = method == 2 ? g_prev[(uint64_t)k * d + i] : 0.0f;
+      const float diff = before - g[(uint64_t)k * d + i];
+      s += (double)diff * (double)diff;
+    }
+  st->sum_sq += s;
+  st->gamma = (float)((double)K / std::sqrt(1.0 + st->sum_sq));
+  for (uint64_t i = 0; i < d; ++i) { const float gy = st->gamma * st->Y[i]; st->X[i] = st->anchor[i] + gy; }
+  const float tf = (float)st->t;
+  for (uint64_t i = 0; i < d; ++i) { const float diff = st->Xhalf[i] - st->Xbar[i]; st->Xbar[i] = st->Xbar[i] + diff / tf; }
+  st->t += 1;
+  if (method == 2) {
+    for (uint64_t i = 0; i < (uint64_t)K * d; ++i) g_prev[i] = g[i];
+    for (uint64_t i = 0; i < d; ++i) mean_prev[i] = mean[i];
+  }
+  if (bits_out) { uint64_t b = 0; for (int k = 0; k < K; ++k) b += tb[k]; *bits_out = b; }
+  return OK;
+}
+
 }  // extern "C"

@@ -378,6 +378,25 @@ def eg_step(state, op, noise_t, noise_half, bucket, levels, cb, seed, norm_type=
     return bits.value
 
 
+METHOD_DE, METHOD_DA, METHOD_OPTDA = 0, 1, 2
+
+
+def family_step(state, method, op, noise, bucket, levels, cb, seed, g_prev=None, mean_prev=None, norm_type=L2,
+                quantizer_off=False, refit=0, code_type=CODE_FIXED, nbins=1024):
+    """One iteration of quantized dual averaging (METHOD_DA) or optimistic dual averaging (METHOD_OPTDA);
+    g_prev [K, d] and mean_prev [d] (float32, OptDA) are updated in place. Returns bits sent."""
+    nz = _f32(noise) if noise is not None else None
+    assert levels.dtype == np.float32 and levels.flags.c_contiguous
+    for arr in (g_prev, mean_prev):
+        assert arr is None or (arr.dtype == np.float32 and arr.flags.c_contiguous)
+    bits = C.c_uint64(0)
+    _chk(lib().qgxo_family_step(C.byref(state.c), int(method), C.byref(op.c), _p(nz), bucket, norm_type,
+                                _p(levels), len(levels), C.byref(cb), C.c_uint64(seed), int(quantizer_off),
+                                int(refit), int(code_type), int(nbins), _p(g_prev), _p(mean_prev), C.byref(bits)),
+         "family_step")
+    return bits.value
+
+
 def exchange(v, bucket, levels, cb, seed, xid, norm_type=L2, return_vhat=False):
     """quantize -> encode -> decode -> average of v[K, d]; returns (mean, total_bits[K]) (+ vhat)."""
     v = _f32(v)

@@ -133,3 +133,121 @@ def test_exchange_matches_its_parts():
     assert np.array_equal(total, tb)
     V = o.form_dual_vectors(v[0], v, 3)
     assert np.array_equal(V, v[0][None, :] + v)
+
+
+# ---- the other two members of the family (Sec. 3.1: quantized dual averaging, optimistic dual averaging) ----
+
+def _tiny(method):
+    op = o.Op(o.OP_BILINEAR, np.array([[1.0]], dtype=np.float32))           # V(x, y) = (y, -x)
+    st = o.EgState(np.array([1.0, 0.0], dtype=np.float32), K=1)
+    lev = np.array([0.0, 1.0], dtype=np.float32)
+    gp, mp = np.zeros((1, 2), np.float32), np.zeros(2, np.float32)
+    step = lambda: o.family_step(st, method, op, None, 2, lev, o.codebook_fixed(2), 0, gp, mp, quantizer_off=True)
+    return st, step, gp, mp
+
+
+def test_dual_averaging_by_hand():
+    """Eq. (Quantized DA) on V(x, y) = (y, -x) from z1 = (1, 0), K = 1, no noise, quantizer bypassed:
+      g_1 = (0, -1); Y_2 = (0, 1); sum = ||g_1||^2 = 1; gamma_2 = 1/sqrt 2; z_2 = (1, 1/sqrt 2);
+      g_2 = (1/sqrt 2, -1); Y_3 = (-1/sqrt 2, 2); sum = 2.5; gamma_3 = 1/sqrt 3.5; z_3 = z_1 + gamma_3 Y_3."""
+    st, step, _, _ = _tiny(o.METHOD_DA)
+    r = 1.0 / math.sqrt(2.0)
+    step()
+    assert st.Xhalf.tolist() == [1.0, 0.0] and st.Y.tolist() == [0.0, 1.0]       # X_{t+1/2} = X_t
+    assert st.sum_sq == 1.0 and abs(st.gamma - r) < 1e-7 and st.t == 2
+    assert np.allclose(st.X, [1.0, r], atol=1e-7) and st.Xbar.tolist() == [1.0, 0.0]
+    step()
+    g3 = 1.0 / math.sqrt(3.5)
+    assert np.allclose(st.Y, [-r, 2.0], atol=1e-6) and abs(st.sum_sq - 2.5) < 1e-6 and abs(st.gamma - g3) < 1e-6
+    assert np.allclose(st.X, [1.0 - g3 * r, 2.0 * g3], atol=1e-6)
+    assert np.allclose(st.Xbar, [1.0, r / 2], atol=1e-6)
+
+
+def test_optimistic_dual_averaging_by_hand():
+    """Eq. (Quantized OptDA), same problem; the first iteration has no earlier feedback (taken as zero):
+      z_{3/2} = z_1; g_{3/2} = (0, -1); Y_2 = (0, 1); sum = 1; gamma_2 = 1/sqrt 2; z_2 = (1, 1/sqrt 2);
+      z_{5/2} = z_2 - gamma_2 g_{3/2} = (1, sqrt 2); g_{5/2} = (sqrt 2, -1); Y_3 = (-sqrt 2, 2);
+      sum = 1 + ||g_{3/2} - g_{5/2}||^2 = 3; gamma_3 = 1/2; z_3 = (1 - sqrt 2 / 2, 1)."""
+    st, step, gp, mp = _tiny(o.METHOD_OPTDA)
+    r, s2 = 1.0 / math.sqrt(2.0), math.sqrt(2.0)
+    step()
+    assert st.Xhalf.tolist() == [1.0, 0.0] and st.Y.tolist() == [0.0, 1.0] and st.sum_sq == 1.0
+    assert gp.tolist() == [[0.0, -1.0]] and mp.tolist() == [0.0, -1.0]
+    assert np.allclose(st.X, [1.0, r], atol=1e-7)
+    step()
+    assert np.allclose(st.Xhalf, [1.0, s2], atol=1e-6) and np.allclose(gp, [[s2, -1.0]], atol=1e-6)
+    assert np.allclose(st.Y, [-s2, 2.0], atol=1e-6) and abs(st.sum_sq - 3.0) < 1e-6 and abs(st.gamma - 0.5) < 1e-6
+    assert np.allclose(st.X, [1.0 - s2 / 2, 1.0], atol=1e-6)
+    assert np.allclose(st.Xbar, [1.0, s2 / 2], atol=1e-6) and st.t == 3
+
+
+def test_family_closed_forms_for_a_constant_operator():
+    """A(x) = b for all x (M = 0), K workers, no noise, quantizer bypassed.
+    DA: sum after t steps = t K ||b||^2, so X_{T+1} = X_1 - T b K / sqrt(1 + T K ||b||^2).
+    OptDA: only the first iteration adds to the sum (K ||b||^2), so X_{T+1} = X_1 - T b K / sqrt(1 + K ||b||^2)."""
+    n, K, T = 6, 3, 7
+    b = np.array([0.5, -1.0, 0.25, 2.0, 0.0, -0.125], dtype=np.float32)
+    x1 = np.arange(n, dtype=np.float32)
+    op = o.Op(o.OP_DENSE_AFFINE, np.zeros((n, n), np.float32), b)
+    nb2 = float(np.dot(b.astype(np.float64), b.astype(np.float64)))
+    lev = np.array([0.0, 1.0], dtype=np.float32)
+    for method, total in ((o.METHOD_DA, T * K * nb2), (o.METHOD_OPTDA, K * nb2)):
+        st = o.EgState(x1, K=K)
+        gp, mp = np.zeros((K, n), np.float32), np.zeros(n, np.float32)
+        for _ in range(T):
+            o.family_step(st, method, op, None, 2, lev, o.codebook_fixed(2), 0, gp, mp, quantizer_off=True)
+        assert abs(st.sum_sq - total) <= 1e-12 * total
+        gam = K / math.sqrt(1.0 + total)
+        assert abs(st.gamma - gam) <= 1e-6 * gam
+        assert np.allclose(st.Y, -T * b.astype(np.float64), rtol=1e-6, atol=1e-6)
+        assert np.allclose(st.X, x1 - gam * T * b.astype(np.float64), rtol=1e-5, atol=1e-5)
+
+
+def test_family_step_is_the_pinned_exchange_plus_the_update_rules():
+    """Quantizer on: the step's feedback is exactly what the (separately pinned) exchange returns for the dual
+    vectors at X_{t+1/2} with exchange id 2t + 1, and the step-size sum grows by the squared differences."""
+    vi = gen.c4_affine(n=96, K=4, seed=7, bucket=32, noise_std=0.5)
+    M, b = vi.M.numpy(), vi.b.numpy()
+    op = o.Op(o.OP_DENSE_AFFINE, M, b)
+    lev = gen.uniform_levels(9).numpy().copy()
+    cb = o.codebook_fixed(9, 16)
+    for method in (o.METHOD_DA, o.METHOD_OPTDA):
+        st = o.EgState(vi.x0.numpy(), K=4)
+        gp, mp = np.zeros((4, 96), np.float32), np.zeros(96, np.float32)
+        for t in range(1, 6):
+            nz = vi.noise(t).numpy()[1]
+            x_before, y_before, s_before, g_before = st.X.copy(), st.Y.copy(), st.sum_sq, gp.copy()
+            gamma_t = np.float32(st.gamma)
+            xh = (x_before - gamma_t * mp).astype(np.float32) if method == o.METHOD_OPTDA else x_before
+            V = o.form_dual_vectors(o.apply_operator(op, xh), nz, 4)
+            mean, tot, vhat = o.exchange(V, vi.bucket, lev, cb, vi.seed, 2 * t + 1, return_vhat=True)
+            bits = o.family_step(st, method, op, nz, vi.bucket, lev, cb, vi.seed, gp, mp)
+            assert np.array_equal(st.Xhalf, xh) and bits == int(tot.sum())
+            assert np.array_equal(st.Y, y_before - mean)
+            before = g_before if method == o.METHOD_OPTDA else np.zeros_like(vhat)
+            inc = np.sum((before - vhat).astype(np.float64) ** 2)
+            assert abs((st.sum_sq - s_before) - inc) <= 1e-12 * max(inc, 1.0)
+            assert abs(st.gamma - 4.0 / math.sqrt(1.0 + st.sum_sq)) <= 1e-6 * st.gamma
+            if method == o.METHOD_OPTDA:
+                assert np.array_equal(gp, vhat) and np.array_equal(mp, mean)
+
+
+def test_optimistic_dual_averaging_solves_the_bilinear_game_where_dual_averaging_does_not():
+    """On min_x max_y x^T A y plain dual averaging is known to cycle or drift, the optimistic variant converges
+    (the reason the family carries an extrapolation step): trend only."""
+    def run(method, T):
+        g = gen.c1_bilinear(n=64, K=4, T=T, seed=11, noise_std=0.05, bucket=64)
+        op = o.Op(o.OP_BILINEAR, g.A.numpy())
+        st = o.EgState(g.z0.numpy(), K=4)
+        lev = gen.uniform_levels(9).numpy().copy()
+        cb = o.codebook_fixed(9, 32)
+        gp, mp = np.zeros((4, 128), np.float32), np.zeros(128, np.float32)
+        noise = g.noise.numpy()
+        for t in range(1, T + 1):
+            o.family_step(st, method, op, noise[t - 1, 1], g.bucket, lev, cb, g.seed, gp, mp)
+        return float(np.linalg.norm(st.Xbar)), float(np.linalg.norm(g.z0.numpy()))
+    e_opt_short, z0 = run(o.METHOD_OPTDA, 40)
+    e_opt_long, _ = run(o.METHOD_OPTDA, 240)
+    e_da_long, _ = run(o.METHOD_DA, 240)
+    assert e_opt_long < e_opt_short < z0
+    assert e_opt_long < e_da_long
