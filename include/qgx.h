@@ -271,6 +271,23 @@ qgx_status qgx_eg_init(qgx_ctx *ctx, qgx_eg_state *st /*[host]*/);
 qgx_status qgx_eg_step(qgx_ctx *ctx, qgx_eg_state *st, const qgx_operator *op,
                        const float *noise_t, const float *noise_half, qgx_quant_cfg *cfg,
                        int refit, uint64_t *bits);
+/* The other two members of the family that Sec. 3.1 lists (Eq. Quantized DA, Eq. Quantized OptDA): one
+ * oracle call and one exchange per iteration, same state, same step-size rule.
+ *   QGX_METHOD_DA:    Vhat_{k,t} = 0, so X_{t+1/2} = X_t;  g_k = Q(A(X_t) + U_k);  Y_{t+1} = Y_t - mean_k g_k;
+ *                     sum += sum_k ||g_k||^2.
+ *   QGX_METHOD_OPTDA: Vhat_{k,t} = g_{k,t-1/2}, the vectors of the previous iteration (zero in the first):
+ *                     X_{t+1/2} = X_t - gamma_t mean_k g_{k,t-1/2};  g_{k,t+1/2} = Q(A(X_{t+1/2}) + U_k);
+ *                     Y_{t+1} = Y_t - mean_k g_{k,t+1/2};  sum += sum_k ||g_{k,t-1/2} - g_{k,t+1/2}||^2.
+ * Then gamma_{t+1}, X_{t+1}, Xbar and t as in qgx_eg_step.  The exchange id is 2t + 1; a refit uses the
+ * iteration's only dual vectors.  noise [dev] float[K][d] or NULL.  mean_prev [dev] float[d] (OPTDA; may be
+ * NULL for DA) holds the mean of g_{k,t-1/2} between calls: read at t > 1, overwritten.  The previous vectors
+ * themselves stay in the context (symbols, norms and their level table), so between two OPTDA steps of one
+ * state no other exchange may run on this context (QGX_ERR_INVALID_ARG if the kept vectors do not fit).
+ * bits [dev] uint64[K], may be NULL. */
+enum { QGX_METHOD_DE = 0, QGX_METHOD_DA = 1, QGX_METHOD_OPTDA = 2 };
+qgx_status qgx_family_step(qgx_ctx *ctx, qgx_eg_state *st, int method, const qgx_operator *op,
+                           const float *noise, qgx_quant_cfg *cfg, int refit, float *mean_prev,
+                           uint64_t *bits);
 /* A(x) alone: out [dev] float[d]. */
 qgx_status qgx_apply_operator(qgx_ctx *ctx, const qgx_operator *op, const float *x, float *out);
 

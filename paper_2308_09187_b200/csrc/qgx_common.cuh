@@ -40,6 +40,8 @@ struct qgx_ctx {
   int sym_K;
   size_t sym_d;
   size_t sym_ld;                         // bytes per worker in the kept-symbol layout
+  int sym_nlev;                          // the level table those symbols were quantized with
+  float sym_levels[QGX_MAX_LEVELS];
   // optional per-kernel timing: pairs of events recorded around instrumented launches
   int timing_on;
   int timing_cap;                        // pairs allocated

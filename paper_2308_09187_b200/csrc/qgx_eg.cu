@@ -92,6 +92,14 @@ __global__ void __launch_bounds__(256) k_eg_finish(float* __restrict__ X, const 
   if (blockIdx.x == 0 && threadIdx.x == 0) scalars[1] = (double)gamma;
 }
 
+// X_{t+1/2} = X_t - gamma_t * m (optimistic dual averaging: m is the mean of the previous iteration's quantized vectors)
+__global__ void __launch_bounds__(256) k_half_from_mean(const float* __restrict__ X, const float* __restrict__ m,
+                                                        const double* __restrict__ scalars, float* __restrict__ Xhalf, size_t d) {
+  const float gamma = (float)scalars[1];
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (size_t)gridDim.x * blockDim.x)
+    Xhalf[i] = __fsub_rn(X[i], __fmul_rn(gamma, m[i]));
+}
+
 static unsigned grid_for(size_t n, int threads) {
   return (unsigned)std::max<size_t>(1, std::min<size_t>((n + threads - 1) / threads, 148 * 8));
 }
@@ -171,6 +179,53 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
   DualSource src2{noise_half, a, 0};
   ExchangeUpdate dual{2, st->Y, st->Y, st->scalars};                          // Y_{t+1} = Y_t - mean
   rc = exchange_impl(c, src2, K, d, cfg, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 2, st->scalars, 0);
+  if (rc != QGX_OK) return rc;
+  {
+    ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);
+    k_eg_finish<<<grid_for(d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->Xhalf, st->anchor, st->scalars, d, K, st->t);
+  }
+  count_launch(c);
+  st->t += 1;
+  return cuda_status(cudaGetLastError());
+}
+
+qgx_status qgx_family_step(qgx_ctx* c, qgx_eg_state* st, int method, const qgx_operator* op, const float* noise,
+                           qgx_quant_cfg* cfg, int refit, float* mean_prev, uint64_t* bits) {
+  if (!c || !st || !op || !cfg || !st->X || !st->Y || !st->Xbar || !st->Xhalf || !st->anchor || !st->scalars || st->t < 1 ||
+      op->d != st->d || st->K < 1)
+    return QGX_ERR_INVALID_ARG;
+  if (method != QGX_METHOD_DA && method != QGX_METHOD_OPTDA) return QGX_ERR_INVALID_ARG;
+  if (method == QGX_METHOD_OPTDA && !mean_prev) return QGX_ERR_INVALID_ARG;
+  if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
+  const size_t d = st->d;
+  const int K = st->K;
+  float* a = (float*)ws_get(c, WS_OPVAL, sizeof(float) * d);
+  float* mean = method == QGX_METHOD_OPTDA ? mean_prev : (float*)ws_get(c, WS_MEAN, sizeof(float) * d);
+  if (!a || !mean) return QGX_ERR_CUDA;
+
+  if (method == QGX_METHOD_OPTDA && st->t > 1) {
+    ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);
+    k_half_from_mean<<<grid_for(d, 256), 256, 0, c->stream>>>(st->X, mean_prev, st->scalars, st->Xhalf, d);   // g_{k,t-1/2}
+    count_launch(c);
+  } else {                                                                       // no earlier feedback: X_{t+1/2} = X_t
+    if (cudaMemcpyAsync(st->Xhalf, st->X, sizeof(float) * d, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
+      return QGX_ERR_CUDA;
+  }
+  qgx_status rc = apply_operator_impl(c, op, st->Xhalf, a);                    // A(X_{t+1/2})
+  if (rc != QGX_OK) return rc;
+  DualSource src{noise, a, 0};
+  if (refit != QGX_REFIT_NONE) {
+    double* hist = (double*)ws_get(c, WS_HIST, sizeof(double) * (size_t)std::max(cfg->nbins, 1));
+    if (!hist) return QGX_ERR_CUDA;
+    rc = refit_from_source(c, src, K, d, cfg, refit, hist, nullptr);
+    if (rc != QGX_OK) return rc;
+  }
+  // the symbol modes of the decode pass: dual averaging adds the squared vectors themselves; the optimistic variant
+  // compares with the vectors kept by the previous iteration (none in the first) and keeps the new ones
+  const int sym_mode = method == QGX_METHOD_DA ? 4 : (st->t == 1 ? 5 : 3);
+  const int slot = st->t & 1;                                                    // the kept norms live in the other slot
+  ExchangeUpdate dual{2, st->Y, st->Y, st->scalars};                            // Y_{t+1} = Y_t - mean
+  rc = exchange_impl(c, src, K, d, cfg, 2u * (uint32_t)st->t + 1u, slot, mean, bits, &dual, sym_mode, st->scalars, 0);
   if (rc != QGX_OK) return rc;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);

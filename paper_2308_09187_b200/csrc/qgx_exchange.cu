@@ -494,21 +494,24 @@ __device__ __forceinline__ void stage_symbol_row(uint32_t* dst, const uint8_t* s
   }
 }
 
-// shared memory of the decode kernel after its table: two stream rows and (SYM == 2) two symbol rows per warp
+// shared memory of the decode kernel after its table: two stream rows and (when comparing) two symbol rows per warp
 template <int G, int SYM>
 struct DecodeSmem {
   static constexpr int kStreamRow = 9 * G + 64;         // words, a multiple of 4
-  static constexpr size_t kBytes = sizeof(uint32_t) * 2 * (128 / 32) * (size_t)(kStreamRow + (SYM == 2 ? G * 8 : 0));
+  static constexpr size_t kBytes = sizeof(uint32_t) * 2 * (128 / 32) * (size_t)(kStreamRow + ((SYM & 2) ? G * 8 : 0));
 };
 
-// SYM: 0 plain, 1 also keeps the decoded symbols, 2 also compares with the symbols kept by the other exchange
+// SYM, a set of bits: 1 keeps the decoded symbols; 2 adds the squared differences between the vectors kept by an
+// earlier exchange (whose level table is `lt`) and the ones decoded now to *sum_sq; 4 adds the squared decoded values
+// themselves (an earlier vector of zero).  1 | 2 compares first and then overwrites the kept symbols in place.
 template <int G, int SYM>
 __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6)) k_exchange_decode(const __grid_constant__ DecodeArgs a,
                                                                       const __grid_constant__ CodeTable ct,
                                                                       const __grid_constant__ LevelTable lt) {
+  constexpr bool kStore = (SYM & 1) != 0, kCompare = (SYM & 2) != 0, kSquare = (SYM & 4) != 0;
   extern __shared__ __align__(16) unsigned char s_raw[];
-  __shared__ float s_lev[QGX_MAX_LEVELS];
-  // SYM == 2: the other exchange's symbol words of the warp's 32 sub-blocks, one worker ahead (asynchronous copies)
+  __shared__ float s_lev[QGX_MAX_LEVELS];            // the table of the kept symbols (comparing)
+  // comparing: the kept symbol words of the warp's 32 sub-blocks, one worker ahead (asynchronous copies)
   constexpr int kRowWords = G * 8;                      // 32 sub-blocks x G bytes
   // the stream words of the warp's 32 sub-blocks, one worker ahead (asynchronous copies): room for 8 bits per
   // symbol and sign on average; longer rows are partly read from the stream itself
@@ -550,11 +553,11 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
     float acc[G];
 #pragma unroll
     for (int i = 0; i < G; ++i) acc[i] = 0.0f;
-    uint32_t* my_rows = s_prev + (SYM == 2 ? (tid >> 5) * 2 * kRowWords : 0);
+    uint32_t* my_rows = s_prev + (kCompare ? (tid >> 5) * 2 * kRowWords : 0);
     uint32_t* my_stream = s_rows + (tid >> 5) * 2 * kStreamRow;
     __syncwarp();                                         // the previous sub-block's rows are no longer read
     SubBlockAt nxt = find_subblock<G>(a, 0, b, hdr_bits, s, count > 0, uniform, lane, my_stream, kStreamRow);
-    if (SYM == 2) stage_symbol_row<kRowWords>(my_rows, a.sym_prev + (gs >> 5) * (size_t)(32 * G), lane);
+    if (kCompare) stage_symbol_row<kRowWords>(my_rows, a.sym_prev + (gs >> 5) * (size_t)(32 * G), lane);
     asm volatile("cp.async.commit_group;" ::: "memory");
     for (int k = 0; k < a.K; ++k) {
       const SubBlockAt cur = nxt;
@@ -562,7 +565,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
       __syncwarp();                                       // every lane is done with the rows that are overwritten next
       if (k + 1 < a.K) {
         nxt = find_subblock<G>(a, k + 1, b, hdr_bits, s, count > 0, uniform, lane, my_stream + ((k + 1) & 1) * kStreamRow, kStreamRow);
-        if (SYM == 2)
+        if (kCompare)
           stage_symbol_row<kRowWords>(my_rows + ((k + 1) & 1) * kRowWords,
                                       a.sym_prev + (size_t)(k + 1) * a.sym_ld + (gs >> 5) * (size_t)(32 * G), lane);
       }
@@ -580,7 +583,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
           if ((i & 1) == 0) {                              // two symbols use at most 26 bits
             if (win.avail <= 32) win.refill();
           }
-          if (SYM == 2 && (i & 3) == 0) prev4 = prev_row[(i >> 2) * 32];
+          if (kCompare && (i & 3) == 0) prev4 = prev_row[(i >> 2) * 32];
           const DecEntry e = s_lut[win.lo & mask];
           const uint32_t L = e.len & 31u;
           flags |= e.len;
@@ -588,13 +591,14 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
           used += L;
           const float val = __fmul_rn(cur.norm, e.val);
           acc[i] = __fadd_rn(acc[i], val);
-          if (SYM == 1) {
-            pack |= ((e.len >> 8) & 0xffu) << (8 * (i & 3));
-            if ((i & 3) == 3) { *reinterpret_cast<uint32_t*>(a.sym_out + (size_t)k * a.sym_ld + sbase + (i >> 2) * 128) = pack; pack = 0; }
-          }
-          if (SYM == 2) {
+          if (kCompare) {
             const float dlt = __fsub_rn(dequantize_symbol((prev4 >> (8 * (i & 3))) & 0xffu, cur.norm_prev, s_lev), val);
             sq = fma((double)dlt, (double)dlt, sq);
+          }
+          if (kSquare) sq = fma((double)val, (double)val, sq);
+          if (kStore) {
+            pack |= ((e.len >> 8) & 0xffu) << (8 * (i & 3));
+            if ((i & 3) == 3) { *reinterpret_cast<uint32_t*>(a.sym_out + (size_t)k * a.sym_ld + sbase + (i >> 2) * 128) = pack; pack = 0; }
           }
         }
       } else {
@@ -611,11 +615,12 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
             used += L;
             const float val = __fmul_rn(cur.norm, e.val);
             acc[i] = __fadd_rn(acc[i], val);
-            if (SYM == 1) a.sym_out[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)] = (uint8_t)((e.len >> 8) & 0xffu);
-            if (SYM == 2) {
+            if (kCompare) {
               const float dlt = __fsub_rn(dequantize_symbol(a.sym_prev[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)], cur.norm_prev, s_lev), val);
               sq = fma((double)dlt, (double)dlt, sq);
             }
+            if (kSquare) sq = fma((double)val, (double)val, sq);
+            if (kStore) a.sym_out[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)] = (uint8_t)((e.len >> 8) & 0xffu);
           }
         }
       }
@@ -650,7 +655,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
       }
     }
   }
-  if (SYM == 2) {
+  if (kCompare || kSquare) {
     sq = warp_sum(sq);
     if (lane == 0 && sq != 0.0) atomicAdd(a.sum_sq, sq);
   }
@@ -721,14 +726,22 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const uint8_t* sym_prev = nullptr;
   const size_t sym_ld = ((nb * (size_t)(bucket / ct.G) + 31) / 32) * 32 * (size_t)ct.G;   // see DecodeArgs::sym_out
   const float* norms_prev = nullptr;
-  if (sym_mode == 1) {
+  if (sym_mode < 0 || sym_mode > 5) return QGX_ERR_INVALID_ARG;
+  if ((sym_mode & 6) && !sum_sq) return QGX_ERR_INVALID_ARG;
+  LevelTable lt_kept = lt;                                  // the table of the symbols compared with
+  if (sym_mode & 2) {
+    if (c->sym_slot != 1 - slot || c->sym_K != K || c->sym_d != d || c->sym_ld != sym_ld || c->slot_nb[1 - slot] != nb) return QGX_ERR_INVALID_ARG;
+    sym_prev = (const uint8_t*)c->ws[WS_SYM];
+    norms_prev = (const float*)c->ws[slot == 0 ? WS_NORMS2 : WS_NORMS];
+    lt_kept.nlev = c->sym_nlev;
+    for (int j = 0; j < QGX_MAX_LEVELS; ++j) lt_kept.lev[j] = j < c->sym_nlev ? c->sym_levels[j] : 1.0f;
+  }
+  if (sym_mode & 1) {
     sym_out = (uint8_t*)ws_get(c, WS_SYM, (size_t)K * sym_ld + 16);
     if (!sym_out) return QGX_ERR_CUDA;
     c->sym_slot = slot; c->sym_K = K; c->sym_d = d; c->sym_ld = sym_ld;
-  } else if (sym_mode == 2) {
-    if (!sum_sq || c->sym_slot != 1 - slot || c->sym_K != K || c->sym_d != d || c->sym_ld != sym_ld || c->slot_nb[1 - slot] != nb) return QGX_ERR_INVALID_ARG;
-    sym_prev = (const uint8_t*)c->ws[WS_SYM];
-    norms_prev = (const float*)c->ws[slot == 0 ? WS_NORMS2 : WS_NORMS];
+    c->sym_nlev = cfg->nlev;
+    for (int j = 0; j < cfg->nlev; ++j) c->sym_levels[j] = cfg->levels[j];
   }
   const PhiloxKey key = make_philox_key(cfg->seed);
   RoundTable qt;
@@ -797,7 +810,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   da.scalars = upd ? upd->scalars : nullptr; da.st = c->dstatus;
   da.vec_out = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(mean_out) & 15u) == 0) &&
                ((reinterpret_cast<uintptr_t>(da.xin) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(da.xout) & 15u) == 0);
-  return launch_decode_average(c, da, ct, lt, sym_mode);
+  return launch_decode_average(c, da, ct, lt_kept, sym_mode);
 }
 
 template <int G, int SYM>
@@ -820,9 +833,14 @@ static qgx_status launch_decode_gs(qgx_ctx* c, const DecodeArgs& da, const CodeT
 
 template <int G>
 static qgx_status launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt, int sym_mode) {
-  if (sym_mode == 1) return launch_decode_gs<G, 1>(c, da, ct, lt);
-  if (sym_mode == 2) return launch_decode_gs<G, 2>(c, da, ct, lt);
-  return launch_decode_gs<G, 0>(c, da, ct, lt);
+  switch (sym_mode) {
+    case 1: return launch_decode_gs<G, 1>(c, da, ct, lt);
+    case 2: return launch_decode_gs<G, 2>(c, da, ct, lt);
+    case 3: return launch_decode_gs<G, 3>(c, da, ct, lt);
+    case 4: return launch_decode_gs<G, 4>(c, da, ct, lt);
+    case 5: return launch_decode_gs<G, 5>(c, da, ct, lt);
+    default: return launch_decode_gs<G, 0>(c, da, ct, lt);
+  }
 }
 
 qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt, int sym_mode) {

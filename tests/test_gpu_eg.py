@@ -162,3 +162,65 @@ def test_diagonal_operator_scale_shape(q):
         o.eg_step(st_o, opo, noise[0], noise[1], c5.bucket, lev, cbo, c5.seed)
         qgx.qgx_sync_status(ctx)
         _compare(st, st_o)
+
+
+@pytest.mark.parametrize("method", ["da", "optda"])
+def test_dual_averaging_and_optimistic_variant(q, method):
+    """The one-exchange members of the family (Eq. Quantized DA, Eq. Quantized OptDA) against the oracle, teacher
+    forced, with refits in between (the optimistic variant then compares vectors quantized with two different
+    level tables).  Diagonal operator: the dual vectors are bit-identical on both sides."""
+    qgx, ctx = q
+    K, d, bucket, sub = 4, 3 * 2048 + 100, 2048, 64
+    c5 = gen.c5_diagonal(K=K, d=d, device="cuda", bucket=bucket, seed=77)
+    D, x0, noise = c5.D.cpu().numpy(), c5.x0.cpu().numpy(), c5.noise.cpu().numpy()
+    m_gpu = qgx.QGX_METHOD_DA if method == "da" else qgx.QGX_METHOD_OPTDA
+    m_or = o.METHOD_DA if method == "da" else o.METHOD_OPTDA
+    lev = gen.uniform_levels(17).numpy().copy()
+    cfg = qgx.make_quant_cfg(lev, bucket, qgx.qgx_build_codebook_fixed(17, sub), c5.seed, code_type=qgx.QGX_CODE_HUFFMAN)
+    op, opo = qgx.make_operator(qgx.QGX_OP_DIAGONAL, c5.D), o.Op(o.OP_DIAGONAL, D)
+    st = qgx.EgState(c5.x0, K)
+    qgx.qgx_eg_init(ctx, st)
+    st_o = o.EgState(x0, K)
+    cbo = o.codebook_fixed(17, sub)
+    mean_prev = torch.zeros(d, dtype=torch.float32, device="cuda")
+    gp, mp = np.zeros((K, d), np.float32), np.zeros(d, np.float32)
+    bits = torch.zeros(K, dtype=torch.int64, device="cuda")
+    for t in range(1, 8):
+        refit = 2 if t == 1 else (1 if t % 3 == 0 else 0)
+        nz_t = (t % 2)                                   # alternate the two noise sets
+        _load_state(qgx, st, st_o)
+        mean_prev.copy_(torch.from_numpy(mp))
+        qgx.qgx_family_step(ctx, st, m_gpu, op, c5.noise[nz_t], cfg, refit=refit, mean_prev=mean_prev, bits=bits)
+        qgx.qgx_sync_status(ctx)
+        if refit:
+            lev = np.array(cfg.level_list(), dtype=np.float32)
+            cbo = o.codebook_from(cfg.cb.lengths(), cfg.cb.codes(), subblock=sub)
+        sent = o.family_step(st_o, m_or, opo, noise[nz_t], bucket, lev, cbo, c5.seed, gp, mp)
+        _compare(st, st_o, tol=1e-6)
+        assert int(bits.sum().item()) == sent
+        if method == "optda":
+            assert np.array_equal(mean_prev.cpu().numpy(), mp)
+    assert st_o.sum_sq > 0
+
+
+def test_optimistic_dual_averaging_free_running_on_the_affine_problem(q):
+    """c4 at reduced size, free running (no teacher forcing): the library's own iterates approach the solution."""
+    qgx, ctx = q
+    n, T = 512, 120
+    vi = gen.c4_affine(n=n, K=8, device="cuda", bucket=128)
+    M, b = vi.M.cpu().numpy(), vi.b.cpu().numpy()
+    xstar = np.linalg.solve(M.astype(np.float64), -b.astype(np.float64))
+    cfg = qgx.make_quant_cfg(gen.uniform_levels(17).numpy(), vi.bucket, qgx.qgx_build_codebook_fixed(17, 32), vi.seed,
+                             code_type=qgx.QGX_CODE_HUFFMAN, nbins=256)
+    op = qgx.make_operator(qgx.QGX_OP_DENSE_AFFINE, vi.M, vi.b)
+    st = qgx.EgState(vi.x0, vi.K)
+    qgx.qgx_eg_init(ctx, st)
+    mean_prev = torch.zeros(n, dtype=torch.float32, device="cuda")
+    errs = {}
+    for t in range(1, T + 1):
+        refit = 2 if t == 1 else (1 if (t - 1) % 10 == 0 else 0)
+        qgx.qgx_family_step(ctx, st, qgx.QGX_METHOD_OPTDA, op, vi.noise(t)[1], cfg, refit=refit, mean_prev=mean_prev)
+        if t in (15, T):
+            qgx.qgx_sync_status(ctx)
+            errs[t] = float(np.linalg.norm(st.Xbar.cpu().numpy() - xstar) / np.linalg.norm(xstar))
+    assert errs[T] < errs[15] < 1.0
