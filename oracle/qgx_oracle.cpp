@@ -188,7 +188,7 @@ struct qgxo_codebook {
 
 struct qgxo_operator {
   int32_t kind;            // 0 dense affine (M row-major d x d, b), 1 bilinear (A n x n, d = 2n), 2 diagonal (D)
-  int32_t pad;
+  int32_t noise_model;     // how a worker's noise enters its dual vector: 0 V_k = A(x) + U_k, 1 V_k = A(x) .* U_k
   uint64_t d;
   const float* mat;        // M, A or D
   const float* bias;       // b (dense affine) or null
@@ -766,9 +766,23 @@ int qgxo_apply_operator(const qgxo_operator* op, const float* x, float* out) {
 
 // Stochastic dual vectors of the K workers at one point: V_k = A(x) + U_k (Eq. "oracle"),
 // one fp32 addition per coordinate; U null means no noise.
+// The relative-noise oracles of Assumption 3 (random coordinate descent, random player updating: App. on
+// examples): worker k sees A(x) through a random non-negative scale, V_k = A(x) .* S_k with E[S_k] = 1 (S_k = 0 on
+// the coordinates that are not drawn, 1/p on those drawn with probability p), so the noise V_k - A(x) vanishes
+// where A does.  One fp32 multiplication per coordinate; S null means no noise.
+void qgxo_form_dual_vectors_relative(const float* a, const float* S, int K, uint64_t d, float* V) {
+  for (int k = 0; k < K; ++k)
+    for (uint64_t i = 0; i < d; ++i) V[(uint64_t)k * d + i] = S ? a[i] * S[(uint64_t)k * d + i] : a[i];
+}
+
 void qgxo_form_dual_vectors(const float* a, const float* U, int K, uint64_t d, float* V) {
   for (int k = 0; k < K; ++k)
     for (uint64_t i = 0; i < d; ++i) V[(uint64_t)k * d + i] = U ? a[i] + U[(uint64_t)k * d + i] : a[i];
+}
+
+static void form_by_model(const qgxo_operator* op, const float* a, const float* noise, int K, uint64_t d, float* V) {
+  if (op->noise_model == 1) qgxo_form_dual_vectors_relative(a, noise, K, d, V);
+  else qgxo_form_dual_vectors(a, noise, K, d, V);
 }
 
 // One exchange of Algorithm 1: every worker quantizes and encodes its vector, every stream is
@@ -855,7 +869,7 @@ int qgxo_eg_step(qgxo_eg_state* st, const qgxo_operator* op, const float* noise_
   std::vector<uint64_t> tb1(K), tb2(K);
   int rc = qgxo_apply_operator(op, st->X, a.data());
   if (rc) return rc;
-  qgxo_form_dual_vectors(a.data(), noise_t, K, d, V.data());
+  form_by_model(op, a.data(), noise_t, K, d, V.data());
   if (refit && !quantizer_off) {
     rc = qgxo_refit(V.data(), K, d, bucket, norm_type, nbins, refit == 2, code_type, lev, nlev, cb, nullptr);
     if (rc) return rc;
@@ -866,7 +880,7 @@ int qgxo_eg_step(qgxo_eg_state* st, const qgxo_operator* op, const float* noise_
   for (uint64_t i = 0; i < d; ++i) { const float step = st->gamma * mean[i]; st->Xhalf[i] = st->X[i] - step; }
   rc = qgxo_apply_operator(op, st->Xhalf, a.data());
   if (rc) return rc;
-  qgxo_form_dual_vectors(a.data(), noise_half, K, d, V.data());
+  form_by_model(op, a.data(), noise_half, K, d, V.data());
   rc = qgxo_exchange_full(V.data(), K, d, bucket, norm_type, lev, nlev, cb, seed, 2u * (uint32_t)st->t + 1u,
                           quantizer_off, vhat2.data(), mean.data(), tb2.data());
   if (rc) return rc;
@@ -913,7 +927,7 @@ int qgxo_family_step(qgxo_eg_state* st, int method, const qgxo_operator* op, con
   }
   int rc = qgxo_apply_operator(op, st->Xhalf, a.data());
   if (rc) return rc;
-  qgxo_form_dual_vectors(a.data(), noise, K, d, V.data());
+  form_by_model(op, a.data(), noise, K, d, V.data());
   if (refit && !quantizer_off) {
     rc = qgxo_refit(V.data(), K, d, bucket, norm_type, nbins, refit == 2, code_type, lev, nlev, cb, nullptr);
     if (rc) return rc;

@@ -33,7 +33,7 @@ class Codebook(C.Structure):
 
 
 class Operator(C.Structure):
-    _fields_ = [("kind", C.c_int32), ("pad", C.c_int32), ("d", C.c_uint64),
+    _fields_ = [("kind", C.c_int32), ("noise_model", C.c_int32), ("d", C.c_uint64),
                 ("mat", C.c_void_p), ("bias", C.c_void_p)]
 
 
@@ -66,6 +66,7 @@ def lib():
         _lib.qgxo_stationarity.restype = C.c_double
         _lib.qgxo_stationarity.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_double]
         _lib.qgxo_form_dual_vectors.restype = None
+        _lib.qgxo_form_dual_vectors_relative.restype = None
     return _lib
 
 
@@ -304,14 +305,17 @@ def refit(v, bucket, nbins, levels, cb, first_fit, code_type, norm_type=L2):
 
 
 # ------------------------------------------------------------------ operator and iteration
+NOISE_ADDITIVE, NOISE_RELATIVE = 0, 1
+
+
 class Op:
-    def __init__(self, kind, mat, bias=None):
+    def __init__(self, kind, mat, bias=None, noise_model=NOISE_ADDITIVE):
         self.kind = kind
         self.mat = _f32(mat)
         self.bias = _f32(bias) if bias is not None else None
         d = 2 * self.mat.shape[0] if kind == OP_BILINEAR else self.mat.shape[0]
         self.d = d
-        self.c = Operator(kind, 0, d, self.mat.ctypes.data, self.bias.ctypes.data if self.bias is not None else None)
+        self.c = Operator(kind, noise_model, d, self.mat.ctypes.data, self.bias.ctypes.data if self.bias is not None else None)
 
 
 def apply_operator(op, x):
@@ -327,6 +331,16 @@ def form_dual_vectors(a, noise, K):
     n = _f32(noise) if noise is not None else None
     V = np.zeros((K, d), dtype=np.float32)
     lib().qgxo_form_dual_vectors(_p(a), _p(n), K, C.c_uint64(d), _p(V))
+    return V
+
+
+def form_dual_vectors_relative(a, scales, K):
+    """V_k = A(x) .* S_k (relative noise)."""
+    a = _f32(a)
+    d = a.shape[0]
+    n = _f32(scales) if scales is not None else None
+    V = np.zeros((K, d), dtype=np.float32)
+    lib().qgxo_form_dual_vectors_relative(_p(a), _p(n), K, C.c_uint64(d), _p(V))
     return V
 
 

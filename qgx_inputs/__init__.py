@@ -171,6 +171,18 @@ def c5_diagonal(K=32, d=1 << 26, device="cpu", seed=1005, bucket=16384) -> Diago
     return DiagonalScale(D, x0, noise, K=K, bucket=bucket, seed=seed)
 
 
+def player_scales(shape, block: int, p: float, seed: int, device="cpu") -> torch.Tensor:
+    """Random player updating / random block coordinate descent as a relative-noise oracle: the last axis is cut
+    into blocks of `block` coordinates (players); every (leading index, block) is drawn independently with
+    probability p and its coordinates get the scale 1/p, all others 0 -- so the scales have mean one."""
+    d = shape[-1]
+    nblk = (d + block - 1) // block
+    g = torch.Generator(device="cpu").manual_seed(int(seed))
+    drawn = (torch.rand(tuple(shape[:-1]) + (nblk,), generator=g) < p).to(torch.float32) / float(p)
+    out = drawn.repeat_interleave(block, dim=-1)[..., :d].contiguous()
+    return out.to(device)
+
+
 def uniform_levels(nlev: int) -> torch.Tensor:
     """l_j = j/(nlev-1): the level table before the first fit."""
     return torch.arange(nlev, dtype=torch.float64).div(nlev - 1).to(torch.float32)

@@ -251,3 +251,77 @@ def test_optimistic_dual_averaging_solves_the_bilinear_game_where_dual_averaging
     e_da_long, _ = run(o.METHOD_DA, 240)
     assert e_opt_long < e_opt_short < z0
     assert e_opt_long < e_da_long
+
+
+# ---- relative noise (Assumption 3; random player updating of the appendix on examples) ----
+
+def test_relative_noise_oracle_is_a_product_with_mean_one_scales():
+    a = np.array([2.0, -3.0, 0.0, 0.5], dtype=np.float32)
+    S = np.array([[2.0, 0.0, 2.0, 0.0], [0.0, 2.0, 2.0, 2.0]], dtype=np.float32)
+    assert o.form_dual_vectors_relative(a, S, 2).tolist() == [[4.0, -0.0, 0.0, 0.0], [0.0, -6.0, 0.0, 1.0]]
+    assert o.form_dual_vectors_relative(a, None, 3).tolist() == [a.tolist()] * 3
+    # where the operator vanishes the dual vectors vanish, whatever was drawn: the noise is relative
+    assert not o.form_dual_vectors_relative(np.zeros(4, np.float32), S, 2).any()
+    # the seeded scales: blocks of equal values in {0, 1/p}, mean one, relative variance 1/p - 1
+    s = gen.player_scales((4, 1 << 16), 64, 0.25, seed=3).numpy()
+    assert set(np.unique(s).tolist()) == {0.0, 4.0}
+    assert np.all(s.reshape(4, -1, 64) == s.reshape(4, -1, 64)[:, :, :1])
+    assert abs(s.mean() - 1.0) < 0.05 and abs(s.var() - 3.0) < 0.3
+    assert np.array_equal(s, gen.player_scales((4, 1 << 16), 64, 0.25, seed=3).numpy())
+
+
+def _relative_run(model, T, K=4, d=256, seed=5):
+    D = gen.uniform((d,), seed, "cpu", 0.2, 1.0).numpy()
+    x0 = gen.gaussian((d,), seed + 1, "cpu").numpy()
+    op = o.Op(o.OP_DIAGONAL, D, noise_model=model)                 # gradient of a convex quadratic: co-coercive
+    st = o.EgState(x0, K)
+    lev = gen.uniform_levels(17).numpy().copy()
+    cb = o.codebook_fixed(17, 32)
+    sigma = float(np.linalg.norm(D * x0) / math.sqrt(d))          # absolute noise as large as the relative one at x0
+    marks = {}
+    for t in range(1, T + 1):
+        if model == o.NOISE_RELATIVE:
+            nz = gen.player_scales((2, K, d), 64, 0.5, seed * 1000 + t).numpy()
+        else:
+            nz = gen.gaussian((2, K, d), seed * 1000 + t, "cpu", std=sigma).numpy()
+        refit = 2 if t == 1 else (1 if t % 20 == 1 else 0)
+        o.eg_step(st, op, nz[0], nz[1], 512, lev, cb, seed, refit=refit, code_type=o.CODE_HUFFMAN, nbins=256)
+        if t in (T // 4, T):
+            nx = float(np.linalg.norm(x0))
+            marks[t] = (float(np.linalg.norm(st.Xbar)) / nx, float(np.linalg.norm(st.X)) / nx, st.gamma)
+    return marks
+
+
+def test_relative_noise_gives_the_fast_regime():
+    """Theorem 4 against Theorem 3, as trends: with relative noise and a co-coercive operator the squared differences
+    are summable, so the adaptive step stops shrinking, the iterates themselves converge and the ergodic average
+    gains about 1/T; with absolute noise of the same initial size the step keeps shrinking like 1/sqrt t and the
+    average gains about 1/sqrt T."""
+    T = 800
+    rel, ab = _relative_run(o.NOISE_RELATIVE, T), _relative_run(o.NOISE_ADDITIVE, T)
+    assert rel[T][2] > 0.95 * rel[T // 4][2]                       # step size settled
+    assert ab[T][2] < 0.65 * ab[T // 4][2]                         # step size still falling
+    assert rel[T // 4][0] / rel[T][0] > 2.5                        # four times the iterations: close to 4x
+    assert ab[T // 4][0] / ab[T][0] < 2.0                          # close to 2x
+    assert rel[T][1] < 0.02 < ab[T][1]                             # the last iterate itself
+
+
+def test_relative_noise_special_cases():
+    d, K = 96, 3
+    D = gen.uniform((d,), 1, "cpu", 0.2, 1.0).numpy()
+    lev = gen.uniform_levels(9).numpy().copy()
+    cb = o.codebook_fixed(9, 32)
+    # the solution is a fixed point whatever is drawn (under additive noise it is not)
+    st = o.EgState(np.zeros(d, np.float32), K)
+    S = gen.player_scales((2, K, d), 8, 0.5, seed=2).numpy()
+    for _ in range(3):
+        o.eg_step(st, o.Op(o.OP_DIAGONAL, D, noise_model=o.NOISE_RELATIVE), S[0], S[1], 32, lev, cb, 9)
+    assert not st.X.any() and not st.Y.any() and st.sum_sq == 0.0 and st.gamma == K
+    # scales of one are no noise at all
+    x0 = gen.gaussian((d,), 4, "cpu").numpy()
+    a, b = o.EgState(x0, K), o.EgState(x0, K)
+    ones = np.ones((K, d), np.float32)
+    for _ in range(3):
+        o.eg_step(a, o.Op(o.OP_DIAGONAL, D, noise_model=o.NOISE_RELATIVE), ones, ones, 32, lev, cb, 9)
+        o.eg_step(b, o.Op(o.OP_DIAGONAL, D), None, None, 32, lev, cb, 9)
+    assert np.array_equal(a.X, b.X) and a.sum_sq == b.sum_sq
