@@ -79,12 +79,16 @@ typedef struct {
   qgx_codebook cb;
 } qgx_quant_cfg;
 
+enum { QGX_NOISE_ADDITIVE = 0, QGX_NOISE_RELATIVE = 1 };
+
 /* Monotone operator A of the VI (Sec. 2).  DENSE_AFFINE: A(x) = M x + b, M row-major d x d.
  * BILINEAR: the game min_x max_y x^T A y with z = (x, y), A n x n row-major, d = 2n,
  * A(z) = (A y, -A^T x).  DIAGONAL: A(x) = D .* x.  mat and bias are [dev]. */
 typedef struct {
   int32_t kind;
-  int32_t pad;
+  int32_t noise_model;      /* how a worker's noise array enters its dual vector: QGX_NOISE_ADDITIVE (Assumption 2)
+                             * V_k = A(x) + U_k; QGX_NOISE_RELATIVE (Assumption 3, e.g. random player updating)
+                             * V_k = A(x) .* S_k with non-negative scales of mean one */
   uint64_t d;
   const float *mat;
   const float *bias;        /* DENSE_AFFINE only; may be NULL */

@@ -55,7 +55,8 @@ class qgx_quant_cfg(C.Structure):
 
 
 class qgx_operator(C.Structure):
-    _fields_ = [("kind", C.c_int32), ("pad", C.c_int32), ("d", C.c_uint64), ("mat", C.c_void_p), ("bias", C.c_void_p)]
+    _fields_ = [("kind", C.c_int32), ("noise_model", C.c_int32), ("d", C.c_uint64), ("mat", C.c_void_p),
+                ("bias", C.c_void_p)]
 
 
 class qgx_eg_state(C.Structure):
@@ -382,9 +383,12 @@ class EgState:
         return float(s[0]), float(s[1])
 
 
-def make_operator(kind, mat, bias=None):
+QGX_NOISE_ADDITIVE, QGX_NOISE_RELATIVE = 0, 1
+
+
+def make_operator(kind, mat, bias=None, noise_model=QGX_NOISE_ADDITIVE):
     d = 2 * mat.shape[0] if kind == QGX_OP_BILINEAR else mat.shape[0]
-    op = qgx_operator(kind, 0, d, mat.data_ptr(), bias.data_ptr() if bias is not None else None)
+    op = qgx_operator(kind, noise_model, d, mat.data_ptr(), bias.data_ptr() if bias is not None else None)
     op._keep = (mat, bias)
     return op
 

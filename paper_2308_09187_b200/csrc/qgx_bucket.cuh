@@ -23,17 +23,24 @@ inline int bucket_v4(int bucket) {
 }
 
 // Source of a dual vector's coordinates: v alone, or a + u (V_k = A(x) + U_k of Eq. "oracle",
-// one fp32 addition), or a alone when u is null.
+// one fp32 addition), or a * u (relative noise, Assumption 3: one fp32 multiplication), or a alone when u is null.
 struct DualSource {
   const float* v;        // [K][d] plain vectors, or the noise U; may be null when a is given
   const float* a;        // [d] operator value A(x) shared by all workers; null for plain vectors
   size_t ld;             // distance between workers' rows of v in floats; 0 means d
+  int mul;               // with both arrays: 0 the sum a + v, 1 the product a * v (relative noise: v holds scales)
 };
+
+__device__ __forceinline__ float dual_combine(float a, float v, int mul) { return mul ? __fmul_rn(a, v) : __fadd_rn(a, v); }
+__device__ __forceinline__ float4 dual_combine(float4 a, float4 v, int mul) {
+  return mul ? make_float4(__fmul_rn(a.x, v.x), __fmul_rn(a.y, v.y), __fmul_rn(a.z, v.z), __fmul_rn(a.w, v.w))
+             : make_float4(__fadd_rn(a.x, v.x), __fadd_rn(a.y, v.y), __fadd_rn(a.z, v.z), __fadd_rn(a.w, v.w));
+}
 
 __device__ __forceinline__ float dual_value(const DualSource& s, size_t k, size_t d, size_t i) {
   const size_t ld = s.ld ? s.ld : d;
   if (s.a == nullptr) return s.v[k * ld + i];
-  return s.v ? __fadd_rn(s.a[i], s.v[k * ld + i]) : s.a[i];
+  return s.v ? dual_combine(s.a[i], s.v[k * ld + i], s.mul) : s.a[i];
 }
 
 template <int V4>
@@ -58,7 +65,7 @@ __device__ __forceinline__ void load_bucket(BucketRegs<V4>& r, const DualSource&
         const float4 a = __ldg(reinterpret_cast<const float4*>(s.a + lo + e));
         if (s.v) {
           const float4 u = __ldcs(reinterpret_cast<const float4*>(s.v + k * ld + lo + e));
-          x = make_float4(__fadd_rn(a.x, u.x), __fadd_rn(a.y, u.y), __fadd_rn(a.z, u.z), __fadd_rn(a.w, u.w));
+          x = dual_combine(a, u, s.mul);
         } else {
           x = a;
         }

@@ -163,7 +163,8 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
 
   qgx_status rc = apply_operator_impl(c, op, st->X, a);                      // A(X_t)
   if (rc != QGX_OK) return rc;
-  DualSource src{noise_t, a, 0};                                                // V_{k,t} = A(X_t) + U_{k,t}
+  const int mul = op->noise_model == QGX_NOISE_RELATIVE ? 1 : 0;
+  DualSource src{noise_t, a, 0, mul};                                           // V_{k,t} = A(X_t) + U_{k,t}  (or .* S_{k,t})
   if (refit != QGX_REFIT_NONE) {
     double* hist = (double*)ws_get(c, WS_HIST, sizeof(double) * (size_t)std::max(cfg->nbins, 1));
     if (!hist) return QGX_ERR_CUDA;
@@ -176,7 +177,7 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
   if (rc != QGX_OK) return rc;
   rc = apply_operator_impl(c, op, st->Xhalf, a);                              // A(X_{t+1/2})
   if (rc != QGX_OK) return rc;
-  DualSource src2{noise_half, a, 0};
+  DualSource src2{noise_half, a, 0, mul};
   ExchangeUpdate dual{2, st->Y, st->Y, st->scalars};                          // Y_{t+1} = Y_t - mean
   rc = exchange_impl(c, src2, K, d, cfg, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 2, st->scalars, 0);
   if (rc != QGX_OK) return rc;
@@ -213,7 +214,7 @@ qgx_status qgx_family_step(qgx_ctx* c, qgx_eg_state* st, int method, const qgx_o
   }
   qgx_status rc = apply_operator_impl(c, op, st->Xhalf, a);                    // A(X_{t+1/2})
   if (rc != QGX_OK) return rc;
-  DualSource src{noise, a, 0};
+  DualSource src{noise, a, 0, op->noise_model == QGX_NOISE_RELATIVE ? 1 : 0};
   if (refit != QGX_REFIT_NONE) {
     double* hist = (double*)ws_get(c, WS_HIST, sizeof(double) * (size_t)std::max(cfg->nbins, 1));
     if (!hist) return QGX_ERR_CUDA;

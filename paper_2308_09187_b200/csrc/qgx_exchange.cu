@@ -130,7 +130,7 @@ __device__ __forceinline__ void load_bucket_octets(BucketRegs<2 * P>& r, const D
         const float4 av = __ldg(reinterpret_cast<const float4*>(s.a + lo + e));
         if (s.v) {
           const float4 u = __ldcs(reinterpret_cast<const float4*>(s.v + k * ld + lo + e));
-          x = make_float4(__fadd_rn(av.x, u.x), __fadd_rn(av.y, u.y), __fadd_rn(av.z, u.z), __fadd_rn(av.w, u.w));
+          x = dual_combine(av, u, s.mul);
         } else {
           x = av;
         }
@@ -862,7 +862,7 @@ extern "C" {
 qgx_status qgx_exchange(qgx_ctx* c, const float* v, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t exchange_id,
                         int slot, float* mean_out, uint64_t* total_bits) {
   if (!v) return QGX_ERR_INVALID_ARG;
-  DualSource src{v, nullptr, 0};
+  DualSource src{v, nullptr, 0, 0};
   return exchange_impl(c, src, K, d, cfg, exchange_id, slot, mean_out, total_bits, nullptr, 0, nullptr, 0);
 }
 
@@ -884,7 +884,7 @@ qgx_status qgx_exchange_segments(qgx_ctx* c, const float* v, int K, size_t d, co
     if (cudaMemsetAsync(total_bits, 0, sizeof(uint64_t) * (size_t)K, c->stream) != cudaSuccess) return QGX_ERR_CUDA;
   }
   for (int s = 0; s < nseg; ++s) {
-    DualSource src{v + segs[s].offset, nullptr, d};
+    DualSource src{v + segs[s].offset, nullptr, d, 0};
     qgx_status rc = exchange_impl(c, src, K, segs[s].length, segs[s].cfg, exchange_id, 0, mean_out + segs[s].offset, seg_bits,
                                   nullptr, 0, nullptr, segs[s].offset);
     if (rc != QGX_OK) return rc;

@@ -114,14 +114,14 @@ extern "C" {
 qgx_status qgx_histogram(qgx_ctx* c, const float* v, int K, size_t d, int bucket, int norm_type, int nbins, int weighted,
                          double* hist) {
   if (!v) return QGX_ERR_INVALID_ARG;
-  DualSource src{v, nullptr, 0};
+  DualSource src{v, nullptr, 0, 0};
   return launch_histogram(c, src, K, d, bucket, norm_type, nbins, weighted, hist);
 }
 
 qgx_status qgx_update_levels(qgx_ctx* c, const float* v, int K, size_t d, qgx_quant_cfg* cfg, int refit, double* hist,
                              double* hist_host) {
   if (!v) return QGX_ERR_INVALID_ARG;
-  DualSource src{v, nullptr, 0};
+  DualSource src{v, nullptr, 0, 0};
   return refit_from_source(c, src, K, d, cfg, refit, hist, hist_host);
 }
 

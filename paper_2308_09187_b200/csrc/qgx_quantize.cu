@@ -141,7 +141,7 @@ qgx_status qgx_quantize(qgx_ctx* c, const float* v, int K, size_t d, int bucket,
   LevelTable lt;
   lt.nlev = nlev;
   for (int j = 0; j < QGX_MAX_LEVELS; ++j) lt.lev[j] = j < nlev ? levels[j] : 1.0f;
-  DualSource src{v, nullptr, 0};
+  DualSource src{v, nullptr, 0, 0};
   return launch_quantize(c, src, K, d, bucket, lt, norm_type, seed, exchange_id, (flags & QGX_NORMS_SUPPLIED) ? 1 : 0,
                          norms, sym);
 }

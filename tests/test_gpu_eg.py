@@ -224,3 +224,53 @@ def test_optimistic_dual_averaging_free_running_on_the_affine_problem(q):
             qgx.qgx_sync_status(ctx)
             errs[t] = float(np.linalg.norm(st.Xbar.cpu().numpy() - xstar) / np.linalg.norm(xstar))
     assert errs[T] < errs[15] < 1.0
+
+
+def test_relative_noise_iteration(q):
+    """Assumption 3: V_k = A(x) .* S_k with random player-update scales, fused into the quantizer's load; teacher
+    forced against the oracle for the two-exchange iteration and the optimistic variant, then the fixed point."""
+    qgx, ctx = q
+    K, d, bucket, sub = 4, 2 * 4096 + 300, 4096, 64
+    D = gen.uniform((d,), 21, "cuda", 0.2, 1.0)
+    x0 = gen.gaussian((d,), 22, "cuda")
+    op = qgx.make_operator(qgx.QGX_OP_DIAGONAL, D, noise_model=qgx.QGX_NOISE_RELATIVE)
+    opo = o.Op(o.OP_DIAGONAL, D.cpu().numpy(), noise_model=o.NOISE_RELATIVE)
+    lev = gen.uniform_levels(17).numpy().copy()
+    cfg = qgx.make_quant_cfg(lev, bucket, qgx.qgx_build_codebook_fixed(17, sub), 5, code_type=qgx.QGX_CODE_HUFFMAN)
+    cbo = o.codebook_fixed(17, sub)
+    st, st_o = qgx.EgState(x0, K), o.EgState(x0.cpu().numpy(), K)
+    qgx.qgx_eg_init(ctx, st)
+    for t in range(1, 5):
+        S = gen.player_scales((2, K, d), 128, 0.5, 900 + t, device="cuda")
+        refit = 2 if t == 1 else 0
+        _load_state(qgx, st, st_o)
+        qgx.qgx_eg_step(ctx, st, op, S[0], S[1], cfg, refit=refit)
+        qgx.qgx_sync_status(ctx)
+        if refit:
+            lev = np.array(cfg.level_list(), dtype=np.float32)
+            cbo = o.codebook_from(cfg.cb.lengths(), cfg.cb.codes(), subblock=sub)
+        Sh = S.cpu().numpy()
+        o.eg_step(st_o, opo, Sh[0], Sh[1], bucket, lev, cbo, 5)
+        _compare(st, st_o, tol=1e-6)
+    # optimistic variant under the same oracle
+    st2, st2_o = qgx.EgState(x0, K), o.EgState(x0.cpu().numpy(), K)
+    qgx.qgx_eg_init(ctx, st2)
+    mean_prev = torch.zeros(d, dtype=torch.float32, device="cuda")
+    gp, mp = np.zeros((K, d), np.float32), np.zeros(d, np.float32)
+    for t in range(1, 4):
+        S = gen.player_scales((K, d), 128, 0.5, 950 + t, device="cuda")
+        _load_state(qgx, st2, st2_o)
+        mean_prev.copy_(torch.from_numpy(mp))
+        qgx.qgx_family_step(ctx, st2, qgx.QGX_METHOD_OPTDA, op, S, cfg, mean_prev=mean_prev)
+        qgx.qgx_sync_status(ctx)
+        o.family_step(st2_o, o.METHOD_OPTDA, opo, S.cpu().numpy(), bucket, lev, cbo, 5, gp, mp)
+        _compare(st2, st2_o, tol=1e-6)
+    # at the solution nothing moves, whatever is drawn
+    z = torch.zeros(d, dtype=torch.float32, device="cuda")
+    st3 = qgx.EgState(z, K)
+    qgx.qgx_eg_init(ctx, st3)
+    S = gen.player_scales((2, K, d), 128, 0.5, 999, device="cuda")
+    qgx.qgx_eg_step(ctx, st3, op, S[0], S[1], cfg)
+    qgx.qgx_sync_status(ctx)
+    s, g = st3.read_scalars()
+    assert not st3.X.any().item() and s == 0.0 and g == K
