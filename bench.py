@@ -36,7 +36,9 @@ WORKLOAD = "c5-scale: K=32, d=2^26, mixture noise, diagonal operator, bucket 163
 
 
 # measured DRAM traffic of k_exchange_encode per coordinate (ncu, current kernel); None once the kernel has changed
-ENCODE_DRAM_BYTES_PER_COORDINATE = None
+ENCODE_DRAM_BYTES_PER_COORDINATE = 4.889
+# executed thread instructions of k_exchange_encode per coordinate (ncu, same capture); None once the kernel has changed
+ENCODE_INSTRUCTIONS_PER_COORDINATE = 68.7
 
 def exchange_bytes(K, d, nb, stream_words):
     """Algorithmic bytes of one exchange: read V, write + read the streams and their length words, write the mean."""
@@ -201,14 +203,23 @@ def run_ours(args):
     enc_ms = ms_enc / max(n_enc, 1)
     achieved = enc_bytes / (enc_ms * 1e-3) / 1e9 if n_enc else None
     # DRAM bytes per launch of that kernel: counted by ncu on a smaller case of the same kernel (see
-    # profiles/exchange_kernels_K8_d16M.txt: 656.5 MB read + written for K * d = 2^27 coordinates) and scaled by
+    # profiles/exchange_kernels_K8_d16M.txt: 656.2 MB read + written for K * d = 2^27 coordinates) and scaled by
     # the coordinates of a launch, which the traffic is proportional to.  Set to None when the kernel changes.
     traffic = args.traffic_bytes
     if traffic is None and ENCODE_DRAM_BYTES_PER_COORDINATE is not None:
         traffic = ENCODE_DRAM_BYTES_PER_COORDINATE * K * d
+    # The same kernel against the issue ceiling that actually binds it: executed thread instructions per second
+    # (ncu's count per coordinate x coordinates per launch / the event time) over 148 SMs x 128 lanes x the SM clock
+    # seen during the timed region.
+    alu = None
+    if n_enc and ENCODE_INSTRUCTIONS_PER_COORDINATE is not None:
+        sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        alu_peak = 148 * 128 * sm_mhz * 1e6 / 1e12
+        alu_ach = ENCODE_INSTRUCTIONS_PER_COORDINATE * K * d / (enc_ms * 1e-3) / 1e12
+        alu = {"achieved": alu_ach, "peak": alu_peak, "unit": "T thread-instructions/s", "frac": alu_ach / alu_peak}
     roofline = {"bound": "hbm", "kernel": "k_exchange_encode", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None, "peak_kind": "of " + peak_kind,
-                "traffic": traffic, "ms_per_launch": enc_ms,
+                "traffic": traffic, "ms_per_launch": enc_ms, "alu": alu,
                 "kernels_ms_per_step": {"encode": ms_enc / args.steps, "decode": ms_dec / args.steps,
                                         "histogram": ms_his / args.steps, "operator": ms_op / args.steps,
                                         "finish": ms_fin / args.steps}}
