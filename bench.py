@@ -379,7 +379,7 @@ def main():
     ap.add_argument("--subblock", type=int, default=64)
     ap.add_argument("--refit-every", type=int, default=10)
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-buckets", type=int, default=16, help="buckets per worker in the timed oracle sample")
+    ap.add_argument("--cpu-buckets", type=int, default=320, help="buckets per worker in the timed oracle sample")
     ap.add_argument("--ref-buckets", type=int, default=2, help="buckets per worker per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic-bytes", type=float, default=None,
