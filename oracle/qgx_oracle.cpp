@@ -861,27 +861,36 @@ int qgxo_refit(const float* V, int K, uint64_t d, int bucket, int norm_type, int
 // Exchange ids 2t and 2t+1 key the two independent quantizer draws.
 // refit: 0 none, 1 refit from the current levels, 2 first fit (quantile start).
 // Optional outputs (may be null): the two means and the two sets of decoded vectors.
-int qgxo_eg_step(qgxo_eg_state* st, const qgxo_operator* op, const float* noise_t, const float* noise_half,
-                 int bucket, int norm_type, float* lev, int nlev, qgxo_codebook* cb,
-                 uint64_t seed, int quantizer_off, int refit, int code_type, int nbins, uint64_t* bits_out) {
+// The iteration with its own level table and code for each of the two exchanges (footnote of Sec. 3.3: one
+// sequence of adaptive levels for the V_{k,t} and another one for the V_{k,t+1/2}); lev_t == lev_h and cb_t == cb_h
+// give the single-table iteration.  At an update step each table is refitted on its own dual vectors.
+static int eg_step_core(qgxo_eg_state* st, const qgxo_operator* op, const float* noise_t, const float* noise_half,
+                        int bucket, int norm_type, float* lev_t, int nlev_t, qgxo_codebook* cb_t,
+                        float* lev_h, int nlev_h, qgxo_codebook* cb_h,
+                        uint64_t seed, int quantizer_off, int refit, int code_type, int nbins, uint64_t* bits_out) {
   const uint64_t d = st->d; const int K = st->K;
+  const bool two = (lev_h != lev_t) || (cb_h != cb_t);
   std::vector<float> a(d), V((uint64_t)K * d), vhat1((uint64_t)K * d), vhat2((uint64_t)K * d), mean(d);
   std::vector<uint64_t> tb1(K), tb2(K);
   int rc = qgxo_apply_operator(op, st->X, a.data());
   if (rc) return rc;
   form_by_model(op, a.data(), noise_t, K, d, V.data());
   if (refit && !quantizer_off) {
-    rc = qgxo_refit(V.data(), K, d, bucket, norm_type, nbins, refit == 2, code_type, lev, nlev, cb, nullptr);
+    rc = qgxo_refit(V.data(), K, d, bucket, norm_type, nbins, refit == 2, code_type, lev_t, nlev_t, cb_t, nullptr);
     if (rc) return rc;
   }
-  rc = qgxo_exchange_full(V.data(), K, d, bucket, norm_type, lev, nlev, cb, seed, 2u * (uint32_t)st->t,
+  rc = qgxo_exchange_full(V.data(), K, d, bucket, norm_type, lev_t, nlev_t, cb_t, seed, 2u * (uint32_t)st->t,
                           quantizer_off, vhat1.data(), mean.data(), tb1.data());
   if (rc) return rc;
   for (uint64_t i = 0; i < d; ++i) { const float step = st->gamma * mean[i]; st->Xhalf[i] = st->X[i] - step; }
   rc = qgxo_apply_operator(op, st->Xhalf, a.data());
   if (rc) return rc;
   form_by_model(op, a.data(), noise_half, K, d, V.data());
-  rc = qgxo_exchange_full(V.data(), K, d, bucket, norm_type, lev, nlev, cb, seed, 2u * (uint32_t)st->t + 1u,
+  if (two && refit && !quantizer_off) {
+    rc = qgxo_refit(V.data(), K, d, bucket, norm_type, nbins, refit == 2, code_type, lev_h, nlev_h, cb_h, nullptr);
+    if (rc) return rc;
+  }
+  rc = qgxo_exchange_full(V.data(), K, d, bucket, norm_type, lev_h, nlev_h, cb_h, seed, 2u * (uint32_t)st->t + 1u,
                           quantizer_off, vhat2.data(), mean.data(), tb2.data());
   if (rc) return rc;
   for (uint64_t i = 0; i < d; ++i) st->Y[i] = st->Y[i] - mean[i];
@@ -899,6 +908,22 @@ int qgxo_eg_step(qgxo_eg_state* st, const qgxo_operator* op, const float* noise_
   st->t += 1;
   if (bits_out) { uint64_t b = 0; for (int k = 0; k < K; ++k) b += tb1[k] + tb2[k]; *bits_out = b; }
   return OK;
+}
+
+int qgxo_eg_step(qgxo_eg_state* st, const qgxo_operator* op, const float* noise_t, const float* noise_half,
+                 int bucket, int norm_type, float* lev, int nlev, qgxo_codebook* cb,
+                 uint64_t seed, int quantizer_off, int refit, int code_type, int nbins, uint64_t* bits_out) {
+  return eg_step_core(st, op, noise_t, noise_half, bucket, norm_type, lev, nlev, cb, lev, nlev, cb, seed, quantizer_off,
+                      refit, code_type, nbins, bits_out);
+}
+
+int qgxo_eg_step_two_tables(qgxo_eg_state* st, const qgxo_operator* op, const float* noise_t, const float* noise_half,
+                            int bucket, int norm_type, float* lev_t, int nlev_t, qgxo_codebook* cb_t,
+                            float* lev_h, int nlev_h, qgxo_codebook* cb_h,
+                            uint64_t seed, int quantizer_off, int refit, int code_type, int nbins, uint64_t* bits_out) {
+  if (lev_t == lev_h || cb_t == cb_h) return INVALID_ARG;
+  return eg_step_core(st, op, noise_t, noise_half, bucket, norm_type, lev_t, nlev_t, cb_t, lev_h, nlev_h, cb_h, seed,
+                      quantizer_off, refit, code_type, nbins, bits_out);
 }
 
 // The two other members of the family named in Sec. 3.1, one oracle call and one exchange per iteration.

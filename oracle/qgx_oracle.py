@@ -392,6 +392,22 @@ def eg_step(state, op, noise_t, noise_half, bucket, levels, cb, seed, norm_type=
     return bits.value
 
 
+def eg_step_two_tables(state, op, noise_t, noise_half, bucket, levels_t, cb_t, levels_h, cb_h, seed, norm_type=L2,
+                       quantizer_off=False, refit=0, code_type=CODE_FIXED, nbins=1024):
+    """One iteration with a level table and code of its own for each of the two exchanges; both are updated in place
+    when refit != 0. Returns bits sent."""
+    n1 = _f32(noise_t) if noise_t is not None else None
+    n2 = _f32(noise_half) if noise_half is not None else None
+    for lv in (levels_t, levels_h):
+        assert lv.dtype == np.float32 and lv.flags.c_contiguous
+    bits = C.c_uint64(0)
+    _chk(lib().qgxo_eg_step_two_tables(C.byref(state.c), C.byref(op.c), _p(n1), _p(n2), bucket, norm_type,
+                                       _p(levels_t), len(levels_t), C.byref(cb_t), _p(levels_h), len(levels_h),
+                                       C.byref(cb_h), C.c_uint64(seed), int(quantizer_off), int(refit), int(code_type),
+                                       int(nbins), C.byref(bits)), "eg_step_two_tables")
+    return bits.value
+
+
 METHOD_DE, METHOD_DA, METHOD_OPTDA = 0, 1, 2
 
 

@@ -325,3 +325,42 @@ def test_relative_noise_special_cases():
         o.eg_step(a, o.Op(o.OP_DIAGONAL, D, noise_model=o.NOISE_RELATIVE), ones, ones, 32, lev, cb, 9)
         o.eg_step(b, o.Op(o.OP_DIAGONAL, D), None, None, 32, lev, cb, 9)
     assert np.array_equal(a.X, b.X) and a.sum_sq == b.sum_sq
+
+
+# ---- a level table of its own for each exchange (footnote of Sec. 3.3) ----
+
+def test_two_level_tables():
+    d, K, bucket = 1536, 4, 256
+    D = gen.uniform((d,), 31, "cpu", 0.05, 1.0).numpy()
+    x0 = gen.gaussian((d,), 32, "cpu").numpy()
+    op = o.Op(o.OP_DIAGONAL, D)
+    n_t = gen.gaussian((K, d), 33, "cpu", std=0.2).numpy()
+    n_h = gen.student_t3((K, d), 34, "cpu").numpy() * np.float32(0.3)          # heavier tails at the half step
+    lev0 = gen.uniform_levels(17).numpy()
+    # equal tables, no refit: the single-table iteration, bit for bit
+    a, b = o.EgState(x0, K), o.EgState(x0, K)
+    la, lb, lc = lev0.copy(), lev0.copy(), lev0.copy()
+    ca, cb_, cc = o.codebook_fixed(17, 32), o.codebook_fixed(17, 32), o.codebook_fixed(17, 32)
+    for _ in range(2):
+        bits_a = o.eg_step(a, op, n_t, n_h, bucket, la, ca, 3)
+        bits_b = o.eg_step_two_tables(b, op, n_t, n_h, bucket, lb, cb_, lc, cc, 3)
+        assert bits_a == bits_b and np.array_equal(a.X, b.X) and a.sum_sq == b.sum_sq and np.array_equal(a.Xbar, b.Xbar)
+    # a refit fits each table to its own dual vectors: the pinned refit applied to V_t and to V_{t+1/2}
+    st = o.EgState(x0, K)
+    lt, lh = lev0.copy(), lev0.copy()
+    ct, ch = o.codebook_fixed(17, 32), o.codebook_fixed(17, 32)
+    V_t = o.form_dual_vectors(o.apply_operator(op, st.X), n_t, K)
+    lt_ref, hist_t = o.refit(V_t, bucket, 256, lev0.copy(), o.codebook_fixed(17, 32), True, o.CODE_HUFFMAN)
+    o.eg_step_two_tables(st, op, n_t, n_h, bucket, lt, ct, lh, ch, 3, refit=2, code_type=o.CODE_HUFFMAN, nbins=256)
+    assert np.array_equal(lt, lt_ref)
+    V_h = o.form_dual_vectors(o.apply_operator(op, st.Xhalf), n_h, K)
+    lh_ref, hist_h = o.refit(V_h, bucket, 256, lev0.copy(), o.codebook_fixed(17, 32), True, o.CODE_HUFFMAN)
+    assert np.array_equal(lh, lh_ref) and not np.array_equal(lt, lh)
+    # what the second table is for: on the half-step vectors it has the smaller quantization variance (QAda objective)
+    assert o.objective(hist_h, lh) < o.objective(hist_h, lt)
+    assert o.objective(hist_t, lt) < o.objective(hist_t, lh)
+    # and the realised error of the second exchange is smaller with its own table (same draws)
+    def err(levels, cbk):
+        _, _, vhat = o.exchange(V_h, bucket, levels, cbk, 3, 3, return_vhat=True)
+        return float(np.sum((vhat.astype(np.float64) - V_h) ** 2))
+    assert err(lh, ch) < err(lt, ct)
