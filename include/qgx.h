@@ -275,6 +275,14 @@ qgx_status qgx_eg_init(qgx_ctx *ctx, qgx_eg_state *st /*[host]*/);
 qgx_status qgx_eg_step(qgx_ctx *ctx, qgx_eg_state *st, const qgx_operator *op,
                        const float *noise_t, const float *noise_half, qgx_quant_cfg *cfg,
                        int refit, uint64_t *bits);
+/* qgx_eg_step with a level table and a code of its own for each exchange (the finer scheme that the footnote
+ * of Sec. 3.3 describes: one sequence of adaptive levels for the V_{k,t}, another for the V_{k,t+1/2}).  The first
+ * exchange uses cfg_t, the second cfg_half; when refit != 0 each is refitted on its own dual vectors (one more
+ * histogram pass).  Both must have the same bucket and sub-block sizes; the seeds may differ.  The squared
+ * differences compare vectors dequantized with their own tables. */
+qgx_status qgx_eg_step_two_tables(qgx_ctx *ctx, qgx_eg_state *st, const qgx_operator *op,
+                                  const float *noise_t, const float *noise_half, qgx_quant_cfg *cfg_t,
+                                  qgx_quant_cfg *cfg_half, int refit, uint64_t *bits);
 /* The other two members of the family that Sec. 3.1 lists (Eq. Quantized DA, Eq. Quantized OptDA): one
  * oracle call and one exchange per iteration, same state, same step-size rule.
  *   QGX_METHOD_DA:    Vhat_{k,t} = 0, so X_{t+1/2} = X_t;  g_k = Q(A(X_t) + U_k);  Y_{t+1} = Y_t - mean_k g_k;

@@ -28,7 +28,7 @@ EXPORTS = [
     "qgx_build_codebook_huffman", "qgx_fit_levels", "qgx_symbol_pmf",
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
-    "qgx_eg_init", "qgx_eg_step", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
+    "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
     "qgx_encode_noalloc", "qgx_exchange_segments",
 ]
 QGX_KERNEL_ENCODE, QGX_KERNEL_DECODE, QGX_KERNEL_HISTOGRAM, QGX_KERNEL_OPERATOR, QGX_KERNEL_FINISH = range(5)
@@ -400,6 +400,11 @@ def qgx_eg_init(ctx, state):
 def qgx_eg_step(ctx, state, op, noise_t, noise_half, cfg, refit=QGX_REFIT_NONE, bits=None):
     _chk(lib().qgx_eg_step(ctx.h, C.byref(state.c), C.byref(op), _ptr(noise_t), _ptr(noise_half), C.byref(cfg),
                            refit, _ptr(bits)), "qgx_eg_step")
+
+
+def qgx_eg_step_two_tables(ctx, state, op, noise_t, noise_half, cfg_t, cfg_half, refit=QGX_REFIT_NONE, bits=None):
+    _chk(lib().qgx_eg_step_two_tables(ctx.h, C.byref(state.c), C.byref(op), _ptr(noise_t), _ptr(noise_half),
+                                      C.byref(cfg_t), C.byref(cfg_half), refit, _ptr(bits)), "qgx_eg_step_two_tables")
 
 
 QGX_METHOD_DE, QGX_METHOD_DA, QGX_METHOD_OPTDA = 0, 1, 2

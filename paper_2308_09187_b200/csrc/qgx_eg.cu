@@ -149,9 +149,11 @@ qgx_status qgx_eg_init(qgx_ctx* c, qgx_eg_state* st) {
   return cuda_status(cudaGetLastError());
 }
 
-qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, const float* noise_t, const float* noise_half,
-                       qgx_quant_cfg* cfg, int refit, uint64_t* bits) {
-  if (!c || !st || !op || !cfg || !st->X || !st->Y || !st->Xbar || !st->Xhalf || !st->anchor || !st->scalars || st->t < 1 ||
+// cfg_half == cfg: one level table and code for both exchanges; otherwise each exchange has its own, refitted on
+// its own dual vectors
+static qgx_status eg_step_impl(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, const float* noise_t, const float* noise_half,
+                               qgx_quant_cfg* cfg, qgx_quant_cfg* cfg_half, int refit, uint64_t* bits) {
+  if (!c || !st || !op || !cfg || !cfg_half || !st->X || !st->Y || !st->Xbar || !st->Xhalf || !st->anchor || !st->scalars || st->t < 1 ||
       op->d != st->d || st->K < 1)
     return QGX_ERR_INVALID_ARG;
   if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
@@ -178,8 +180,14 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
   rc = apply_operator_impl(c, op, st->Xhalf, a);                              // A(X_{t+1/2})
   if (rc != QGX_OK) return rc;
   DualSource src2{noise_half, a, 0, mul};
+  if (cfg_half != cfg && refit != QGX_REFIT_NONE) {
+    double* hist = (double*)ws_get(c, WS_HIST, sizeof(double) * (size_t)std::max(cfg_half->nbins, 1));
+    if (!hist) return QGX_ERR_CUDA;
+    rc = refit_from_source(c, src2, K, d, cfg_half, refit, hist, nullptr);
+    if (rc != QGX_OK) return rc;
+  }
   ExchangeUpdate dual{2, st->Y, st->Y, st->scalars};                          // Y_{t+1} = Y_t - mean
-  rc = exchange_impl(c, src2, K, d, cfg, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 2, st->scalars, 0);
+  rc = exchange_impl(c, src2, K, d, cfg_half, xid + 1u, 1, mean, bits ? bits + K : nullptr, &dual, 2, st->scalars, 0);
   if (rc != QGX_OK) return rc;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);
@@ -188,6 +196,21 @@ qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, con
   count_launch(c);
   st->t += 1;
   return cuda_status(cudaGetLastError());
+}
+
+qgx_status qgx_eg_step(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, const float* noise_t, const float* noise_half,
+                       qgx_quant_cfg* cfg, int refit, uint64_t* bits) {
+  return eg_step_impl(c, st, op, noise_t, noise_half, cfg, cfg, refit, bits);
+}
+
+qgx_status qgx_eg_step_two_tables(qgx_ctx* c, qgx_eg_state* st, const qgx_operator* op, const float* noise_t,
+                                  const float* noise_half, qgx_quant_cfg* cfg_t, qgx_quant_cfg* cfg_half, int refit,
+                                  uint64_t* bits) {
+  if (!cfg_t || !cfg_half || cfg_t == cfg_half) return QGX_ERR_INVALID_ARG;
+  // the decode pass compares sub-block by sub-block: both exchanges need the same bucket and sub-block sizes
+  if (cfg_t->bucket != cfg_half->bucket || eff_subblock(cfg_t->bucket, cfg_t->cb.subblock) != eff_subblock(cfg_half->bucket, cfg_half->cb.subblock))
+    return QGX_ERR_INVALID_ARG;
+  return eg_step_impl(c, st, op, noise_t, noise_half, cfg_t, cfg_half, refit, bits);
 }
 
 qgx_status qgx_family_step(qgx_ctx* c, qgx_eg_state* st, int method, const qgx_operator* op, const float* noise,

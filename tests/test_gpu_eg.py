@@ -274,3 +274,44 @@ def test_relative_noise_iteration(q):
     qgx.qgx_sync_status(ctx)
     s, g = st3.read_scalars()
     assert not st3.X.any().item() and s == 0.0 and g == K
+
+
+def test_two_level_tables(q):
+    """A level table and a code of its own for each exchange (footnote of Sec. 3.3): teacher forced against the
+    oracle with refits, the second exchange on heavier-tailed vectors than the first."""
+    qgx, ctx = q
+    K, d, bucket, sub = 4, 2 * 2048 + 500, 2048, 64
+    D = gen.uniform((d,), 31, "cuda", 0.05, 1.0)
+    x0 = gen.gaussian((d,), 32, "cuda")
+    n_t = gen.gaussian((K, d), 33, "cuda", std=0.2)
+    n_h = gen.student_t3((K, d), 34, "cuda") * 0.3
+    op, opo = qgx.make_operator(qgx.QGX_OP_DIAGONAL, D), o.Op(o.OP_DIAGONAL, D.cpu().numpy())
+    lev0 = gen.uniform_levels(17).numpy()
+    cfg_t = qgx.make_quant_cfg(lev0, bucket, qgx.qgx_build_codebook_fixed(17, sub), 8, code_type=qgx.QGX_CODE_HUFFMAN, nbins=512)
+    cfg_h = qgx.make_quant_cfg(lev0, bucket, qgx.qgx_build_codebook_fixed(17, sub), 8, code_type=qgx.QGX_CODE_HUFFMAN, nbins=512)
+    st, st_o = qgx.EgState(x0, K), o.EgState(x0.cpu().numpy(), K)
+    qgx.qgx_eg_init(ctx, st)
+    lt, lh = lev0.copy(), lev0.copy()
+    ct, ch = o.codebook_fixed(17, sub), o.codebook_fixed(17, sub)
+    nth, nhh = n_t.cpu().numpy(), n_h.cpu().numpy()
+    for t in range(1, 6):
+        refit = 2 if t == 1 else (1 if t == 4 else 0)
+        _load_state(qgx, st, st_o)
+        qgx.qgx_eg_step_two_tables(ctx, st, op, n_t, n_h, cfg_t, cfg_h, refit=refit)
+        qgx.qgx_sync_status(ctx)
+        if refit:
+            # both sides quantize with the library's tables and codes (the fits themselves are compared below)
+            got_t, got_h = np.array(cfg_t.level_list(), np.float32), np.array(cfg_h.level_list(), np.float32)
+            lt_o, lh_o = lt.copy(), lh.copy()
+            probe = o.EgState(st_o.X.copy(), K)
+            probe.load(st_o.X, st_o.Y, st_o.Xbar, st_o.sum_sq, st_o.gamma, st_o.t)
+            o.eg_step_two_tables(probe, opo, nth, nhh, bucket, lt_o, o.codebook_fixed(17, sub), lh_o, o.codebook_fixed(17, sub),
+                                 8, refit=refit, code_type=o.CODE_HUFFMAN, nbins=512)
+            if refit == 2:
+                assert np.max(np.abs(got_t - lt_o)) < 5e-5 and np.max(np.abs(got_h - lh_o)) < 5e-5
+            assert not np.array_equal(got_t, got_h)
+            lt, lh = got_t.copy(), got_h.copy()
+            ct = o.codebook_from(cfg_t.cb.lengths(), cfg_t.cb.codes(), subblock=sub)
+            ch = o.codebook_from(cfg_h.cb.lengths(), cfg_h.cb.codes(), subblock=sub)
+        o.eg_step_two_tables(st_o, opo, nth, nhh, bucket, lt, ct, lh, ch, 8)
+        _compare(st, st_o, tol=1e-6)
