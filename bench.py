@@ -36,9 +36,9 @@ WORKLOAD = "c5-scale: K=32, d=2^26, mixture noise, diagonal operator, bucket 163
 
 
 # measured DRAM traffic of k_exchange_encode per coordinate (ncu, current kernel); None once the kernel has changed
-ENCODE_DRAM_BYTES_PER_COORDINATE = 4.889
+ENCODE_DRAM_BYTES_PER_COORDINATE = None
 # executed thread instructions of k_exchange_encode per coordinate (ncu, same capture); None once the kernel has changed
-ENCODE_INSTRUCTIONS_PER_COORDINATE = 68.7
+ENCODE_INSTRUCTIONS_PER_COORDINATE = None
 
 def exchange_bytes(K, d, nb, stream_words):
     """Algorithmic bytes of one exchange: read V, write + read the streams and their length words, write the mean."""

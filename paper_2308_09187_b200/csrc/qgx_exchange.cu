@@ -119,6 +119,25 @@ __device__ __forceinline__ void load_bucket_octets(BucketRegs<2 * P>& r, const D
                                                    size_t lo, int len, bool vec_ok) {
   const size_t ld = s.ld ? s.ld : d;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (vec_ok && len == 256 * P * (int)(blockDim.x >> 5)) {
+    // every lane holds full octets: the kind of source is decided once, not per quad
+    const float4* pv = s.v ? reinterpret_cast<const float4*>(s.v + k * ld + lo) + ((warp * P * 32 + lane) << 1) : nullptr;
+    const float4* pa = s.a ? reinterpret_cast<const float4*>(s.a + lo) + ((warp * P * 32 + lane) << 1) : nullptr;
+    if (pa == nullptr) {
+#pragma unroll
+      for (int j = 0; j < 2 * P; ++j) r.x[j] = __ldcs(pv + (j >> 1) * 64 + (j & 1));
+    } else if (pv == nullptr) {
+#pragma unroll
+      for (int j = 0; j < 2 * P; ++j) r.x[j] = __ldg(pa + (j >> 1) * 64 + (j & 1));
+    } else if (s.mul) {
+#pragma unroll
+      for (int j = 0; j < 2 * P; ++j) r.x[j] = dual_combine(__ldg(pa + (j >> 1) * 64 + (j & 1)), __ldcs(pv + (j >> 1) * 64 + (j & 1)), 1);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 2 * P; ++j) r.x[j] = dual_combine(__ldg(pa + (j >> 1) * 64 + (j & 1)), __ldcs(pv + (j >> 1) * 64 + (j & 1)), 0);
+    }
+    return;
+  }
 #pragma unroll
   for (int j = 0; j < 2 * P; ++j) {
     const int e = ((((warp * P + (j >> 1)) * 32 + lane) << 1) + (j & 1)) * kQuad;
@@ -216,6 +235,21 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
 
     uint64_t qbits[2 * P];
     uint32_t qn[P], qoff[P];                              // qn: bits of the first quad | bits of the second << 8
+    if (whole && live) {                                  // the common case, without per-quad decisions
+#pragma unroll
+      for (int j = 0; j < P; ++j) {
+        const int o = (warp * P + j) * 32 + lane;
+        const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + 2ull * (uint64_t)o;
+        uint4 w0, w1;
+        philox4x32_10_x2(ctr, ctr + 1ull, (uint32_t)k, a.xid, key, &w0, &w1);
+        const uint32_t code0 = quantize_quad_codes(r.x[2 * j], w0, rc, norm, s_bin, s_lev, nlev);
+        const uint32_t code1 = quantize_quad_codes(r.x[2 * j + 1], w1, rc, norm, s_bin, s_lev, nlev);
+        uint32_t n0, n1;
+        pack_quad_codes(code0, s_pair, &qbits[2 * j], &n0);
+        pack_quad_codes(code1, s_pair, &qbits[2 * j + 1], &n1);
+        qn[j] = n0 | (n1 << 8);
+      }
+    } else {
 #pragma unroll
     for (int j = 0; j < P; ++j) {
       const int o = (warp * P + j) * 32 + lane;           // octet of the bucket
@@ -238,6 +272,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
         pack_quad((code1 & 0x1f1f1f1fu) | ((code1 & 0x20202020u) << 2), nv1, &s_lut, &qbits[2 * j + 1], &n1);
       }
       qn[j] = n0 | (n1 << 8);
+    }
     }
     // warp scans of the bit counts, two rows per 32-bit word (a row holds at most 32 * 104 bits);
     // qoff[j] becomes the octet's bit offset inside the warp's part of the payload
