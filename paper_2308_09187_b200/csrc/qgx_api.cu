@@ -160,6 +160,7 @@ void qgx_destroy(qgx_ctx* c) {
   cudaSetDevice(c->device);
   cudaStreamSynchronize(c->stream);
   if (c->timing_ev) timing_free(c);
+  free_table_cache(c);
   for (int i = 0; i < 24; ++i)
     if (c->ws[i]) cudaFree(c->ws[i]);
   cudaFree(c->dstatus);

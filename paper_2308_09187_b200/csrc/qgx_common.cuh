@@ -42,6 +42,9 @@ struct qgx_ctx {
   size_t sym_ld;                         // bytes per worker in the kept-symbol layout
   int sym_nlev;                          // the level table those symbols were quantized with
   float sym_levels[QGX_MAX_LEVELS];
+  // host-side cache of the fused calls: tables derived from a quantizer configuration (with their device copies)
+  // and launch shapes; owned by qgx_exchange.cu
+  void* table_cache;
   // optional per-kernel timing: pairs of events recorded around instrumented launches
   int timing_on;
   int timing_cap;                        // pairs allocated
@@ -292,6 +295,7 @@ qgx_status check_levels_host(const float* lev, int nlev);
 qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out);
 void make_round_table(const float* lev, int nlev, RoundTable* out);
 void* ws_get(qgx_ctx* c, int which, size_t bytes);          // nullptr on failure
+void free_table_cache(qgx_ctx* c);
 qgx_status cuda_status(cudaError_t e);
 inline void count_launch(qgx_ctx* c, int n = 1) { c->launches += (uint64_t)n; }
 

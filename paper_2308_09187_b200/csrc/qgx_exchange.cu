@@ -5,6 +5,8 @@
 #include "qgx_codec.cuh"
 
 #include <algorithm>
+#include <cstring>
+#include <new>
 #include <vector>
 
 namespace qgx {
@@ -713,6 +715,96 @@ __global__ void k_add_u64(uint64_t* acc, const uint64_t* x, int n) {
 
 qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct, const LevelTable& lt, int sym_mode);
 
+// ---- what a call derives from a quantizer configuration, kept between calls --------------------
+// Building the rounding table, the code table and the decoder table and copying the latter to the device costs
+// more host time than a small exchange; iterations reuse a handful of configurations, so the results are kept,
+// keyed by the configuration's contents (compared in full on a hit).
+struct CachedTables {
+  bool valid;
+  int nlev, bucket;
+  float levels[QGX_MAX_LEVELS];
+  qgx_codebook cb;
+  CodeTable ct;
+  RoundTable rt;
+  DecEntry* lut_dev;                    // 2 * kDecLutMax entries, owned
+};
+constexpr int kTableCacheSlots = 32;
+struct LaunchShape { size_t smem; int per_sm; };      // smem == 0: not asked yet
+struct TableCache {
+  CachedTables e[kTableCacheSlots];
+  LaunchShape enc[3][3];                // [octets per thread 1, 2, 4][sub-block 32, 64, 128]
+  LaunchShape dec[3][6];                // [sub-block][symbol mode]
+};
+
+void free_table_cache(qgx_ctx* c) {
+  TableCache* tc = (TableCache*)c->table_cache;
+  if (!tc) return;
+  for (int i = 0; i < kTableCacheSlots; ++i)
+    if (tc->e[i].lut_dev) cudaFree(tc->e[i].lut_dev);
+  delete tc;
+  c->table_cache = nullptr;
+}
+
+static TableCache* table_cache(qgx_ctx* c) {
+  if (!c->table_cache) c->table_cache = new (std::nothrow) TableCache();   // value-initialized: all zero
+  return (TableCache*)c->table_cache;
+}
+
+// tables of cfg (built, and the decoder table copied to the device, on a miss)
+static qgx_status cached_tables(qgx_ctx* c, const qgx_quant_cfg* cfg, const CachedTables** out) {
+  TableCache* tc = table_cache(c);
+  if (!tc) return QGX_ERR_CUDA;
+  uint64_t h = 1469598103934665603ull;
+  auto mix = [&](const void* p, size_t n) {
+    const unsigned char* b = (const unsigned char*)p;
+    for (size_t i = 0; i < n; ++i) { h ^= b[i]; h *= 1099511628211ull; }
+  };
+  mix(&cfg->nlev, sizeof(int)); mix(&cfg->bucket, sizeof(int)); mix(cfg->levels, sizeof(float) * (size_t)cfg->nlev);
+  mix(&cfg->cb.subblock, sizeof(int)); mix(cfg->cb.len, (size_t)cfg->nlev); mix(cfg->cb.code, sizeof(uint32_t) * (size_t)cfg->nlev);
+  CachedTables* e = &tc->e[h % kTableCacheSlots];
+  const bool hit = e->valid && e->nlev == cfg->nlev && e->bucket == cfg->bucket && e->cb.nlev == cfg->cb.nlev &&
+                   e->cb.subblock == cfg->cb.subblock &&
+                   std::memcmp(e->levels, cfg->levels, sizeof(float) * (size_t)cfg->nlev) == 0 &&
+                   std::memcmp(e->cb.len, cfg->cb.len, (size_t)cfg->nlev) == 0 &&
+                   std::memcmp(e->cb.code, cfg->cb.code, sizeof(uint32_t) * (size_t)cfg->nlev) == 0;
+  if (!hit) {
+    e->valid = false;
+    qgx_status rc = make_code_table(&cfg->cb, cfg->bucket, &e->ct);
+    if (rc != QGX_OK) return rc;
+    make_round_table(cfg->levels, cfg->nlev, &e->rt);
+    if (!e->lut_dev && cudaMalloc((void**)&e->lut_dev, sizeof(DecEntry) * (size_t)(2 * kDecLutMax)) != cudaSuccess) {
+      cudaGetLastError();
+      e->lut_dev = nullptr;
+      return QGX_ERR_CUDA;
+    }
+    // decoder table: the next maxlen + 1 bits -> signed level value and bits consumed
+    const CodeTable& ct = e->ct;
+    std::vector<uint16_t> by_code((size_t)1 << ct.maxlen);
+    build_dec_lut_host(ct, by_code.data());
+    std::vector<DecEntry> h_lut((size_t)2 << ct.maxlen);
+    for (size_t i = 0; i < h_lut.size(); ++i) {
+      const uint16_t w = by_code[i & (((size_t)1 << ct.maxlen) - 1)];
+      const uint32_t L = w >> 8, idx = w & 0xffu;
+      if (L == 0) { h_lut[i].val = 0.0f; h_lut[i].len = 1u | 0x80u; continue; }
+      if (idx == 0) { h_lut[i].val = 0.0f; h_lut[i].len = L; continue; }       // symbol byte 0
+      const bool neg = (i >> L) & 1u;
+      h_lut[i].val = neg ? -cfg->levels[idx] : cfg->levels[idx];
+      h_lut[i].len = (L + 1u) | ((idx | (neg ? 0x80u : 0u)) << 8);       // bits 8..15: the symbol byte
+    }
+    // stream-ordered after the kernels that still read this slot's previous table; the source is pageable, so
+    // the call returns once it has been staged
+    if (cudaMemcpyAsync(e->lut_dev, h_lut.data(), h_lut.size() * sizeof(DecEntry), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+      return QGX_ERR_CUDA;
+    e->nlev = cfg->nlev;
+    e->bucket = cfg->bucket;
+    std::memcpy(e->levels, cfg->levels, sizeof(e->levels));
+    e->cb = cfg->cb;
+    e->valid = true;
+  }
+  *out = e;
+  return QGX_OK;
+}
+
 // The whole exchange.  sym_mode 1 keeps the decoded symbols (and the norms) in the workspace; sym_mode 2
 // adds sum_k ||vhat_k kept by the other slot - vhat_k decoded in this exchange||^2 to *sum_sq.
 qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
@@ -725,10 +817,11 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   if (cfg->norm_type != QGX_NORM_L2 && cfg->norm_type != QGX_NORM_LINF) return QGX_ERR_INVALID_ARG;
   if (check_levels_host(cfg->levels, cfg->nlev) != QGX_OK) return QGX_ERR_BAD_LEVELS;
   if (cfg->cb.nlev != cfg->nlev) return QGX_ERR_INVALID_ARG;
-  CodeTable ct;
-  qgx_status rc = make_code_table(&cfg->cb, bucket, &ct);
-  if (rc != QGX_OK) return rc;
   if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
+  const CachedTables* tables = nullptr;
+  qgx_status rc = cached_tables(c, cfg, &tables);
+  if (rc != QGX_OK) return rc;
+  const CodeTable& ct = tables->ct;
   LevelTable lt;
   lt.nlev = cfg->nlev;
   for (int j = 0; j < QGX_MAX_LEVELS; ++j) lt.lev[j] = j < cfg->nlev ? cfg->levels[j] : 1.0f;
@@ -742,7 +835,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   unsigned long long* tot = (unsigned long long*)ws_get(c, base + 3, sizeof(uint64_t) * (size_t)K);
   unsigned long long* status = (unsigned long long*)ws_get(c, WS_STATUS, sizeof(uint64_t) * ((size_t)K * nb + 2));
   float* norms = (float*)ws_get(c, slot == 0 ? WS_NORMS : WS_NORMS2, sizeof(float) * (size_t)K * nb);
-  DecEntry* lut = (DecEntry*)ws_get(c, WS_DLUT, sizeof(DecEntry) * (size_t)(2 * kDecLutMax));
+  const DecEntry* lut = tables->lut_dev;
   if (!stream || !bbits || !offs || !tot || !status || !norms || !lut) return QGX_ERR_CUDA;
   c->slot_cap_words[slot] = cap;
   c->slot_K[slot] = K;
@@ -779,8 +872,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
     for (int j = 0; j < cfg->nlev; ++j) c->sym_levels[j] = cfg->levels[j];
   }
   const PhiloxKey key = make_philox_key(cfg->seed);
-  RoundTable qt;
-  make_round_table(cfg->levels, cfg->nlev, &qt);
+  const RoundTable& qt = tables->rt;
   if (!ct.has_header || bucket % ct.G != 0 || (ct.G != 32 && ct.G != 64 && ct.G != 128)) return QGX_ERR_INVALID_ARG;
   // octets per thread chosen so that CTAs have at most 256 / 512 / 512 threads
   const int pp = bucket <= 2048 ? 1 : (bucket <= 8192 ? 2 : 4);
@@ -790,9 +882,14 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   int per_sm = 1;
 #define QGX_LAUNCH_E(V, GG)                                                                                    \
   do {                                                                                                         \
-    cudaFuncSetAttribute(k_exchange_encode<V, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG>, threads, smem);           \
-    if (per_sm < 1) per_sm = 1;                                                                                \
+    LaunchShape& shape = table_cache(c)->enc[V == 1 ? 0 : (V == 2 ? 1 : 2)][GG == 32 ? 0 : (GG == 64 ? 1 : 2)];  \
+    if (shape.smem != smem + 1 + (size_t)threads * 0x100000) {   /* asked once per shape, not per call */        \
+      cudaFuncSetAttribute(k_exchange_encode<V, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG>, threads, smem);         \
+      shape.smem = smem + 1 + (size_t)threads * 0x100000;                                                      \
+      shape.per_sm = per_sm < 1 ? 1 : per_sm;                                                                  \
+    }                                                                                                          \
+    per_sm = shape.per_sm;                                                                                     \
     const unsigned long long want = (unsigned long long)nb * (unsigned long long)K;                            \
     const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);   \
     k_exchange_encode<V, GG><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                          \
@@ -819,24 +916,6 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
       cudaMemcpyAsync(total_bits_out, tot, sizeof(uint64_t) * (size_t)K, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
     return QGX_ERR_CUDA;
 
-  // decoder table: the next maxlen + 1 bits -> signed level value and bits consumed
-  {
-    std::vector<uint16_t> by_code((size_t)1 << ct.maxlen);
-    build_dec_lut_host(ct, by_code.data());
-    std::vector<DecEntry> h_lut((size_t)2 << ct.maxlen);
-    for (size_t i = 0; i < h_lut.size(); ++i) {
-      const uint16_t e = by_code[i & (((size_t)1 << ct.maxlen) - 1)];
-      const uint32_t L = e >> 8, idx = e & 0xffu;
-      if (L == 0) { h_lut[i].val = 0.0f; h_lut[i].len = 1u | 0x80u; continue; }
-      if (idx == 0) { h_lut[i].val = 0.0f; h_lut[i].len = L; continue; }       // symbol byte 0
-      const bool neg = (i >> L) & 1u;
-      h_lut[i].val = neg ? -cfg->levels[idx] : cfg->levels[idx];
-      h_lut[i].len = (L + 1u) | ((idx | (neg ? 0x80u : 0u)) << 8);       // bits 8..15: the symbol byte
-    }
-    if (cudaMemcpyAsync(lut, h_lut.data(), h_lut.size() * sizeof(DecEntry), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
-      return QGX_ERR_CUDA;
-  }
-
   DecodeArgs da;
   da.stream = stream; da.cap_words = cap; da.bucket_bits = bbits; da.offsets = offs;
   da.sym_out = sym_out; da.sym_prev = sym_prev; da.sym_ld = sym_ld; da.norms_prev = norms_prev; da.sum_sq = sum_sq;
@@ -856,9 +935,14 @@ static qgx_status launch_decode_gs(qgx_ctx* c, const DecodeArgs& da, const CodeT
   int per_sm = 1;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
-    cudaFuncSetAttribute(k_exchange_decode<G, SYM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lut_bytes);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, SYM>, kDecThreads, lut_bytes);
-    if (per_sm < 1) per_sm = 1;
+    LaunchShape& shape = table_cache(c)->dec[G == 32 ? 0 : (G == 64 ? 1 : 2)][SYM];
+    if (shape.smem != lut_bytes + 1) {                       // asked once per shape, not per call
+      cudaFuncSetAttribute(k_exchange_decode<G, SYM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lut_bytes);
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, SYM>, kDecThreads, lut_bytes);
+      shape.smem = lut_bytes + 1;
+      shape.per_sm = per_sm < 1 ? 1 : per_sm;
+    }
+    per_sm = shape.per_sm;
     const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
     k_exchange_decode<G, SYM><<<grid, kDecThreads, lut_bytes, c->stream>>>(da, ct, lt);
   }
