@@ -236,6 +236,14 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(args, cfg, prob)
 
+    others = None
+    if rank == 0 and world == 1 and not args.no_other_configs:
+        del prob                                      # the scale workload's 17 GB of noise
+        try:
+            others = other_configs(qgx, ctx)
+        except Exception as ex:
+            others = {"error": str(ex)[:200]}
+
     if rank == 0:
         s_val, g_val = st.read_scalars()
         line = {
@@ -251,12 +259,79 @@ def run_ours(args):
             "bits_per_coordinate": sum(total_bits) / (2.0 * K * d),
             "algorithmic_bytes_per_step": bytes_step,
             "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
-            "gamma": g_val, "sum_sq": s_val,
+            "gamma": g_val, "sum_sq": s_val, "other_configs": others,
         }
         print(json.dumps(line))
     qgx.qgx_destroy(ctx)
     if world > 1:
         dist.destroy_process_group()
+
+
+def other_configs(qgx, ctx):
+    """The smaller configurations, timed by the wall clock around a synchronize (they are launch- and
+    latency-bound): supplementary figures, not the headline."""
+    import numpy as np
+    import torch
+    import qgx_inputs as gen
+
+    def timed(fn, n, warm=3):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n):
+            fn()
+        torch.cuda.synchronize()
+        return (time.perf_counter() - t0) / n
+
+    out = {}
+    g = gen.c1_bilinear(T=100, device="cuda")
+    cfg = qgx.make_quant_cfg(gen.uniform_levels(9).numpy(), g.bucket, qgx.qgx_build_codebook_fixed(9, 32), g.seed)
+    op = qgx.make_operator(qgx.QGX_OP_BILINEAR, g.A)
+    st = qgx.EgState(g.z0, g.K)
+    qgx.qgx_eg_init(ctx, st)
+    i = [0]
+
+    def c1_step():
+        t = i[0] % 100
+        i[0] += 1
+        qgx.qgx_eg_step(ctx, st, op, g.noise[t, 0], g.noise[t, 1], cfg)
+    out["c1_bilinear_n1024_K4_iterations_per_s"] = 1.0 / timed(c1_step, 200)
+
+    vi = gen.c4_affine(device="cuda")
+    cfg4 = qgx.make_quant_cfg(gen.uniform_levels(17).numpy(), vi.bucket, qgx.qgx_build_codebook_fixed(17, 32), vi.seed,
+                              code_type=qgx.QGX_CODE_HUFFMAN)
+    op4 = qgx.make_operator(qgx.QGX_OP_DENSE_AFFINE, vi.M, vi.b)
+    st4 = qgx.EgState(vi.x0, vi.K)
+    qgx.qgx_eg_init(ctx, st4)
+    nz = vi.noise(1)
+    qgx.qgx_eg_step(ctx, st4, op4, nz[0], nz[1], cfg4, refit=qgx.QGX_REFIT_FIRST)
+    out["c4_affine_n8192_K8_iterations_per_s"] = 1.0 / timed(lambda: qgx.qgx_eg_step(ctx, st4, op4, nz[0], nz[1], cfg4), 100)
+    del vi, op4, st4
+
+    c2 = gen.c2_gaussian(device="cuda")
+    cfg2 = qgx.make_quant_cfg(np.linspace(0, 1, 17), c2.bucket, qgx.qgx_build_codebook_fixed(17, 64), c2.seed,
+                              code_type=qgx.QGX_CODE_HUFFMAN)
+    qgx.qgx_update_levels(ctx, c2.v, cfg2, qgx.QGX_REFIT_FIRST)
+    K2, d2 = c2.v.shape
+    mean, tot = qgx.qgx_exchange(ctx, c2.v, cfg2, 3, slot=0)
+    sec = timed(lambda: qgx.qgx_exchange(ctx, c2.v, cfg2, 3, slot=0), 20)
+    nb2 = d2 // c2.bucket
+    words = int(((tot.cpu().numpy().astype(np.int64) + 31) // 32).sum()) + K2 * nb2
+    out["c2_exchange_K8_d2p24_GBps"] = exchange_bytes(K2, d2, nb2, words) / sec / 1e9
+    del c2
+
+    lw = gen.c3_layerwise(K=16, device="cuda")
+    cfgs, at = [], 0
+    for n in lw.sizes:
+        c = qgx.make_quant_cfg(np.linspace(0, 1, lw.nlev), lw.bucket, qgx.qgx_build_codebook_fixed(lw.nlev, 32), lw.seed,
+                               code_type=qgx.QGX_CODE_HUFFMAN)
+        qgx.qgx_update_levels(ctx, lw.v[:, at:at + n].contiguous(), c, qgx.QGX_REFIT_FIRST)
+        cfgs.append(c)
+        at += n
+    out["c3_layerwise_16_tensors_K16_ms_per_exchange"] = 1e3 * timed(lambda: qgx.qgx_exchange_segments(ctx, lw.v, lw.sizes, cfgs, 9), 20)
+    qgx.qgx_sync_status(ctx)
+    return out
 
 
 def run_e2e(args, qgx, ctx, st, op, cfg, prob, world, bytes_step):
@@ -382,6 +457,7 @@ def main():
     ap.add_argument("--cpu-buckets", type=int, default=320, help="buckets per worker in the timed oracle sample")
     ap.add_argument("--ref-buckets", type=int, default=2, help="buckets per worker per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the supplementary timings of the smaller configurations")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the dominant kernel from the last ncu capture (null once the kernel changed)")
     args = ap.parse_args()
