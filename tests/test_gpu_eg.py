@@ -315,3 +315,44 @@ def test_two_level_tables(q):
             ch = o.codebook_from(cfg_h.cb.lengths(), cfg_h.cb.codes(), subblock=sub)
         o.eg_step_two_tables(st_o, opo, nth, nhh, bucket, lt, ct, lh, ch, 8)
         _compare(st, st_o, tol=1e-6)
+
+
+def test_argument_errors_of_the_iteration_calls(q):
+    """Wrong arguments come back as error codes; nothing is launched and the context stays usable."""
+    qgx, ctx = q
+    K, d, bucket = 2, 1024, 256
+    D = gen.uniform((d,), 1, "cuda", 0.1, 1.0)
+    x0 = gen.gaussian((d,), 2, "cuda")
+    nz = gen.gaussian((K, d), 3, "cuda")
+    op = qgx.make_operator(qgx.QGX_OP_DIAGONAL, D)
+    cfg = qgx.make_quant_cfg(gen.uniform_levels(9).numpy(), bucket, qgx.qgx_build_codebook_fixed(9, 32), 1)
+    st = qgx.EgState(x0, K)
+    qgx.qgx_eg_init(ctx, st)
+    mean_prev = torch.zeros(d, dtype=torch.float32, device="cuda")
+    with pytest.raises(qgx.QgxError) as e:
+        qgx.qgx_family_step(ctx, st, 7, op, nz, cfg, mean_prev=mean_prev)              # no such method
+    assert e.value.status == qgx.QGX_ERR_INVALID_ARG
+    with pytest.raises(qgx.QgxError) as e:
+        qgx.qgx_family_step(ctx, st, qgx.QGX_METHOD_OPTDA, op, nz, cfg)                # needs mean_prev
+    assert e.value.status == qgx.QGX_ERR_INVALID_ARG
+    with pytest.raises(qgx.QgxError) as e:
+        qgx.qgx_eg_step_two_tables(ctx, st, op, nz, nz, cfg, cfg)                      # one table given twice
+    assert e.value.status == qgx.QGX_ERR_INVALID_ARG
+    other = qgx.make_quant_cfg(gen.uniform_levels(9).numpy(), bucket, qgx.qgx_build_codebook_fixed(9, 64), 1)
+    with pytest.raises(qgx.QgxError) as e:
+        qgx.qgx_eg_step_two_tables(ctx, st, op, nz, nz, cfg, other)                    # different sub-block sizes
+    assert e.value.status == qgx.QGX_ERR_INVALID_ARG
+    # an optimistic step that is not the first needs the vectors kept by the step before it
+    st.c.t = 5
+    ctx2 = qgx.qgx_create(0)
+    try:
+        with pytest.raises(qgx.QgxError) as e:
+            qgx.qgx_family_step(ctx2, st, qgx.QGX_METHOD_OPTDA, op, nz, cfg, mean_prev=mean_prev)
+        assert e.value.status == qgx.QGX_ERR_INVALID_ARG
+    finally:
+        qgx.qgx_destroy(ctx2)
+    st.c.t = 1
+    assert st.t == 1
+    qgx.qgx_family_step(ctx, st, qgx.QGX_METHOD_OPTDA, op, nz, cfg, mean_prev=mean_prev)   # and the context still works
+    qgx.qgx_sync_status(ctx)
+    assert st.t == 2
