@@ -240,6 +240,13 @@ typedef struct {
 } qgx_segment;
 qgx_status qgx_exchange_segments(qgx_ctx *ctx, const float *v, int K, size_t d, const qgx_segment *segs /*[host]*/,
                                  int nseg, uint32_t exchange_id, float *mean_out, uint64_t *total_bits);
+/* How the decode pass of the fused calls spreads its work.  By default (QGX_SPLIT_AUTO) vectors with few
+ * sub-blocks are decoded one worker per thread, followed by a kernel that adds the workers' values in worker
+ * order (same results, K times more threads, K * d floats of workspace, at most 256 MB); large vectors are decoded
+ * by one thread per sub-block over all workers.  QGX_SPLIT_NEVER / QGX_SPLIT_ALWAYS force one way (ALWAYS still
+ * falls back when the workspace would exceed 256 MB). */
+enum { QGX_SPLIT_AUTO = 0, QGX_SPLIT_NEVER = 1, QGX_SPLIT_ALWAYS = 2 };
+qgx_status qgx_set_decode_split(qgx_ctx *ctx, int mode);
 /* Where the last qgx_exchange on `slot` left its streams: all [dev], valid until the next call
  * that uses the slot.  Any output pointer may be NULL. */
 qgx_status qgx_exchange_streams(qgx_ctx *ctx, int slot, const uint32_t **stream, size_t *cap_words,

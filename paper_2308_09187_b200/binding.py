@@ -28,7 +28,7 @@ EXPORTS = [
     "qgx_build_codebook_huffman", "qgx_fit_levels", "qgx_symbol_pmf",
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
-    "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
+    "qgx_set_decode_split", "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
     "qgx_encode_noalloc", "qgx_exchange_segments",
 ]
 QGX_KERNEL_ENCODE, QGX_KERNEL_DECODE, QGX_KERNEL_HISTOGRAM, QGX_KERNEL_OPERATOR, QGX_KERNEL_FINISH = range(5)
@@ -327,6 +327,13 @@ def qgx_exchange_segments(ctx, v, sizes, cfgs, exchange_id, mean_out=None, total
     _chk(lib().qgx_exchange_segments(ctx.h, _ptr(v), K, C.c_size_t(d), segs, len(sizes), C.c_uint32(exchange_id),
                                      _ptr(mean_out), _ptr(total_bits)), "qgx_exchange_segments")
     return mean_out, total_bits
+
+
+QGX_SPLIT_AUTO, QGX_SPLIT_NEVER, QGX_SPLIT_ALWAYS = 0, 1, 2
+
+
+def qgx_set_decode_split(ctx, mode):
+    _chk(lib().qgx_set_decode_split(ctx.h, int(mode)), "qgx_set_decode_split")
 
 
 def qgx_exchange_streams(ctx, slot, K, nb):

@@ -42,6 +42,7 @@ struct qgx_ctx {
   size_t sym_ld;                         // bytes per worker in the kept-symbol layout
   int sym_nlev;                          // the level table those symbols were quantized with
   float sym_levels[QGX_MAX_LEVELS];
+  int decode_split;                      // QGX_SPLIT_AUTO / NEVER / ALWAYS: see qgx_set_decode_split
   // host-side cache of the fused calls: tables derived from a quantizer configuration (with their device copies)
   // and launch shapes; owned by qgx_exchange.cu
   void* table_cache;

@@ -372,6 +372,9 @@ struct DecodeArgs {
   float* xout;
   const double* scalars;        // scalars[1] = gamma_t
   bool vec_out;                 // d % 4 == 0 and mean, xin, xout 16-byte aligned: 128-bit stores
+  // small vectors: a thread decodes its sub-block of ONE worker and stores the values to values[K][d]; the
+  // ordered sum over the workers, the division and the state update follow in k_sum_workers
+  float* values;                // [K][d] or null
   // optional: keep the decoded symbols (1 byte per coordinate and worker) ...
   // Symbol bytes are kept transposed, so that a warp's accesses coalesce: worker k, sub-block gs, coordinate i of the
   // sub-block -> byte k * sym_ld + (gs / 32) * 32 * G + (i / 4) * 128 + (gs % 32) * 4 + i % 4.
@@ -573,7 +576,12 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
   bool bad = false;
   double sq = 0.0;
 
-  for (size_t gs = (size_t)blockIdx.x * blockDim.x + tid; gs - lane < total_sub; gs += (size_t)gridDim.x * blockDim.x) {
+  const bool wide = a.values != nullptr;
+  const size_t sub_pad = (total_sub + 31) & ~(size_t)31;                // whole warps per worker
+  const size_t items = wide ? sub_pad * (size_t)a.K : total_sub;
+  for (size_t item = (size_t)blockIdx.x * blockDim.x + tid; item - lane < items; item += (size_t)gridDim.x * blockDim.x) {
+    const size_t gs = wide ? item % sub_pad : item;                      // the sub-block
+    const int kbeg = wide ? (int)(item / sub_pad) : 0, kend = wide ? kbeg + 1 : a.K;
     const bool live = gs < total_sub;
     const size_t b = live ? gs / spb : a.nb - 1;
     const uint32_t s = live ? (uint32_t)(gs % spb) : 0u;
@@ -593,14 +601,15 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
     uint32_t* my_rows = s_prev + (kCompare ? (tid >> 5) * 2 * kRowWords : 0);
     uint32_t* my_stream = s_rows + (tid >> 5) * 2 * kStreamRow;
     __syncwarp();                                         // the previous sub-block's rows are no longer read
-    SubBlockAt nxt = find_subblock<G>(a, 0, b, hdr_bits, s, count > 0, uniform, lane, my_stream, kStreamRow);
-    if (kCompare) stage_symbol_row<kRowWords>(my_rows, a.sym_prev + (gs >> 5) * (size_t)(32 * G), lane);
+    SubBlockAt nxt = find_subblock<G>(a, kbeg, b, hdr_bits, s, count > 0, uniform, lane, my_stream + (kbeg & 1) * kStreamRow, kStreamRow);
+    if (kCompare)
+      stage_symbol_row<kRowWords>(my_rows + (kbeg & 1) * kRowWords, a.sym_prev + (size_t)kbeg * a.sym_ld + (gs >> 5) * (size_t)(32 * G), lane);
     asm volatile("cp.async.commit_group;" ::: "memory");
-    for (int k = 0; k < a.K; ++k) {
+    for (int k = kbeg; k < kend; ++k) {
       const SubBlockAt cur = nxt;
       const uint32_t* prev_row = my_rows + (k & 1) * kRowWords + lane;
       __syncwarp();                                       // every lane is done with the rows that are overwritten next
-      if (k + 1 < a.K) {
+      if (k + 1 < kend) {
         nxt = find_subblock<G>(a, k + 1, b, hdr_bits, s, count > 0, uniform, lane, my_stream + ((k + 1) & 1) * kStreamRow, kStreamRow);
         if (kCompare)
           stage_symbol_row<kRowWords>(my_rows + ((k + 1) & 1) * kRowWords,
@@ -664,6 +673,18 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
       bad = bad || (flags & 0x80u) || (count > 0 && used != cur.want);   // every sub-block uses exactly its length
     }
     if (count <= 0) continue;
+    if (wide) {                                         // the worker's values; summed by k_sum_workers
+      float* out = a.values + (size_t)kbeg * a.d + e0;
+      if (count == G && a.vec_out) {
+#pragma unroll
+        for (int i = 0; i < G; i += 4) *reinterpret_cast<float4*>(out + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < G; ++i)
+          if (i < count) out[i] = acc[i];
+      }
+      continue;
+    }
 
     float gam = 1.0f;
     if (a.update == 1) gam = (float)a.scalars[1];
@@ -706,7 +727,23 @@ namespace qgx {
 
 // workspace slots of a context
 enum { WS_OFF64 = 0, WS_FLAGS = 1, WS_LUT = 2, WS_SLOT0 = 3 /* stream, bits, offsets, total: 3..6 and 7..10 */,
-       WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18, WS_SEGBITS = 19 };
+       WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18, WS_SEGBITS = 19, WS_VALUES = 20 };
+
+// Small vectors, second part: mean_i = (((0 + v_{0,i}) + v_{1,i}) + ...) / K in worker order (the same sequential
+// sum as in the fused decode pass), then the optional state update.
+__global__ void __launch_bounds__(256) k_sum_workers(const float* __restrict__ values, int K, size_t d, float* __restrict__ mean,
+                                                     int update, const float* xin, float* xout, const double* scalars) {
+  const float Kf = (float)K;
+  const float gam = update == 1 ? (float)scalars[1] : 1.0f;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (size_t)gridDim.x * blockDim.x) {
+    float acc = 0.0f;
+    for (int k = 0; k < K; ++k) acc = __fadd_rn(acc, values[(size_t)k * d + i]);
+    const float m = __fdiv_rn(acc, Kf);
+    mean[i] = m;
+    if (update == 1) xout[i] = __fsub_rn(xin[i], __fmul_rn(gam, m));
+    if (update == 2) xout[i] = __fsub_rn(xin[i], m);
+  }
+}
 
 __global__ void k_add_u64(uint64_t* acc, const uint64_t* x, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -924,12 +961,31 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   da.scalars = upd ? upd->scalars : nullptr; da.st = c->dstatus;
   da.vec_out = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(mean_out) & 15u) == 0) &&
                ((reinterpret_cast<uintptr_t>(da.xin) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(da.xout) & 15u) == 0);
-  return launch_decode_average(c, da, ct, lt_kept, sym_mode);
+  // Small vectors leave most of the GPU idle and make every thread walk all K workers one after the other: there
+  // the decode pass runs one worker per thread and a second kernel forms the ordered sums.
+  const size_t total_sub = nb * (size_t)(bucket / ct.G);
+  da.values = nullptr;
+  const bool fits = (size_t)K * d * sizeof(float) <= ((size_t)256 << 20);
+  const bool small = total_sub * 2 < (size_t)148 * kDecThreads * 4;
+  if (K > 1 && fits && c->decode_split != QGX_SPLIT_NEVER && (small || c->decode_split == QGX_SPLIT_ALWAYS)) {
+    da.values = (float*)ws_get(c, WS_VALUES, sizeof(float) * (size_t)K * d);
+    if (!da.values) return QGX_ERR_CUDA;
+  }
+  rc = launch_decode_average(c, da, ct, lt_kept, sym_mode);
+  if (rc != QGX_OK || !da.values) return rc;
+  {
+    ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
+    const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>((d + 255) / 256, (size_t)148 * 8));
+    k_sum_workers<<<grid, 256, 0, c->stream>>>(da.values, K, d, mean_out, da.update, da.xin, da.xout, da.scalars);
+  }
+  count_launch(c);
+  return cuda_status(cudaGetLastError());
 }
 
 template <int G, int SYM>
 static qgx_status launch_decode_gs(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt) {
-  const size_t total_sub = da.nb * ((size_t)da.bucket / G);
+  const size_t subs = da.nb * ((size_t)da.bucket / G);
+  const size_t total_sub = da.values ? ((subs + 31) & ~(size_t)31) * (size_t)da.K : subs;   // threads wanted
   const size_t lut_bytes = sizeof(DecEntry) * ((size_t)2 << ct.maxlen) + DecodeSmem<G, SYM>::kBytes;   // table, then the rows
   const size_t want = (total_sub + kDecThreads - 1) / kDecThreads;
   int per_sm = 1;
@@ -977,6 +1033,12 @@ qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTab
 using namespace qgx;
 
 extern "C" {
+
+qgx_status qgx_set_decode_split(qgx_ctx* c, int mode) {
+  if (!c || mode < QGX_SPLIT_AUTO || mode > QGX_SPLIT_ALWAYS) return QGX_ERR_INVALID_ARG;
+  c->decode_split = mode;
+  return QGX_OK;
+}
 
 qgx_status qgx_exchange(qgx_ctx* c, const float* v, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t exchange_id,
                         int slot, float* mean_out, uint64_t* total_bits) {
