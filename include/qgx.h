@@ -224,7 +224,10 @@ qgx_status qgx_average(qgx_ctx *ctx, const float *norms, const uint8_t *sym, int
 /* quantize -> encode -> decode -> average in two kernels, same streams and same mean as the four
  * calls above in sequence.  v [dev] float[K][d]; mean_out [dev] float[d]; total_bits [dev]
  * uint64[K] (may be NULL).  The streams live in the context's workspace (slot 0 or 1, so that
- * the two exchanges of one iteration can both be kept). */
+ * the two exchanges of one iteration can both be kept); the workspace grows on first use (cudaMalloc) and is
+ * freed by qgx_destroy.  The code must have sub-blocks of 32, 64 or 128 coordinates that divide the bucket
+ * (QGX_ERR_INVALID_ARG otherwise: use the four calls).  Device-side errors: QGX_ERR_NONFINITE,
+ * QGX_ERR_CAPACITY, QGX_ERR_TIMEOUT (a bounded wait between CTAs ran out), QGX_ERR_CORRUPT. */
 qgx_status qgx_exchange(qgx_ctx *ctx, const float *v, int K, size_t d, const qgx_quant_cfg *cfg /*[host]*/,
                         uint32_t exchange_id, int slot, float *mean_out, uint64_t *total_bits);
 /* Layer-wise exchange: v [dev] float[K][d] holds nseg tensors back to back (segment s = coordinates
