@@ -727,7 +727,7 @@ namespace qgx {
 
 // workspace slots of a context
 enum { WS_OFF64 = 0, WS_FLAGS = 1, WS_LUT = 2, WS_SLOT0 = 3 /* stream, bits, offsets, total: 3..6 and 7..10 */,
-       WS_STATUS = 11, WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18, WS_SEGBITS = 19, WS_VALUES = 20 };
+       WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18, WS_SEGBITS = 19, WS_VALUES = 20 };
 
 // Small vectors, second part: mean_i = (((0 + v_{0,i}) + v_{1,i}) + ...) / K in worker order (the same sequential
 // sum as in the fused decode pass), then the optional state update.
@@ -869,8 +869,9 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   uint32_t* stream = (uint32_t*)ws_get(c, base + 0, sizeof(uint32_t) * ((size_t)K * cap + 64));   // slack: see Window
   uint32_t* bbits = (uint32_t*)ws_get(c, base + 1, sizeof(uint32_t) * (size_t)K * nb);
   uint32_t* offs = (uint32_t*)ws_get(c, base + 2, sizeof(uint32_t) * (size_t)K * nb);
-  unsigned long long* tot = (unsigned long long*)ws_get(c, base + 3, sizeof(uint64_t) * (size_t)K);
-  unsigned long long* status = (unsigned long long*)ws_get(c, WS_STATUS, sizeof(uint64_t) * ((size_t)K * nb + 2));
+  // one block per slot, zeroed by one memset: the per-worker bit totals, the ticket counter, the status words of the scan
+  unsigned long long* tot = (unsigned long long*)ws_get(c, base + 3, sizeof(uint64_t) * ((size_t)K + 2 + (size_t)K * nb));
+  unsigned long long* status = tot ? tot + K + 2 : nullptr;
   float* norms = (float*)ws_get(c, slot == 0 ? WS_NORMS : WS_NORMS2, sizeof(float) * (size_t)K * nb);
   const DecEntry* lut = tables->lut_dev;
   if (!stream || !bbits || !offs || !tot || !status || !norms || !lut) return QGX_ERR_CUDA;
@@ -878,15 +879,13 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   c->slot_K[slot] = K;
   c->slot_nb[slot] = nb;
 
-  if (cudaMemsetAsync(status, 0, sizeof(uint64_t) * ((size_t)K * nb + 2), c->stream) != cudaSuccess ||
-      cudaMemsetAsync(tot, 0, sizeof(uint64_t) * (size_t)K, c->stream) != cudaSuccess)
-    return QGX_ERR_CUDA;
+  if (cudaMemsetAsync(tot, 0, sizeof(uint64_t) * ((size_t)K + 2 + (size_t)K * nb), c->stream) != cudaSuccess) return QGX_ERR_CUDA;
 
   EncodeArgs ea;
   ea.src = src; ea.d = d; ea.bucket = bucket; ea.K = K; ea.nb = nb; ea.norm_type = cfg->norm_type; ea.xid = xid; ea.quad_base = coord_base / kQuad;
   ea.vec_ok = (d % kQuad == 0) && (src.ld % kQuad == 0) && ((reinterpret_cast<uintptr_t>(src.v) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
   ea.stream = stream; ea.cap_words = cap; ea.bucket_bits = bbits; ea.offsets = offs; ea.total_bits = tot; ea.norms = norms;
-  ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(status + (size_t)K * nb); ea.st = c->dstatus;
+  ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(tot + K); ea.st = c->dstatus;
   uint8_t* sym_out = nullptr;
   const uint8_t* sym_prev = nullptr;
   const size_t sym_ld = ((nb * (size_t)(bucket / ct.G) + 31) / 32) * 32 * (size_t)ct.G;   // see DecodeArgs::sym_out
