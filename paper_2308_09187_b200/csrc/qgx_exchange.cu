@@ -172,7 +172,7 @@ __device__ __forceinline__ void load_bucket_octets(BucketRegs<2 * P>& r, const D
 // The bucket image is double buffered, so the copy-out of one bucket needs no barrier before the next
 // bucket starts.  A thread works on P octets; warp w owns the 256 * P coordinates [w * 256 * P, ...).
 template <int P, int G>
-__global__ void __launch_bounds__(P == 1 ? 256 : 512, P == 4 ? 2 : 1)
+__global__ void __launch_bounds__(P == 1 ? 256 : 512, P == 1 ? 4 : 2)
 k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
                   const __grid_constant__ RoundTable rt) {
