@@ -36,9 +36,9 @@ WORKLOAD = "c5-scale: K=32, d=2^26, mixture noise, diagonal operator, bucket 163
 
 
 # measured DRAM traffic of k_exchange_encode per coordinate (ncu, current kernel); None once the kernel has changed
-ENCODE_DRAM_BYTES_PER_COORDINATE = 4.890
+ENCODE_DRAM_BYTES_PER_COORDINATE = 4.882
 # executed thread instructions of k_exchange_encode per coordinate (ncu, same capture); None once the kernel has changed
-ENCODE_INSTRUCTIONS_PER_COORDINATE = 60.6
+ENCODE_INSTRUCTIONS_PER_COORDINATE = 60.7
 
 def exchange_bytes(K, d, nb, stream_words):
     """Algorithmic bytes of one exchange: read V, write + read the streams and their length words, write the mean."""
@@ -203,7 +203,7 @@ def run_ours(args):
     enc_ms = ms_enc / max(n_enc, 1)
     achieved = enc_bytes / (enc_ms * 1e-3) / 1e9 if n_enc else None
     # DRAM bytes per launch of that kernel: counted by ncu on a smaller case of the same kernel (see
-    # profiles/exchange_kernels_K8_d16M.txt: 656.4 MB read + written for K * d = 2^27 coordinates) and scaled by
+    # profiles/exchange_kernels_K8_d16M.txt: 655.2 MB read + written for K * d = 2^27 coordinates) and scaled by
     # the coordinates of a launch, which the traffic is proportional to.  Set to None when the kernel changes.
     traffic = args.traffic_bytes
     if traffic is None and ENCODE_DRAM_BYTES_PER_COORDINATE is not None:
