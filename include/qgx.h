@@ -234,8 +234,10 @@ qgx_status qgx_exchange(qgx_ctx *ctx, const float *v, int K, size_t d, const qgx
  * [offset, offset + length) of every worker, offsets multiples of 4, the segments tiling [0, d) in order);
  * every segment is exchanged with its own table and code (segs[s].cfg), buckets never cross a segment, and
  * coordinate offset + i of worker k uses the generator counter of coordinate offset + i.  mean_out [dev]
- * float[d]; total_bits [dev] uint64[K] (may be NULL) receives the stream bits summed over segments.  The
- * streams of one segment are overwritten by the next (slot 0 of the workspace). */
+ * float[d]; total_bits [dev] uint64[K] (may be NULL) receives the stream bits summed over segments.  With more
+ * than one segment the tensors run side by side on a few streams and workspaces of the context's own, forked
+ * from and joined back into the context's stream (the call stays asynchronous and ordered on that stream); their
+ * streams are not reachable through qgx_exchange_streams. */
 typedef struct {
   size_t offset;
   size_t length;

@@ -160,6 +160,7 @@ void qgx_destroy(qgx_ctx* c) {
   cudaSetDevice(c->device);
   cudaStreamSynchronize(c->stream);
   if (c->timing_ev) timing_free(c);
+  free_seg_children(c);
   free_table_cache(c);
   for (int i = 0; i < 24; ++i)
     if (c->ws[i]) cudaFree(c->ws[i]);
@@ -195,7 +196,7 @@ const char* qgx_status_str(qgx_status s) {
   return "unknown status";
 }
 
-uint64_t qgx_launch_count(const qgx_ctx* c) { return c ? c->launches : 0; }
+uint64_t qgx_launch_count(const qgx_ctx* c) { return c ? c->launches + seg_children_launches(c) : 0; }
 
 qgx_status qgx_timing_enable(qgx_ctx* c, int max_records) {
   if (!c || max_records < 0 || max_records > (1 << 20)) return QGX_ERR_INVALID_ARG;

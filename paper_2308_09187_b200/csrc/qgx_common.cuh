@@ -46,6 +46,9 @@ struct qgx_ctx {
   // host-side cache of the fused calls: tables derived from a quantizer configuration (with their device copies)
   // and launch shapes; owned by qgx_exchange.cu
   void* table_cache;
+  // helper contexts (own streams and workspaces) that run the tensors of a layer-wise exchange side by side;
+  // owned by qgx_exchange.cu
+  void* seg_children;
   // optional per-kernel timing: pairs of events recorded around instrumented launches
   int timing_on;
   int timing_cap;                        // pairs allocated
@@ -297,6 +300,8 @@ qgx_status make_code_table(const qgx_codebook* cb, int bucket, CodeTable* out);
 void make_round_table(const float* lev, int nlev, RoundTable* out);
 void* ws_get(qgx_ctx* c, int which, size_t bytes);          // nullptr on failure
 void free_table_cache(qgx_ctx* c);
+void free_seg_children(qgx_ctx* c);
+uint64_t seg_children_launches(const qgx_ctx* c);
 qgx_status cuda_status(cudaError_t e);
 inline void count_launch(qgx_ctx* c, int n = 1) { c->launches += (uint64_t)n; }
 

@@ -745,11 +745,6 @@ __global__ void __launch_bounds__(256) k_sum_workers(const float* __restrict__ v
   }
 }
 
-__global__ void k_add_u64(uint64_t* acc, const uint64_t* x, int n) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) acc[i] += x[i];
-}
-
 qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct, const LevelTable& lt, int sym_mode);
 
 // ---- what a call derives from a quantizer configuration, kept between calls --------------------
@@ -772,6 +767,27 @@ struct TableCache {
   LaunchShape enc[3][3];                // [octets per thread 1, 2, 4][sub-block 32, 64, 128]
   LaunchShape dec[3][6];                // [sub-block][symbol mode]
 };
+
+// Lets a kernel use all the dynamic shared memory that the device allows, once per kernel and device.  (The
+// attribute belongs to the function, not to a context: a per-context "largest size asked so far" would be undone
+// by another context asking for less.)
+template <typename Kernel>
+static void allow_max_dynamic_smem(Kernel kernel, int device) {
+  struct Seen { const void* fn; int device; };
+  static Seen seen[256];                                // all template instances of a kernel share this function
+  static int nseen = 0;
+  const void* fn = reinterpret_cast<const void*>(kernel);
+  for (int i = 0; i < nseen; ++i)
+    if (seen[i].fn == fn && seen[i].device == device) return;
+  int optin = 0;
+  cudaFuncAttributes fa;
+  if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) == cudaSuccess &&
+      cudaFuncGetAttributes(&fa, kernel) == cudaSuccess && optin > (int)fa.sharedSizeBytes)
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)fa.sharedSizeBytes);
+  else
+    cudaGetLastError();
+  if (nseen < 256) { seen[nseen].fn = fn; seen[nseen].device = device; ++nseen; }
+}
 
 void free_table_cache(qgx_ctx* c) {
   TableCache* tc = (TableCache*)c->table_cache;
@@ -918,9 +934,9 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   int per_sm = 1;
 #define QGX_LAUNCH_E(V, GG)                                                                                    \
   do {                                                                                                         \
+    allow_max_dynamic_smem(k_exchange_encode<V, GG>, c->device);                                               \
     LaunchShape& shape = table_cache(c)->enc[V == 1 ? 0 : (V == 2 ? 1 : 2)][GG == 32 ? 0 : (GG == 64 ? 1 : 2)];  \
-    if (shape.smem != smem + 1 + (size_t)threads * 0x100000) {   /* asked once per shape, not per call */        \
-      cudaFuncSetAttribute(k_exchange_encode<V, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+    if (shape.smem != smem + 1 + (size_t)threads * 0x100000) {   /* occupancy asked once per shape */              \
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG>, threads, smem);         \
       shape.smem = smem + 1 + (size_t)threads * 0x100000;                                                      \
       shape.per_sm = per_sm < 1 ? 1 : per_sm;                                                                  \
@@ -990,9 +1006,9 @@ static qgx_status launch_decode_gs(qgx_ctx* c, const DecodeArgs& da, const CodeT
   int per_sm = 1;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
+    allow_max_dynamic_smem(k_exchange_decode<G, SYM>, c->device);
     LaunchShape& shape = table_cache(c)->dec[G == 32 ? 0 : (G == 64 ? 1 : 2)][SYM];
-    if (shape.smem != lut_bytes + 1) {                       // asked once per shape, not per call
-      cudaFuncSetAttribute(k_exchange_decode<G, SYM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lut_bytes);
+    if (shape.smem != lut_bytes + 1) {                       // occupancy asked once per shape, not per call
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, SYM>, kDecThreads, lut_bytes);
       shape.smem = lut_bytes + 1;
       shape.per_sm = per_sm < 1 ? 1 : per_sm;
@@ -1027,6 +1043,75 @@ qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTab
   }
 }
 
+// ---- helper contexts of the layer-wise exchange -------------------------------------------------
+// The tensors of a layer-wise vector are independent; most are small, so one after the other they leave the GPU
+// mostly idle.  They are spread over a few helper contexts, each with its own stream and workspace; the caller's
+// stream forks into them and joins them again (events), so the call stays asynchronous and ordered on that stream.
+constexpr int kSegStreams = 4;
+struct SegChildren {
+  qgx_ctx* ctx[kSegStreams];
+  cudaEvent_t fork, join[kSegStreams];
+};
+
+void free_seg_children(qgx_ctx* c) {
+  SegChildren* sc = (SegChildren*)c->seg_children;
+  if (!sc) return;
+  for (int i = 0; i < kSegStreams; ++i) {
+    qgx_ctx* h = sc->ctx[i];
+    if (!h) continue;
+    cudaStreamSynchronize(h->stream);
+    free_table_cache(h);
+    for (int w = 0; w < 24; ++w)
+      if (h->ws[w]) cudaFree(h->ws[w]);
+    cudaStreamDestroy(h->stream);
+    cudaEventDestroy(sc->join[i]);
+    delete h;                                           // the status block belongs to the parent
+  }
+  cudaEventDestroy(sc->fork);
+  delete sc;
+  c->seg_children = nullptr;
+}
+
+uint64_t seg_children_launches(const qgx_ctx* c) {
+  const SegChildren* sc = (const SegChildren*)c->seg_children;
+  uint64_t n = 0;
+  if (sc)
+    for (int i = 0; i < kSegStreams; ++i) n += sc->ctx[i] ? sc->ctx[i]->launches : 0;
+  return n;
+}
+
+static SegChildren* seg_children(qgx_ctx* c) {
+  if (c->seg_children) return (SegChildren*)c->seg_children;
+  SegChildren* sc = new (std::nothrow) SegChildren();
+  if (!sc) return nullptr;
+  bool ok = cudaEventCreateWithFlags(&sc->fork, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < kSegStreams && ok; ++i) {
+    qgx_ctx* h = new (std::nothrow) qgx_ctx();
+    if (!h) { ok = false; break; }
+    std::memset(h, 0, sizeof(*h));
+    h->device = c->device;
+    h->sym_slot = -1;
+    h->decode_split = c->decode_split;
+    h->dstatus = c->dstatus;                            // errors latch into the parent's status block
+    if (cudaStreamCreateWithFlags(&h->stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&sc->join[i], cudaEventDisableTiming) != cudaSuccess) {
+      delete h;
+      ok = false;
+      break;
+    }
+    sc->ctx[i] = h;
+  }
+  c->seg_children = sc;
+  if (!ok) { cudaGetLastError(); free_seg_children(c); return nullptr; }
+  return sc;
+}
+
+// acc[i] += x[i]; several streams may add into the same totals
+__global__ void k_add_u64_atomic(unsigned long long* acc, const unsigned long long* x, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) atomicAdd(acc + i, x[i]);
+}
+
 }  // namespace qgx
 
 using namespace qgx;
@@ -1057,22 +1142,41 @@ qgx_status qgx_exchange_segments(qgx_ctx* c, const float* v, int K, size_t d, co
   }
   if (at != d) return QGX_ERR_INVALID_ARG;
   if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
-  uint64_t* seg_bits = nullptr;
-  if (total_bits) {
-    seg_bits = (uint64_t*)ws_get(c, WS_SEGBITS, sizeof(uint64_t) * (size_t)K);
-    if (!seg_bits) return QGX_ERR_CUDA;
-    if (cudaMemsetAsync(total_bits, 0, sizeof(uint64_t) * (size_t)K, c->stream) != cudaSuccess) return QGX_ERR_CUDA;
-  }
-  for (int s = 0; s < nseg; ++s) {
-    DualSource src{v + segs[s].offset, nullptr, d, 0};
-    qgx_status rc = exchange_impl(c, src, K, segs[s].length, segs[s].cfg, exchange_id, 0, mean_out + segs[s].offset, seg_bits,
-                                  nullptr, 0, nullptr, segs[s].offset);
-    if (rc != QGX_OK) return rc;
-    if (total_bits) {
-      k_add_u64<<<(K + 255) / 256, 256, 0, c->stream>>>(total_bits, seg_bits, K);
-      count_launch(c);
+  if (total_bits && cudaMemsetAsync(total_bits, 0, sizeof(uint64_t) * (size_t)K, c->stream) != cudaSuccess) return QGX_ERR_CUDA;
+  SegChildren* sc = nseg > 1 ? seg_children(c) : nullptr;
+  if (nseg > 1 && !sc) return QGX_ERR_CUDA;
+  const int lanes = sc ? std::min(nseg, kSegStreams) : 0;
+  if (sc) {                                             // fork: the helpers start after everything queued so far
+    if (cudaEventRecord(sc->fork, c->stream) != cudaSuccess) return QGX_ERR_CUDA;
+    for (int i = 0; i < lanes; ++i) {
+      sc->ctx[i]->decode_split = c->decode_split;
+      if (cudaStreamWaitEvent(sc->ctx[i]->stream, sc->fork, 0) != cudaSuccess) return QGX_ERR_CUDA;
     }
   }
+  qgx_status rc = QGX_OK;
+  for (int s = 0; s < nseg && rc == QGX_OK; ++s) {
+    qgx_ctx* h = sc ? sc->ctx[s % lanes] : c;
+    uint64_t* seg_bits = nullptr;
+    if (total_bits) {
+      seg_bits = (uint64_t*)ws_get(h, WS_SEGBITS, sizeof(uint64_t) * (size_t)K);
+      if (!seg_bits) { rc = QGX_ERR_CUDA; break; }
+    }
+    DualSource src{v + segs[s].offset, nullptr, d, 0};
+    rc = exchange_impl(h, src, K, segs[s].length, segs[s].cfg, exchange_id, 0, mean_out + segs[s].offset, seg_bits,
+                       nullptr, 0, nullptr, segs[s].offset);
+    if (rc == QGX_OK && total_bits) {
+      k_add_u64_atomic<<<(K + 255) / 256, 256, 0, h->stream>>>(reinterpret_cast<unsigned long long*>(total_bits),
+                                                               reinterpret_cast<const unsigned long long*>(seg_bits), K);
+      count_launch(h);
+    }
+  }
+  if (sc) {                                             // join, also after an error: the caller's stream waits for the helpers
+    for (int i = 0; i < lanes; ++i)
+      if (cudaEventRecord(sc->join[i], sc->ctx[i]->stream) != cudaSuccess ||
+          cudaStreamWaitEvent(c->stream, sc->join[i], 0) != cudaSuccess)
+        rc = rc == QGX_OK ? QGX_ERR_CUDA : rc;
+  }
+  if (rc != QGX_OK) return rc;
   return cuda_status(cudaGetLastError());
 }
 
