@@ -20,6 +20,8 @@ QGX_CODE_FIXED, QGX_CODE_HUFFMAN, QGX_CODE_ELIAS = 0, 1, 2
 QGX_OP_DENSE_AFFINE, QGX_OP_BILINEAR, QGX_OP_DIAGONAL = 0, 1, 2
 QGX_REFIT_NONE, QGX_REFIT_CONTINUE, QGX_REFIT_FIRST = 0, 1, 2
 QGX_NORMS_SUPPLIED = 1
+QGX_QUANTIZE_RNG_HALF32 = 2
+QGX_RNG_WORD24, QGX_RNG_HALF32 = 0, 1
 QGX_MAX_LEVELS, QGX_MAX_CODE_LEN, QGX_MAX_BUCKET = 32, 12, 16384
 
 EXPORTS = [
@@ -28,7 +30,7 @@ EXPORTS = [
     "qgx_build_codebook_huffman", "qgx_fit_levels", "qgx_symbol_pmf",
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
-    "qgx_set_decode_split", "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
+    "qgx_set_decode_split", "qgx_set_encode_path", "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
     "qgx_encode_noalloc", "qgx_exchange_segments",
 ]
 QGX_KERNEL_ENCODE, QGX_KERNEL_DECODE, QGX_KERNEL_HISTOGRAM, QGX_KERNEL_OPERATOR, QGX_KERNEL_FINISH = range(5)
@@ -47,7 +49,7 @@ class qgx_codebook(C.Structure):
 
 class qgx_quant_cfg(C.Structure):
     _fields_ = [("nlev", C.c_int32), ("bucket", C.c_int32), ("norm_type", C.c_int32), ("code_type", C.c_int32),
-                ("nbins", C.c_int32), ("pad", C.c_int32), ("seed", C.c_uint64),
+                ("nbins", C.c_int32), ("rng_mode", C.c_int32), ("seed", C.c_uint64),
                 ("levels", C.c_float * 32), ("cb", qgx_codebook)]
 
     def level_list(self):
@@ -334,6 +336,13 @@ QGX_SPLIT_AUTO, QGX_SPLIT_NEVER, QGX_SPLIT_ALWAYS = 0, 1, 2
 
 def qgx_set_decode_split(ctx, mode):
     _chk(lib().qgx_set_decode_split(ctx.h, int(mode)), "qgx_set_decode_split")
+
+
+QGX_ENCODE_AUTO, QGX_ENCODE_REGISTERS = 0, 1
+
+
+def qgx_set_encode_path(ctx, mode):
+    _chk(lib().qgx_set_encode_path(ctx.h, int(mode)), "qgx_set_encode_path")
 
 
 def qgx_exchange_streams(ctx, slot, K, nb):

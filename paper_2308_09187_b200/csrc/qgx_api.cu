@@ -84,19 +84,41 @@ void make_round_table(const float* lev, int nlev, RoundTable* out) {
     margin = std::max(margin, e);
   }
   margin = (margin + 2.0) * 1.01;
-  bool usable = std::isfinite(margin) && margin < S / 4.0;
-  for (int i = 0; i < kKeyBins && usable; ++i) {
-    const uint32_t lo_bits = (uint32_t)(i + kKeyMin) << kKeyShift, hi_bits = ((uint32_t)(i + 1 + kKeyMin) << kKeyShift) - 1u;
-    float lo, hi;
-    std::memcpy(&lo, &lo_bits, 4);
-    std::memcpy(&hi, &hi_bits, 4);
-    int inside = 0;
-    for (int j = 1; j <= nlev - 2; ++j) inside += (out->knot[j] > lo && out->knot[j] <= hi) ? 1 : 0;
-    if (inside > 1) usable = false;
+  // the octet encoder's variant: only the leading 16 bits h of the variate are subtracted, as the float 2^23 + h
+  // times -S 2^-16 (the 2^23 part is folded into a16); r lies within 2^-17 of the centre (h + 1/2) 2^-16
+  double margin16 = 0.0;
+  for (int t = 0; t <= nlev - 2; ++t) {
+    out->a16[t] = (float)(S * t - b[t] * ((double)lev[t] + c0) + 0.5 * S - S / 131072.0 + 8388608.0 * (S / 65536.0));
+    const double wmin = std::min(width[t], t + 1 <= nlev - 2 ? width[t + 1] : width[t]);
+    const double a_ulp = (double)std::nextafter(std::fabs(out->a16[t]), INFINITY) - (double)std::fabs(out->a16[t]);
+    const double e = 2.0 * S * 0x1p-22 * ((double)lev[t + 1] + c0) / wmin + a_ulp + 1.5 + 1.0 + 1.01 * S / 131072.0;
+    margin16 = std::max(margin16, e);
   }
+  margin16 = (margin16 + 2.0) * 1.01;
+  bool usable = std::isfinite(margin) && margin < S / 4.0 && std::isfinite(margin16) && margin16 < S / 4.0;
+  // the coarsest bins that still hold at most one level each (coarser bins are stored in more copies: see kKeyShiftMin)
+  int shift = -1;
+  for (int sh = kKeyShiftMax; sh >= kKeyShiftMin && usable && shift < 0; --sh) {
+    const uint32_t nbins = ((kKeyTop - kKeyBase) >> sh) + 1u;
+    bool ok = true;
+    for (uint32_t i = 0; i < nbins && ok; ++i) {
+      const uint32_t lo_bits = kKeyBase + (i << sh), hi_bits = kKeyBase + ((i + 1u) << sh) - 1u;
+      float lo, hi;
+      std::memcpy(&lo, &lo_bits, 4);
+      std::memcpy(&hi, &hi_bits, 4);
+      int inside = 0;
+      for (int j = 1; j <= nlev - 2; ++j) inside += (out->knot[j] > lo && out->knot[j] <= hi) ? 1 : 0;
+      if (inside > 1) ok = false;
+    }
+    if (ok) shift = sh;
+  }
+  if (shift < 0) usable = false;
+  out->key_shift = shift < 0 ? kKeyShiftMin : shift;
   out->usable = usable ? 1 : 0;
   out->thr = usable ? (float)(S / 2.0 - margin) : -1.0f;
   out->neg_qscale = (float)(-S / 8388608.0);
+  out->thr16 = usable ? (float)(S / 2.0 - margin16) : -1.0f;
+  out->neg_qscale16 = (float)(-S / 65536.0);
   out->magic = (float)(1.5 * 8388608.0 * S);
 }
 
@@ -142,6 +164,8 @@ qgx_status qgx_create(qgx_ctx** out, int device, void* cuda_stream) {
   std::memset(c, 0, sizeof(*c));
   c->device = device;
   c->sym_slot = -1;
+  c->num_sms = 1;
+  if (cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->num_sms < 1) { cudaGetLastError(); c->num_sms = 1; }
   c->stream = (cudaStream_t)cuda_stream;
   if (cudaMalloc((void**)&c->dstatus, sizeof(DevStatus)) != cudaSuccess ||
       cudaMemsetAsync(c->dstatus, 0, sizeof(DevStatus), c->stream) != cudaSuccess ||

@@ -64,6 +64,31 @@ __device__ __forceinline__ void pack_quad_codes(uint32_t t, const uint32_t* pair
   *bits = ((uint64_t)hi << 32) | lo;
   *nbits = n01 + n23;
 }
+// Pair table of the octet encoder: indexed by (first + 64 * second) mod 4096, first and second the signed level
+// indices (negative for a negative coordinate) of two consecutive coordinates -- the low 12 bits of that sum as
+// a two's complement number, which is how it comes out of the float arithmetic of the rounding.
+__device__ __forceinline__ void fill_pair_lut_signed(uint32_t* pair, const EncLut* lut) {
+  for (int i = threadIdx.x; i < kPairLutSize; i += blockDim.x) {
+    const int lo6 = i & 63;
+    const int first = lo6 >= 32 ? lo6 - 64 : lo6;
+    const int hi6 = ((i - first) >> 6) & 63;
+    const int second = hi6 >= 32 ? hi6 - 64 : hi6;
+    const uint32_t a = lut->e[((first < 0 ? -first : first) & 31) | (first < 0 ? 32 : 0)];
+    const uint32_t b = lut->e[((second < 0 ? -second : second) & 31) | (second < 0 ? 32 : 0)];
+    const uint32_t na = a >> 16, nb = b >> 16;
+    pair[i] = ((a & 0xffffu) | ((b & 0xffffu) << na)) | ((na + nb) << 26);
+  }
+}
+
+// stream bits of four consecutive coordinates from their two pair-table entries
+__device__ __forceinline__ void pack_pair_entries(uint32_t e01, uint32_t e23, uint64_t* bits, uint32_t* nbits) {
+  const uint32_t b01 = e01 & 0x3ffffffu, n01 = e01 >> 26, b23 = e23 & 0x3ffffffu, n23 = e23 >> 26;
+  const uint32_t lo = b01 | (b23 << n01);
+  const uint32_t hi = __funnelshift_l(b23, 0u, n01);
+  *bits = ((uint64_t)hi << 32) | lo;
+  *nbits = n01 + n23;
+}
+
 // OR `nbits` (<= 52) bits into the bucket image at bit position pos (shared memory, zeroed before).
 // Two words are always touched; a third only when the bits reach it.
 __device__ __forceinline__ void put_bits(uint32_t* img, uint32_t pos, uint64_t bits, uint32_t nbits) {

@@ -43,6 +43,8 @@ struct qgx_ctx {
   int sym_nlev;                          // the level table those symbols were quantized with
   float sym_levels[QGX_MAX_LEVELS];
   int decode_split;                      // QGX_SPLIT_AUTO / NEVER / ALWAYS: see qgx_set_decode_split
+  int encode_path;                       // QGX_ENCODE_AUTO / REGISTERS: see qgx_set_encode_path
+  int num_sms;                           // multiprocessors of the device
   // host-side cache of the fused calls: tables derived from a quantizer configuration (with their device copies)
   // and launch shapes; owned by qgx_exchange.cu
   void* table_cache;
@@ -65,10 +67,18 @@ struct LevelTable {
   float lev[QGX_MAX_LEVELS];
 };
 
-// bins of the rounding table over the float pattern of the normalized coordinate (see round_fast)
-constexpr int kKeyShift = 17;                       // 64 bins per octave of u
-constexpr int kKeyMin = 0x37800000 >> kKeyShift;    // pattern of 2^-16: everything below shares bin 0
-constexpr int kKeyBins = (0x3F800000 >> kKeyShift) - kKeyMin + 1;   // up to u = 1.0: 1025 bins
+// Bins of the rounding table over the float pattern of the normalized coordinate (see round_fast).  A bin covers
+// 2^key_shift consecutive patterns (2^(23 - key_shift) bins per octave of u: 64 at key_shift 17, 8 at 20); patterns
+// below 2^-16 share bin 0 and the table ends at u = 1.  Every bin is stored 2^(key_shift - 17) times, once per
+// residue of the lane number, so that the lanes of a quarter warp read different bank groups whatever bins they
+// hit: the coarser the bins the levels allow (at most one level per bin), the fewer bank conflicts.  All layouts
+// take the same 16.1 KB.
+constexpr int kKeyShiftMin = 17, kKeyShiftMax = 20;
+constexpr uint32_t kKeyBase = 0x37800000u;          // pattern of 2^-16
+constexpr uint32_t kKeyTop = 0x3F800000u;           // pattern of 1.0
+constexpr int kBinEntries = ((kKeyTop - kKeyBase) >> kKeyShiftMin) + (1 << (kKeyShiftMax - kKeyShiftMin));   // float4 entries, any layout
+constexpr int kBinAddrShift = kKeyShiftMin - 4;     // pattern >> 13 = byte offset of the bin's first copy (+ a constant)
+constexpr uint32_t kBinAddrBase = kKeyBase >> kBinAddrShift;
 struct CodeTable {
   int nlev;
   int maxlen;
@@ -174,6 +184,7 @@ constexpr float kRoundShift = 1.52587890625e-05f;       // 2^-16: keeps u2 insid
 struct RoundTable {
   int nlev;
   int usable;                            // 0: some bin holds two levels, or the margin is too wide
+  int key_shift;                         // layout of the bin table: kKeyShiftMin..kKeyShiftMax
   float thr;                             // S / 2 - margin
   float neg_qscale;                      // -S / 2^23
   float magic;                           // 1.5 * 2^23 * S
@@ -181,17 +192,25 @@ struct RoundTable {
   float b[QGX_MAX_LEVELS];               //               S / (l_{tau+1} - l_tau)
   float knot[QGX_MAX_LEVELS];            // l_j + 2^-16 for interior levels j, else a value never reached
   float db[QGX_MAX_LEVELS];              // b[j] - b[j - 1]
+  // the same map for the octet encoder, which subtracts only the leading 16 bits h of the variate (as the float
+  // 2^23 + h) and leaves the rest to the exact routine:
+  float a16[QGX_MAX_LEVELS];             // S tau - b (l_tau + 2^-16) + S / 2 - S 2^-17 + 2^23 S 2^-16
+  float thr16;                           // S / 2 - (margin + what the dropped variate bits can move)
+  float neg_qscale16;                    // -S / 2^16
 };
 
-// one entry per bin: {a, b, knot, db} of the interval of the bin's lowest value
-__device__ __forceinline__ void fill_bin_table(float4* bin, const RoundTable& rt) {
-  for (int i = threadIdx.x; i < kKeyBins; i += blockDim.x) {
-    const float lo = __uint_as_float((uint32_t)(i + kKeyMin) << kKeyShift);
-    const float hi = __uint_as_float(((uint32_t)(i + 1 + kKeyMin) << kKeyShift) - 1u);
+// one entry per bin and copy: {a (or a16), b, knot, db} of the interval of the bin's lowest value
+__device__ __forceinline__ void fill_bin_table(float4* bin, const RoundTable& rt, bool octet_encoder = false) {
+  const int rep_log = rt.key_shift - kKeyShiftMin;
+  const int nbins = (int)((kKeyTop - kKeyBase) >> rt.key_shift) + 1;
+  for (int i = threadIdx.x; i < (nbins << rep_log); i += blockDim.x) {
+    const uint32_t b = (uint32_t)(i >> rep_log);
+    const float lo = __uint_as_float(kKeyBase + (b << rt.key_shift));
+    const float hi = __uint_as_float(kKeyBase + ((b + 1u) << rt.key_shift) - 1u);
     int t0 = 0;
     for (int j = 1; j <= rt.nlev - 2; ++j) t0 = (rt.knot[j] <= lo) ? j : t0;
     const bool straddle = (t0 + 1 <= rt.nlev - 2) && (rt.knot[t0 + 1] <= hi);
-    bin[i] = make_float4(rt.a[t0], rt.b[t0], straddle ? rt.knot[t0 + 1] : 4.0f, straddle ? rt.db[t0 + 1] : 0.0f);
+    bin[i] = make_float4(octet_encoder ? rt.a16[t0] : rt.a[t0], rt.b[t0], straddle ? rt.knot[t0 + 1] : 4.0f, straddle ? rt.db[t0 + 1] : 0.0f);
   }
 }
 
@@ -205,6 +224,8 @@ struct RoundConsts {
   float rn;                              // RN(1 / norm)
   float thr;                             // negative: every coordinate goes to the exact routine
   float neg_qscale, magic;
+  uint32_t bin_mask;                     // keeps the bin part of pattern >> kBinAddrShift
+  uint32_t bin_lane;                     // byte offset of this lane's copy inside a bin
 };
 
 __device__ __forceinline__ RoundConsts round_consts(const RoundTable& rt, float norm) {
@@ -214,13 +235,17 @@ __device__ __forceinline__ RoundConsts round_consts(const RoundTable& rt, float 
   c.thr = ok ? rt.thr : -1.0f;
   c.neg_qscale = rt.neg_qscale;
   c.magic = rt.magic;
+  const uint32_t copy_bytes = 16u << (rt.key_shift - kKeyShiftMin);
+  c.bin_mask = ~(copy_bytes - 1u);
+  c.bin_lane = ((threadIdx.x & 31u) << 4) & (copy_bytes - 1u);
   return c;
 }
 
 // pattern of the float whose low mantissa bits are the level index; *unsafe: ask the exact routine
 __device__ __forceinline__ uint32_t round_fast(float absv, const RoundConsts& c, const float4* bin, uint32_t word, bool* unsafe) {
-  const float u2 = fmaf(absv, c.rn, kRoundShift);
-  const float4 e = bin[(int)(__float_as_uint(u2) >> kKeyShift) - kKeyMin];
+  const float u2 = fminf(fmaf(absv, c.rn, kRoundShift), 1.0f + kRoundShift);   // a supplied norm may be smaller than |v|
+  const uint32_t off = ((__float_as_uint(u2) >> kBinAddrShift) & c.bin_mask) | c.bin_lane;
+  const float4 e = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(bin) + off - kBinAddrBase);
   float X = fmaf(u2, e.y, e.x);
   X = fmaf(__saturatef(__fsub_rn(u2, e.z)), e.w, X);
   const float mb = __uint_as_float(0x4B000000u | (word >> 9));                    // 2^23 + (m >> 1), exact
@@ -254,6 +279,95 @@ __device__ __forceinline__ uint32_t quantize_quad_codes(const float4 x, const ui
                            prmt(__float_as_uint(x.z), __float_as_uint(x.w), 0x00fbu), 0x5410u);
   const uint32_t nz = (idx4 + 0x1f1f1f1fu) & 0x20202020u;                          // level indices are < 0x20
   return idx4 | (s4 & nz);
+}
+
+// ---- the octet encoder's rounding ---------------------------------------------------------------
+// How the uniform variate of a coordinate is drawn (the paper says only "with probability xi"):
+//   QGX_RNG_WORD24  r = (w >> 8) 2^-24, w = word (i & 3) of the Philox block with counter (i >> 2, worker, exchange);
+//   QGX_RNG_HALF32  r = (h 2^16 + h') 2^-32: h = 16-bit half (i & 7) of the block with counter (i >> 3, worker,
+//                   exchange) -- half j is bits 16 (j & 1) .. of word j >> 1 --, h' the same half of the block with
+//                   counter (i >> 3, worker | 2^31, exchange).  h alone decides all but about 2^-16 of the
+//                   coordinates, so the second block is generated only for those.
+// In both modes the fast path uses the leading 16 bits h of r (the centre of the interval of r they leave) and
+// sends a coordinate to the exact routine when the outcome could depend on the remaining bits.
+struct RoundK {
+  float rn;                              // RN(1 / norm)
+  float thr;                             // negative: every coordinate goes to the exact routine
+  float nqs, magic;
+  uint32_t bin_mask, bin_lane;
+};
+
+__device__ __forceinline__ RoundK round_k(const RoundTable& rt, float norm) {
+  const bool ok = rt.usable && norm > 7.9e-31f && norm < 1.2e30f;
+  RoundK c;
+  c.rn = ok ? __frcp_rn(norm) : 0.0f;
+  c.thr = ok ? rt.thr16 : -1.0f;
+  c.nqs = rt.neg_qscale16;
+  c.magic = rt.magic;
+  const uint32_t copy_bytes = 16u << (rt.key_shift - kKeyShiftMin);
+  c.bin_mask = ~(copy_bytes - 1u);
+  c.bin_lane = ((threadIdx.x & 31u) << 4) & (copy_bytes - 1u);
+  return c;
+}
+
+// One coordinate: returns S * (signed level index) as a float (the level of x, negative for negative x), and ORs
+// into *unsafe whether the exact routine has to decide.  hbits = pattern of the float 2^23 + h.  binz = the bin
+// table's address (entries with a16) minus kBinAddrBase bytes.
+__device__ __forceinline__ float round_signed(float x, uint32_t hbits, const RoundK& c, const char* binz, bool* unsafe) {
+  const float u2 = fmaf(fabsf(x), c.rn, kRoundShift);
+  const uint32_t off = ((__float_as_uint(u2) >> kBinAddrShift) & c.bin_mask) | c.bin_lane;
+  const float4 e = *reinterpret_cast<const float4*>(binz + off);
+  const float t1 = fmaf(__uint_as_float(hbits), c.nqs, e.x);                       // exact: both are multiples of S 2^-16
+  float X = fmaf(u2, e.y, t1);
+  X = fmaf(__saturatef(__fsub_rn(u2, e.z)), e.w, X);                               // S (F - r~) + S / 2
+  const float sg = __uint_as_float((__float_as_uint(x) & 0x80000000u) | 0x3f800000u);
+  const float Z = fmaf(X, sg, c.magic);
+  const float zi = __fsub_rn(Z, c.magic);                                          // the nearest multiple of S, signed
+  const float rho = fmaf(X, sg, -zi);
+  *unsafe = *unsafe || (fabsf(rho) > c.thr);
+  return zi;
+}
+
+// The variate bits of coordinate e (its index in the generator's counter space) on their own: the 24 bits of
+// QGX_RNG_WORD24 or the 32 bits of QGX_RNG_HALF32.  One or two whole blocks per call: for ragged ends only.
+template <int RNG>
+static __device__ __noinline__ uint32_t variate_bits(uint64_t e, uint32_t k, uint32_t xid, const PhiloxKey& key) {
+  if (RNG == QGX_RNG_WORD24) {
+    const uint64_t q = e >> 2;
+    const uint4 w = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), k, xid, key);
+    const int c = (int)(e & 3u);
+    return (c == 0 ? w.x : (c == 1 ? w.y : (c == 2 ? w.z : w.w))) >> 8;
+  }
+  const uint64_t o = e >> 3;
+  const uint4 w = philox4x32_10((uint32_t)o, (uint32_t)(o >> 32), k, xid, key);
+  const uint4 w2 = philox4x32_10((uint32_t)o, (uint32_t)(o >> 32), k | 0x80000000u, xid, key);
+  const int j = (int)(e & 7u);
+  const uint32_t x = (j >> 1) == 0 ? w.x : ((j >> 1) == 1 ? w.y : ((j >> 1) == 2 ? w.z : w.w));
+  const uint32_t y = (j >> 1) == 0 ? w2.x : ((j >> 1) == 1 ? w2.y : ((j >> 1) == 2 ? w2.z : w2.w));
+  const uint32_t h = (j & 1) ? (x >> 16) : (x & 0xffffu), h2 = (j & 1) ? (y >> 16) : (y & 0xffffu);
+  return (h << 16) | h2;
+}
+
+// Definition 1 for one coordinate with the variate of either mode: rbits = the 24-bit variate (QGX_RNG_WORD24) or
+// the 32-bit variate (QGX_RNG_HALF32).  Out of line: it runs for about 1e-4 of the coordinates.
+template <int RNG>
+static __device__ __noinline__ int quantize_level_exact(float absv, float norm, const float* lev, int nlev, uint32_t rbits) {
+  float u = (norm > 0.0f) ? __fdiv_rn(absv, norm) : 0.0f;
+  u = fminf(u, 1.0f);
+  int tau = 0;
+  for (int j = 1; j <= nlev - 2; ++j) tau = (lev[j] <= u) ? j : tau;
+  const float num = __fsub_rn(u, lev[tau]);
+  const float den = __fsub_rn(lev[tau + 1], lev[tau]);
+  const float xi = __fdiv_rn(num, den);
+  bool up;
+  if (RNG == QGX_RNG_WORD24) {
+    const float r = __fmul_rn(__uint2float_rn(rbits), 5.9604644775390625e-8f);    // exact
+    up = r < xi;
+  } else {
+    const double r = (double)rbits * 2.3283064365386962890625e-10;                 // exact
+    up = r < (double)xi;
+  }
+  return tau + (up ? 1 : 0);
 }
 
 __device__ __forceinline__ uint32_t symbol_of(float v, int idx) {

@@ -100,8 +100,8 @@ __global__ void __launch_bounds__(256) k_half_from_mean(const float* __restrict_
     Xhalf[i] = __fsub_rn(X[i], __fmul_rn(gamma, m[i]));
 }
 
-static unsigned grid_for(size_t n, int threads) {
-  return (unsigned)std::max<size_t>(1, std::min<size_t>((n + threads - 1) / threads, 148 * 8));
+static unsigned grid_for(const qgx_ctx* c, size_t n, int threads) {
+  return (unsigned)std::max<size_t>(1, std::min<size_t>((n + threads - 1) / threads, (size_t)c->num_sms * 8));
 }
 
 qgx_status apply_operator_impl(qgx_ctx* c, const qgx_operator* op, const float* x, float* out) {
@@ -110,17 +110,17 @@ qgx_status apply_operator_impl(qgx_ctx* c, const qgx_operator* op, const float* 
   ScopedKernelTimer timer(c, QGX_KERNEL_OPERATOR);
   if (op->kind == QGX_OP_DENSE_AFFINE) {
     const bool vec_ok = (d % 4 == 0) && ((reinterpret_cast<uintptr_t>(op->mat) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(x) & 15u) == 0);
-    k_gemv_rows<<<grid_for(d * 32, 256), 256, 0, c->stream>>>(op->mat, d, d, x, op->bias, out, vec_ok);
+    k_gemv_rows<<<grid_for(c, d * 32, 256), 256, 0, c->stream>>>(op->mat, d, d, x, op->bias, out, vec_ok);
     count_launch(c);
   } else if (op->kind == QGX_OP_BILINEAR) {
     if (d % 2) return QGX_ERR_INVALID_ARG;
     const size_t n = d / 2;
     const bool vec_ok = (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(op->mat) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(x + n) & 15u) == 0);
-    k_gemv_rows<<<grid_for(n * 32, 256), 256, 0, c->stream>>>(op->mat, n, n, x + n, nullptr, out, vec_ok);
+    k_gemv_rows<<<grid_for(c, n * 32, 256), 256, 0, c->stream>>>(op->mat, n, n, x + n, nullptr, out, vec_ok);
     k_gemv_cols_neg<<<(unsigned)((n + 31) / 32), dim3(32, 32), 0, c->stream>>>(op->mat, n, x, out + n);
     count_launch(c, 2);
   } else if (op->kind == QGX_OP_DIAGONAL) {
-    k_diag<<<grid_for(d, 256), 256, 0, c->stream>>>(op->mat, x, out, d);
+    k_diag<<<grid_for(c, d, 256), 256, 0, c->stream>>>(op->mat, x, out, d);
     count_launch(c);
   } else {
     return QGX_ERR_INVALID_ARG;
@@ -143,7 +143,7 @@ qgx_status qgx_eg_init(qgx_ctx* c, qgx_eg_state* st) {
   if (!c || !st || !st->X || !st->Y || !st->Xbar || !st->Xhalf || !st->anchor || !st->scalars || st->d < 1 || st->K < 1)
     return QGX_ERR_INVALID_ARG;
   if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
-  k_eg_init<<<grid_for(st->d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->anchor, st->scalars, st->d, st->K);
+  k_eg_init<<<grid_for(c, st->d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->anchor, st->scalars, st->d, st->K);
   count_launch(c);
   st->t = 1;
   return cuda_status(cudaGetLastError());
@@ -191,7 +191,7 @@ static qgx_status eg_step_impl(qgx_ctx* c, qgx_eg_state* st, const qgx_operator*
   if (rc != QGX_OK) return rc;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);
-    k_eg_finish<<<grid_for(d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->Xhalf, st->anchor, st->scalars, d, K, st->t);
+    k_eg_finish<<<grid_for(c, d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->Xhalf, st->anchor, st->scalars, d, K, st->t);
   }
   count_launch(c);
   st->t += 1;
@@ -229,7 +229,7 @@ qgx_status qgx_family_step(qgx_ctx* c, qgx_eg_state* st, int method, const qgx_o
 
   if (method == QGX_METHOD_OPTDA && st->t > 1) {
     ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);
-    k_half_from_mean<<<grid_for(d, 256), 256, 0, c->stream>>>(st->X, mean_prev, st->scalars, st->Xhalf, d);   // g_{k,t-1/2}
+    k_half_from_mean<<<grid_for(c, d, 256), 256, 0, c->stream>>>(st->X, mean_prev, st->scalars, st->Xhalf, d);   // g_{k,t-1/2}
     count_launch(c);
   } else {                                                                       // no earlier feedback: X_{t+1/2} = X_t
     if (cudaMemcpyAsync(st->Xhalf, st->X, sizeof(float) * d, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
@@ -253,7 +253,7 @@ qgx_status qgx_family_step(qgx_ctx* c, qgx_eg_state* st, int method, const qgx_o
   if (rc != QGX_OK) return rc;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_FINISH);
-    k_eg_finish<<<grid_for(d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->Xhalf, st->anchor, st->scalars, d, K, st->t);
+    k_eg_finish<<<grid_for(c, d, 256), 256, 0, c->stream>>>(st->X, st->Y, st->Xbar, st->Xhalf, st->anchor, st->scalars, d, K, st->t);
   }
   count_launch(c);
   st->t += 1;

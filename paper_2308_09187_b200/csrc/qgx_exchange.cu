@@ -4,8 +4,11 @@
 #include "qgx_bucket.cuh"
 #include "qgx_codec.cuh"
 
+#include <cuda.h>
+
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -78,6 +81,8 @@ struct EncodeArgs {
   unsigned long long* status;   // [K][nb], zeroed before the launch
   unsigned int* ticket;         // zeroed before the launch
   DevStatus* st;
+  size_t nb_whole;              // buckets [0, nb_whole) of every worker belong to k_encode_staged ...
+  size_t b_first;               // ... and buckets [b_first, nb) to k_exchange_encode
 };
 
 // Norm of the bucket held by the CTA, one barrier: per-warp partials go to shared memory and every
@@ -166,18 +171,94 @@ __device__ __forceinline__ void load_bucket_octets(BucketRegs<2 * P>& r, const D
   }
 }
 
+// ---- rounding of one octet (eight consecutive coordinates of one lane) ---------------------------
+// The rare way through an octet, out of line: every coordinate is tested again and the ones whose outcome the
+// leading variate bits do not settle go through the exact routine.  Returns the eight signed level indices, one
+// per byte.
+template <int RNG>
+static __device__ __noinline__ uint64_t redo_octet(const float4 xa, const float4 xb, const uint4 w0, const uint4 w1, uint64_t oct,
+                                                   uint32_t k, uint32_t xid, const PhiloxKey* key, const RoundK rc, float norm,
+                                                   const char* binz, const float* lev, int nlev) {
+  const float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+  const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+  const float inv_S = -1.0f / (rc.nqs * 65536.0f);
+  uint4 w2 = make_uint4(0u, 0u, 0u, 0u);
+  bool have2 = false;
+  uint64_t out = 0;
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t h = RNG == QGX_RNG_HALF32 ? ((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xffffu)) : (w[i] >> 16);
+    bool unsafe = false;
+    const float zi = round_signed(x[i], 0x4B000000u | h, rc, binz, &unsafe);
+    int idx = (int)fabsf(__fmul_rn(zi, inv_S));
+    if (unsafe) {
+      uint32_t rb;
+      if (RNG == QGX_RNG_HALF32) {
+        if (!have2) { w2 = philox4x32_10((uint32_t)oct, (uint32_t)(oct >> 32), k | 0x80000000u, xid, *key); have2 = true; }
+        const uint32_t y = (i >> 1) == 0 ? w2.x : ((i >> 1) == 1 ? w2.y : ((i >> 1) == 2 ? w2.z : w2.w));
+        rb = (h << 16) | ((i & 1) ? (y >> 16) : (y & 0xffffu));
+      } else {
+        rb = w[i] >> 8;
+      }
+      idx = quantize_level_exact<RNG>(fabsf(x[i]), norm, lev, nlev, rb);
+    }
+    const int sidx = (__float_as_uint(x[i]) >> 31) ? -idx : idx;
+    out |= (uint64_t)(uint8_t)(signed char)sidx << (8 * i);
+  }
+  return out;
+}
+
+// S * (signed level index) of the eight coordinates xa, xb of octet `oct` (its index in the generator's counter
+// space) of worker k.  S = the scale of the rounding table.
+template <int RNG>
+__device__ __forceinline__ void octet_levels(const float4 xa, const float4 xb, uint64_t oct, uint32_t k, uint32_t xid,
+                                             const PhiloxKey& key, const RoundK& rc, float norm, float S, const char* binz,
+                                             const float* lev, int nlev, float* z) {
+  constexpr uint32_t kTwo23 = 0x4B000000u;              // pattern of 2^23: its low mantissa bytes are replaced by h
+  const float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+  uint4 w0, w1;
+  uint32_t hb[8];
+  if (RNG == QGX_RNG_HALF32) {
+    w0 = philox4x32_10((uint32_t)oct, (uint32_t)(oct >> 32), k, xid, key);
+    w1 = w0;
+    hb[0] = prmt(w0.x, kTwo23, 0x7610u); hb[1] = prmt(w0.x, kTwo23, 0x7632u);
+    hb[2] = prmt(w0.y, kTwo23, 0x7610u); hb[3] = prmt(w0.y, kTwo23, 0x7632u);
+    hb[4] = prmt(w0.z, kTwo23, 0x7610u); hb[5] = prmt(w0.z, kTwo23, 0x7632u);
+    hb[6] = prmt(w0.w, kTwo23, 0x7610u); hb[7] = prmt(w0.w, kTwo23, 0x7632u);
+  } else {
+    philox4x32_10_x2(2ull * oct, 2ull * oct + 1ull, k, xid, key, &w0, &w1);
+    hb[0] = prmt(w0.x, kTwo23, 0x7632u); hb[1] = prmt(w0.y, kTwo23, 0x7632u);
+    hb[2] = prmt(w0.z, kTwo23, 0x7632u); hb[3] = prmt(w0.w, kTwo23, 0x7632u);
+    hb[4] = prmt(w1.x, kTwo23, 0x7632u); hb[5] = prmt(w1.y, kTwo23, 0x7632u);
+    hb[6] = prmt(w1.z, kTwo23, 0x7632u); hb[7] = prmt(w1.w, kTwo23, 0x7632u);
+  }
+  bool unsafe = false;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) z[i] = round_signed(x[i], hb[i], rc, binz, &unsafe);
+  if (unsafe) {                                         // some coordinate of the octet needs the exact routine
+    const uint64_t fixed = redo_octet<RNG>(xa, xb, w0, w1, oct, k, xid, &key, rc, norm, binz, lev, nlev);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) z[i] = __fmul_rn((float)(int)(signed char)(uint8_t)(fixed >> (8 * i)), S);
+  }
+}
+
+// the pair table's byte offset for two consecutive coordinates: 4 * ((first + 64 * second) mod 4096)
+__device__ __forceinline__ uint32_t pair_offset(float z_first, float z_second, float four_over_S) {
+  const float t = fmaf(z_second, 64.0f * four_over_S, fmaf(z_first, four_over_S, 12582912.0f));   // 1.5 * 2^23 + 4 first + 256 second
+  return __float_as_uint(t) & 0x3ffcu;
+}
+
 // One persistent CTA per SM slot; each ticket is one bucket (k = ticket % K, b = ticket / K).
 //   loads, zero the image | barrier | norm, Philox, rounding, packing, sub-block lengths, warp scans |
 //   barrier | warp offsets, bit scatter, look-back (warp 0) | barrier | copy out
 // The bucket image is double buffered, so the copy-out of one bucket needs no barrier before the next
 // bucket starts.  A thread works on P octets; warp w owns the 256 * P coordinates [w * 256 * P, ...).
-template <int P, int G>
+template <int P, int G, int RNG>
 __global__ void __launch_bounds__(P == 1 ? 256 : 512, P == 1 ? 4 : 2)
 k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
                   const __grid_constant__ RoundTable rt) {
   extern __shared__ __align__(16) uint32_t s_dyn[];
-  __shared__ float4 s_bin[kKeyBins];
+  __shared__ float4 s_bin[kBinEntries];
   __shared__ EncLut s_lut;
   __shared__ uint32_t s_pair[kPairLutSize];
   __shared__ float s_lev[QGX_MAX_LEVELS];
@@ -190,26 +271,28 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   // words of one image, a multiple of 4 so that both images are 16-byte aligned
   const int img_words = (int)((((((uint32_t)a.bucket * (uint32_t)(ct.maxlen + 1) + 16u * (uint32_t)(a.bucket / G + 1) + kNormBits + 31u) >> 5) + 4) + 3u) & ~3u);
-  const unsigned long long total = (unsigned long long)a.nb * (unsigned long long)a.K;
+  const unsigned long long total = (unsigned long long)(a.nb - a.b_first) * (unsigned long long)a.K;
   constexpr int kOctet = 2 * kQuad;
   constexpr int kSegLanes = G / kOctet;                 // lanes per sub-block within a row of 256 coordinates
   constexpr int kSegs = 32 / kSegLanes;                 // sub-blocks per row
 
   fill_enc_lut(&s_lut, ct);
-  fill_bin_table(s_bin, rt);
+  fill_bin_table(s_bin, rt, true);
   if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 1.0f;
   if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
   for (int i = threadIdx.x; i < 2 * img_words; i += blockDim.x) s_dyn[i] = 0;
   __syncthreads();
-  fill_pair_lut(s_pair, &s_lut);
+  fill_pair_lut_signed(s_pair, &s_lut);
   __syncthreads();
   const int nlev = lt.nlev;
+  const char* binz = reinterpret_cast<const char*>(s_bin) - kBinAddrBase;
+  const float S = -rt.neg_qscale16 * 65536.0f, four_over_S = 4.0f / S;
   uint32_t used_words[2] = {0u, 0u};                    // words of each image that the last bucket in it dirtied
 
   for (int par = 0;; par ^= 1) {
     const unsigned long long t = s_ticket[par];
     if (t >= total) break;
-    const size_t b = (size_t)(t / (unsigned long long)a.K), k = (size_t)(t % (unsigned long long)a.K);
+    const size_t b = a.b_first + (size_t)(t / (unsigned long long)a.K), k = (size_t)(t % (unsigned long long)a.K);
     const size_t lo = b * (size_t)a.bucket;
     const int len = (int)min((size_t)a.bucket, a.d - lo);
     uint32_t* s_img = s_dyn + par * img_words;
@@ -224,7 +307,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     const float norm = bucket_norm_all<2 * P>(r, a.norm_type, s_red[par]);   // barrier inside: the image is zero
     const bool finite = (norm - norm) == 0.0f;
-    const RoundConsts rc = round_consts(rt, norm);
+    const RoundK rc = round_k(rt, norm);
     if (threadIdx.x == 0) {
       a.norms[k * a.nb + b] = norm;
       if (!finite) latch_error(a.st, QGX_ERR_NONFINITE);
@@ -232,49 +315,50 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     const uint32_t nsub = (uint32_t)((len + G - 1) / G);
     const uint32_t hdr_bits = kNormBits + 16u * nsub;
-    const bool whole = (len == a.bucket) && a.vec_ok && (a.bucket % (32 * kOctet * P) == 0);   // every lane holds full octets: no checks
+    // every lane holds full octets that are octets of the generator's counter space too: no checks
+    const bool whole = (len == a.bucket) && a.vec_ok && (a.bucket % (32 * kOctet * P) == 0) && (((a.quad_base + (uint64_t)(lo >> 2)) & 1ull) == 0);
     const bool live = finite && norm != 0.0f;             // otherwise every coordinate is level 0
+    const uint64_t oct0 = (a.quad_base + (uint64_t)(lo >> 2)) >> 1;   // the bucket's first octet in the counter space (when `whole`)
 
     uint64_t qbits[2 * P];
     uint32_t qn[P], qoff[P];                              // qn: bits of the first quad | bits of the second << 8
-    if (whole && live) {                                  // the common case, without per-quad decisions
+    if (whole && live) {                                  // the common case, without per-coordinate decisions
 #pragma unroll
       for (int j = 0; j < P; ++j) {
         const int o = (warp * P + j) * 32 + lane;
-        const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + 2ull * (uint64_t)o;
-        uint4 w0, w1;
-        philox4x32_10_x2(ctr, ctr + 1ull, (uint32_t)k, a.xid, key, &w0, &w1);
-        const uint32_t code0 = quantize_quad_codes(r.x[2 * j], w0, rc, norm, s_bin, s_lev, nlev);
-        const uint32_t code1 = quantize_quad_codes(r.x[2 * j + 1], w1, rc, norm, s_bin, s_lev, nlev);
+        float z[8];
+        octet_levels<RNG>(r.x[2 * j], r.x[2 * j + 1], oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, binz, s_lev, nlev, z);
+        const char* pz = reinterpret_cast<const char*>(s_pair);
+        const uint32_t e01 = *reinterpret_cast<const uint32_t*>(pz + pair_offset(z[0], z[1], four_over_S));
+        const uint32_t e23 = *reinterpret_cast<const uint32_t*>(pz + pair_offset(z[2], z[3], four_over_S));
+        const uint32_t e45 = *reinterpret_cast<const uint32_t*>(pz + pair_offset(z[4], z[5], four_over_S));
+        const uint32_t e67 = *reinterpret_cast<const uint32_t*>(pz + pair_offset(z[6], z[7], four_over_S));
         uint32_t n0, n1;
-        pack_quad_codes(code0, s_pair, &qbits[2 * j], &n0);
-        pack_quad_codes(code1, s_pair, &qbits[2 * j + 1], &n1);
+        pack_pair_entries(e01, e23, &qbits[2 * j], &n0);
+        pack_pair_entries(e45, e67, &qbits[2 * j + 1], &n1);
         qn[j] = n0 | (n1 << 8);
       }
     } else {
 #pragma unroll
-    for (int j = 0; j < P; ++j) {
-      const int o = (warp * P + j) * 32 + lane;           // octet of the bucket
-      const int nv0 = whole ? kQuad : max(0, min(kQuad, len - o * kOctet));
-      const int nv1 = whole ? kQuad : max(0, min(kQuad, len - o * kOctet - kQuad));
-      uint32_t code0 = 0, code1 = 0;
-      if (live && nv0 > 0) {
-        const uint64_t ctr = a.quad_base + (uint64_t)(lo >> 2) + 2ull * (uint64_t)o;
-        uint4 w0, w1;
-        philox4x32_10_x2(ctr, ctr + 1ull, (uint32_t)k, a.xid, key, &w0, &w1);
-        code0 = quantize_quad_codes(r.x[2 * j], w0, rc, norm, s_bin, s_lev, nlev);
-        code1 = quantize_quad_codes(r.x[2 * j + 1], w1, rc, norm, s_bin, s_lev, nlev);
+      for (int j = 0; j < P; ++j) {
+        const int o = (warp * P + j) * 32 + lane;           // octet of the bucket
+        const int nv = whole ? kOctet : max(0, min(kOctet, len - o * kOctet));
+        uint32_t sy[2] = {0u, 0u};                          // symbol bytes (level | sign << 7) of the two quads
+        if (live && nv > 0) {
+          const uint64_t e0 = 4ull * (a.quad_base + (uint64_t)(lo >> 2)) + (uint64_t)o * kOctet;   // first coordinate in the counter space
+          const float x[8] = {r.x[2 * j].x, r.x[2 * j].y, r.x[2 * j].z, r.x[2 * j].w,
+                              r.x[2 * j + 1].x, r.x[2 * j + 1].y, r.x[2 * j + 1].z, r.x[2 * j + 1].w};
+          for (int i = 0; i < nv; ++i) {                    // ragged ends and odd offsets: the exact routine throughout
+            const uint32_t rb = variate_bits<RNG>(e0 + (uint64_t)i, (uint32_t)k, a.xid, key);
+            const int idx = quantize_level_exact<RNG>(fabsf(x[i]), norm, s_lev, nlev, rb);
+            sy[i >> 2] |= symbol_of(x[i], idx) << (8 * (i & 3));
+          }
+        }
+        uint32_t n0, n1;
+        pack_quad(sy[0], min(nv, kQuad), &s_lut, &qbits[2 * j], &n0);
+        pack_quad(sy[1], max(nv - kQuad, 0), &s_lut, &qbits[2 * j + 1], &n1);
+        qn[j] = n0 | (n1 << 8);
       }
-      uint32_t n0, n1;
-      if (nv1 == kQuad) {
-        pack_quad_codes(code0, s_pair, &qbits[2 * j], &n0);
-        pack_quad_codes(code1, s_pair, &qbits[2 * j + 1], &n1);
-      } else {                                              // the ragged end of a bucket
-        pack_quad((code0 & 0x1f1f1f1fu) | ((code0 & 0x20202020u) << 2), nv0, &s_lut, &qbits[2 * j], &n0);
-        pack_quad((code1 & 0x1f1f1f1fu) | ((code1 & 0x20202020u) << 2), nv1, &s_lut, &qbits[2 * j + 1], &n1);
-      }
-      qn[j] = n0 | (n1 << 8);
-    }
     }
     // warp scans of the bit counts, two rows per 32-bit word (a row holds at most 32 * 104 bits);
     // qoff[j] becomes the octet's bit offset inside the warp's part of the payload
@@ -345,6 +429,12 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     // two more barriers
   }
 }
+
+}  // namespace qgx
+
+#include "qgx_encode_staged.cuh"
+
+namespace qgx {
 
 // ---- decode + average ------------------------------------------------------------------------
 // Decoder table of the fused path: index = the next maxlen + 1 stream bits (codeword, then the sign
@@ -502,7 +592,9 @@ __device__ __forceinline__ SubBlockAt find_subblock(const DecodeArgs& a, int k, 
   uint32_t st, row_before, row_bits;
   r.ok = locate_subblock(a.stream + (size_t)k * a.cap_words, a.cap_words, a.bucket_bits, a.offsets, (size_t)k * a.nb + b,
                          hdr_bits, s, exists, uniform, lane, &w, &r.norm, &st, &r.want, &row_before, &row_bits);
-  if (!r.ok) { st = 0; r.want = 0; r.norm = 0.0f; }
+  // a bucket whose numbers disagree is reported, and its walk reads the start of the worker's stream instead
+  // (in range whatever the offsets say)
+  if (!r.ok) { st = 0; r.want = 0; r.norm = 0.0f; w = a.stream + (size_t)k * a.cap_words; }
   r.p = w + (st >> 5);
   r.sh = st & 31u;
   // bucket-level validity is the same for all lanes; the lengths are bounded, so the row is at most 2^19 bits
@@ -764,7 +856,8 @@ constexpr int kTableCacheSlots = 32;
 struct LaunchShape { size_t smem; int per_sm; };      // smem == 0: not asked yet
 struct TableCache {
   CachedTables e[kTableCacheSlots];
-  LaunchShape enc[3][3];                // [octets per thread 1, 2, 4][sub-block 32, 64, 128]
+  LaunchShape enc[2][3][3];             // [variate mode][octets per thread 1, 2, 4][sub-block 32, 64, 128]
+  LaunchShape enc_staged[2][3];         // [variate mode][sub-block]
   LaunchShape dec[3][6];                // [sub-block][symbol mode]
 };
 
@@ -858,6 +951,33 @@ static qgx_status cached_tables(qgx_ctx* c, const qgx_quant_cfg* cfg, const Cach
   return QGX_OK;
 }
 
+// Tensor map of `rows` rows of 32 floats (128 bytes) starting at base, copied `box_rows` rows at a time with the
+// 128-byte swizzle: what k_encode_staged's bulk copies read.  The encoder of the map is a driver entry point,
+// looked up once (the library does not link the driver).
+static bool make_rows_map(const float* base, unsigned long long rows, unsigned box_rows, CUtensorMap* out) {
+  typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static encode_fn encode = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+      encode = reinterpret_cast<encode_fn>(fn);
+    else
+      cudaGetLastError();
+  });
+  if (!encode || rows == 0) return false;
+  const cuuint64_t gdim[2] = {(cuuint64_t)kLaneCoords, (cuuint64_t)rows};
+  const cuuint64_t gstride[1] = {(cuuint64_t)(kLaneCoords * sizeof(float))};
+  const cuuint32_t box[2] = {(cuuint32_t)kLaneCoords, (cuuint32_t)box_rows};
+  const cuuint32_t estride[2] = {1u, 1u};
+  return encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), gdim, gstride, box, estride,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // The whole exchange.  sym_mode 1 keeps the decoded symbols (and the norms) in the workspace; sym_mode 2
 // adds sum_k ||vhat_k kept by the other slot - vhat_k decoded in this exchange||^2 to *sum_sq.
 qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t xid, int slot,
@@ -868,6 +988,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const int bucket = cfg->bucket;
   if (bucket < kQuad || bucket > QGX_MAX_BUCKET || bucket % kQuad != 0) return QGX_ERR_INVALID_ARG;
   if (cfg->norm_type != QGX_NORM_L2 && cfg->norm_type != QGX_NORM_LINF) return QGX_ERR_INVALID_ARG;
+  if (cfg->rng_mode != QGX_RNG_WORD24 && cfg->rng_mode != QGX_RNG_HALF32) return QGX_ERR_INVALID_ARG;
   if (check_levels_host(cfg->levels, cfg->nlev) != QGX_OK) return QGX_ERR_BAD_LEVELS;
   if (cfg->cb.nlev != cfg->nlev) return QGX_ERR_INVALID_ARG;
   if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
@@ -932,19 +1053,24 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const size_t img_words = (((((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4) + 3) & ~(size_t)3;
   const size_t smem = sizeof(uint32_t) * 2 * img_words;   // two images: see k_exchange_encode
   int per_sm = 1;
-#define QGX_LAUNCH_E(V, GG)                                                                                    \
+#define QGX_LAUNCH_ER(V, GG, RR)                                                                               \
   do {                                                                                                         \
-    allow_max_dynamic_smem(k_exchange_encode<V, GG>, c->device);                                               \
-    LaunchShape& shape = table_cache(c)->enc[V == 1 ? 0 : (V == 2 ? 1 : 2)][GG == 32 ? 0 : (GG == 64 ? 1 : 2)];  \
-    if (shape.smem != smem + 1 + (size_t)threads * 0x100000) {   /* occupancy asked once per shape */              \
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG>, threads, smem);         \
+    allow_max_dynamic_smem(k_exchange_encode<V, GG, RR>, c->device);                                           \
+    LaunchShape& shape = table_cache(c)->enc[RR][V == 1 ? 0 : (V == 2 ? 1 : 2)][GG == 32 ? 0 : (GG == 64 ? 1 : 2)];  \
+    if (shape.smem != smem + 1 + (size_t)threads * 0x100000) {   /* occupancy asked once per shape */          \
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG, RR>, threads, smem);     \
       shape.smem = smem + 1 + (size_t)threads * 0x100000;                                                      \
       shape.per_sm = per_sm < 1 ? 1 : per_sm;                                                                  \
     }                                                                                                          \
     per_sm = shape.per_sm;                                                                                     \
-    const unsigned long long want = (unsigned long long)nb * (unsigned long long)K;                            \
-    const unsigned grid = (unsigned)std::min<unsigned long long>(want, 148ull * (unsigned long long)per_sm);   \
-    k_exchange_encode<V, GG><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                          \
+    const unsigned long long want = (unsigned long long)(nb - ea.b_first) * (unsigned long long)K;             \
+    const unsigned grid = (unsigned)std::min<unsigned long long>(want, (unsigned long long)c->num_sms * (unsigned long long)per_sm);   \
+    k_exchange_encode<V, GG, RR><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                     \
+  } while (0)
+#define QGX_LAUNCH_E(V, GG)                                          \
+  do {                                                               \
+    if (cfg->rng_mode == QGX_RNG_HALF32) QGX_LAUNCH_ER(V, GG, 1);    \
+    else QGX_LAUNCH_ER(V, GG, 0);                                    \
   } while (0)
 #define QGX_LAUNCH_EG(V)                                   \
   do {                                                     \
@@ -952,17 +1078,65 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
     else if (ct.G == 64) QGX_LAUNCH_E(V, 64);              \
     else QGX_LAUNCH_E(V, 128);                             \
   } while (0)
+  // Whole buckets of a multiple of 1024 coordinates that divides 16384 go through the staged kernel; what is left
+  // (a short last bucket, other bucket sizes, unaligned vectors) through the bucket-in-registers kernel.
+  bool staged_ok = ea.vec_ok && bucket % kWarpCoords == 0 && kStageCoords % bucket == 0 && coord_base % 8 == 0 &&
+                   c->encode_path != QGX_ENCODE_REGISTERS && d / (size_t)bucket > 0;
+  CUtensorMap tmap;
+  std::memset(&tmap, 0, sizeof(tmap));
+  if (staged_ok) {
+    // the staged source: the workers' rows (worker k at k * ld) or, without them, the shared vector a
+    const size_t ldv = src.ld ? src.ld : d;
+    const size_t whole = (d / (size_t)bucket) * (size_t)bucket;
+    const float* base = src.v ? src.v : src.a;
+    const unsigned long long floats = src.v ? (unsigned long long)(K - 1) * ldv + whole : whole;
+    staged_ok = (!src.v || ldv % kLaneCoords == 0) &&
+                make_rows_map(base, floats / kLaneCoords, (unsigned)std::min(256, bucket / kLaneCoords), &tmap);
+  }
+  ea.nb_whole = staged_ok ? d / (size_t)bucket : 0;
+  ea.b_first = ea.nb_whole;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_ENCODE);
-    switch (pp) {
-      case 1: QGX_LAUNCH_EG(1); break;
-      case 2: QGX_LAUNCH_EG(2); break;
-      default: QGX_LAUNCH_EG(4); break;
+    if (ea.nb_whole > 0) {
+      const size_t smem_st = sizeof(float) * kStageCoords * kStageBuffers;
+      const unsigned long long per_group = (unsigned long long)(kStageCoords / bucket);
+      const unsigned long long groups = ((unsigned long long)ea.nb_whole * (unsigned long long)K + per_group - 1ull) / per_group;
+#define QGX_LAUNCH_S(GG, RR)                                                                                         \
+  do {                                                                                                               \
+    allow_max_dynamic_smem(k_encode_staged<GG, RR>, c->device);                                                      \
+    LaunchShape& shape = table_cache(c)->enc_staged[RR][GG == 32 ? 0 : (GG == 64 ? 1 : 2)];                          \
+    if (shape.smem == 0) {                                                                                           \
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_encode_staged<GG, RR>, kStagedThreads, smem_st);      \
+      shape.smem = 1;                                                                                                \
+      shape.per_sm = per_sm < 1 ? 1 : per_sm;                                                                        \
+    }                                                                                                                \
+    const unsigned grid = (unsigned)std::min<unsigned long long>((groups + 1ull) / 2ull, (unsigned long long)c->num_sms * (unsigned long long)shape.per_sm); \
+    k_encode_staged<GG, RR><<<grid, kStagedThreads, smem_st, c->stream>>>(ea, lt, ct, key, qt, tmap);                \
+  } while (0)
+#define QGX_LAUNCH_SG(GG)                                            \
+  do {                                                               \
+    if (cfg->rng_mode == QGX_RNG_HALF32) QGX_LAUNCH_S(GG, 1);        \
+    else QGX_LAUNCH_S(GG, 0);                                        \
+  } while (0)
+      if (ct.G == 32) QGX_LAUNCH_SG(32);
+      else if (ct.G == 64) QGX_LAUNCH_SG(64);
+      else QGX_LAUNCH_SG(128);
+#undef QGX_LAUNCH_SG
+#undef QGX_LAUNCH_S
+      count_launch(c);
+    }
+    if (ea.b_first < nb) {
+      switch (pp) {
+        case 1: QGX_LAUNCH_EG(1); break;
+        case 2: QGX_LAUNCH_EG(2); break;
+        default: QGX_LAUNCH_EG(4); break;
+      }
+      count_launch(c);
     }
   }
 #undef QGX_LAUNCH_EG
 #undef QGX_LAUNCH_E
-  count_launch(c);
+#undef QGX_LAUNCH_ER
   if (cudaGetLastError() != cudaSuccess) return QGX_ERR_CUDA;
   if (total_bits_out &&
       cudaMemcpyAsync(total_bits_out, tot, sizeof(uint64_t) * (size_t)K, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
@@ -981,7 +1155,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const size_t total_sub = nb * (size_t)(bucket / ct.G);
   da.values = nullptr;
   const bool fits = (size_t)K * d * sizeof(float) <= ((size_t)256 << 20);
-  const bool small = total_sub * 2 < (size_t)148 * kDecThreads * 4;
+  const bool small = total_sub * 2 < (size_t)c->num_sms * kDecThreads * 4;
   if (K > 1 && fits && c->decode_split != QGX_SPLIT_NEVER && (small || c->decode_split == QGX_SPLIT_ALWAYS)) {
     da.values = (float*)ws_get(c, WS_VALUES, sizeof(float) * (size_t)K * d);
     if (!da.values) return QGX_ERR_CUDA;
@@ -990,7 +1164,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   if (rc != QGX_OK || !da.values) return rc;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
-    const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>((d + 255) / 256, (size_t)148 * 8));
+    const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>((d + 255) / 256, (size_t)c->num_sms * 8));
     k_sum_workers<<<grid, 256, 0, c->stream>>>(da.values, K, d, mean_out, da.update, da.xin, da.xout, da.scalars);
   }
   count_launch(c);
@@ -1014,7 +1188,7 @@ static qgx_status launch_decode_gs(qgx_ctx* c, const DecodeArgs& da, const CodeT
       shape.per_sm = per_sm < 1 ? 1 : per_sm;
     }
     per_sm = shape.per_sm;
-    const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)148 * per_sm));
+    const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)c->num_sms * per_sm));
     k_exchange_decode<G, SYM><<<grid, kDecThreads, lut_bytes, c->stream>>>(da, ct, lt);
   }
   count_launch(c);
@@ -1092,6 +1266,8 @@ static SegChildren* seg_children(qgx_ctx* c) {
     h->device = c->device;
     h->sym_slot = -1;
     h->decode_split = c->decode_split;
+    h->encode_path = c->encode_path;
+    h->num_sms = c->num_sms;
     h->dstatus = c->dstatus;                            // errors latch into the parent's status block
     if (cudaStreamCreateWithFlags(&h->stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&sc->join[i], cudaEventDisableTiming) != cudaSuccess) {
@@ -1124,6 +1300,12 @@ qgx_status qgx_set_decode_split(qgx_ctx* c, int mode) {
   return QGX_OK;
 }
 
+qgx_status qgx_set_encode_path(qgx_ctx* c, int mode) {
+  if (!c || (mode != QGX_ENCODE_AUTO && mode != QGX_ENCODE_REGISTERS)) return QGX_ERR_INVALID_ARG;
+  c->encode_path = mode;
+  return QGX_OK;
+}
+
 qgx_status qgx_exchange(qgx_ctx* c, const float* v, int K, size_t d, const qgx_quant_cfg* cfg, uint32_t exchange_id,
                         int slot, float* mean_out, uint64_t* total_bits) {
   if (!v) return QGX_ERR_INVALID_ARG;
@@ -1150,6 +1332,7 @@ qgx_status qgx_exchange_segments(qgx_ctx* c, const float* v, int K, size_t d, co
     if (cudaEventRecord(sc->fork, c->stream) != cudaSuccess) return QGX_ERR_CUDA;
     for (int i = 0; i < lanes; ++i) {
       sc->ctx[i]->decode_split = c->decode_split;
+      sc->ctx[i]->encode_path = c->encode_path;
       if (cudaStreamWaitEvent(sc->ctx[i]->stream, sc->fork, 0) != cudaSuccess) return QGX_ERR_CUDA;
     }
   }

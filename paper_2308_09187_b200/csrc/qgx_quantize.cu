@@ -11,7 +11,7 @@ __global__ void __launch_bounds__(512) k_quantize(DualSource src, size_t d, int 
                                                    uint32_t xid, int norm_type, int norms_supplied, bool vec_ok,
                                                    float* __restrict__ norms, uint8_t* __restrict__ sym, DevStatus* st) {
   __shared__ float s_lev[QGX_MAX_LEVELS];
-  __shared__ float4 s_bin[kKeyBins];
+  __shared__ float4 s_bin[kBinEntries];
   fill_bin_table(s_bin, rt);
   __shared__ double s_red[34];
   const size_t b = blockIdx.x, k = blockIdx.y;
@@ -158,7 +158,7 @@ qgx_status qgx_average(qgx_ctx* c, const float* norms, const uint8_t* sym, int K
   const size_t nquads = (d + kQuad - 1) / kQuad;
   const bool vec_ok = (d % kQuad == 0) && ((reinterpret_cast<uintptr_t>(sym) & 3u) == 0);
   const int threads = 256;
-  const unsigned blocks = (unsigned)std::min<size_t>((nquads + threads - 1) / threads, 148u * 16u);
+  const unsigned blocks = (unsigned)std::min<size_t>((nquads + threads - 1) / threads, (size_t)c->num_sms * 16u);
   k_average<<<blocks, threads, 0, c->stream>>>(norms, sym, K, d, bucket, nb, lt, vec_ok, out, c->dstatus);
   count_launch(c);
   return cuda_status(cudaGetLastError());
