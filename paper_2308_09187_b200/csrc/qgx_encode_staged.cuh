@@ -218,6 +218,7 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     if (g >= ngroups) {
       // out of groups: the other team, whose later buffer may still hold a group drawn earlier than this one,
       // finds the end marker in this buffer too when it comes round
+      team_sync(team);                                                // every thread of the team has seen this phase complete
       if (loader) issue_load(buf, ngroups);
       break;
     }
