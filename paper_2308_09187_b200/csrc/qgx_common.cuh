@@ -290,14 +290,42 @@ __device__ __forceinline__ uint32_t quantize_quad_codes(const float4 x, const ui
 //                   coordinates, so the second block is generated only for those.
 // In both modes the fast path uses the leading 16 bits h of r (the centre of the interval of r they leave) and
 // sends a coordinate to the exact routine when the outcome could depend on the remaining bits.
+// Shared memory by 32-bit address (what ld.shared takes): the hot loops compute table addresses themselves.
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// read-only tables: the address depends on the data just loaded, so the compiler cannot move these too early
+__device__ __forceinline__ float4 lds_table128(uint32_t addr) {
+  float4 v;
+  asm("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_table32(uint32_t addr) {
+  uint32_t v;
+  asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+// data that other threads or copies write: ordered with the barriers around them
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
+
 struct RoundK {
   float rn;                              // RN(1 / norm)
   float thr;                             // negative: every coordinate goes to the exact routine
   float nqs, magic;
-  uint32_t bin_mask, bin_lane;
+  uint32_t bin_mask;                     // keeps the bin part of pattern >> kBinAddrShift
+  uint32_t bin_base;                     // shared address of this lane's copy of bin 0, minus kBinAddrBase
 };
 
-__device__ __forceinline__ RoundK round_k(const RoundTable& rt, float norm) {
+// bin = the bin table (entries with a16) in shared memory
+__device__ __forceinline__ RoundK round_k(const RoundTable& rt, float norm, const float4* bin) {
   const bool ok = rt.usable && norm > 7.9e-31f && norm < 1.2e30f;
   RoundK c;
   c.rn = ok ? __frcp_rn(norm) : 0.0f;
@@ -306,17 +334,16 @@ __device__ __forceinline__ RoundK round_k(const RoundTable& rt, float norm) {
   c.magic = rt.magic;
   const uint32_t copy_bytes = 16u << (rt.key_shift - kKeyShiftMin);
   c.bin_mask = ~(copy_bytes - 1u);
-  c.bin_lane = ((threadIdx.x & 31u) << 4) & (copy_bytes - 1u);
+  c.bin_base = smem_addr(bin) - kBinAddrBase + (((threadIdx.x & 31u) << 4) & (copy_bytes - 1u));
   return c;
 }
 
-// One coordinate: returns S * (signed level index) as a float (the level of x, negative for negative x), and ORs
-// into *unsafe whether the exact routine has to decide.  hbits = pattern of the float 2^23 + h.  binz = the bin
-// table's address (entries with a16) minus kBinAddrBase bytes.
-__device__ __forceinline__ float round_signed(float x, uint32_t hbits, const RoundK& c, const char* binz, bool* unsafe) {
+// One coordinate: returns S * (signed level index) as a float (the level of x, negative for negative x) and raises
+// *worst to the distance of S (F - r~) + S / 2 from that multiple of S: above c.thr the exact routine has to decide.
+// hbits = pattern of the float 2^23 + h.
+__device__ __forceinline__ float round_signed(float x, uint32_t hbits, const RoundK& c, float* worst) {
   const float u2 = fmaf(fabsf(x), c.rn, kRoundShift);
-  const uint32_t off = ((__float_as_uint(u2) >> kBinAddrShift) & c.bin_mask) | c.bin_lane;
-  const float4 e = *reinterpret_cast<const float4*>(binz + off);
+  const float4 e = lds_table128(((__float_as_uint(u2) >> kBinAddrShift) & c.bin_mask) + c.bin_base);
   const float t1 = fmaf(__uint_as_float(hbits), c.nqs, e.x);                       // exact: both are multiples of S 2^-16
   float X = fmaf(u2, e.y, t1);
   X = fmaf(__saturatef(__fsub_rn(u2, e.z)), e.w, X);                               // S (F - r~) + S / 2
@@ -324,7 +351,7 @@ __device__ __forceinline__ float round_signed(float x, uint32_t hbits, const Rou
   const float Z = fmaf(X, sg, c.magic);
   const float zi = __fsub_rn(Z, c.magic);                                          // the nearest multiple of S, signed
   const float rho = fmaf(X, sg, -zi);
-  *unsafe = *unsafe || (fabsf(rho) > c.thr);
+  *worst = fmaxf(*worst, fabsf(rho));
   return zi;
 }
 

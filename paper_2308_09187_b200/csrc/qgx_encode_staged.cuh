@@ -39,9 +39,10 @@ __device__ __forceinline__ void merge_octet(uint32_t e0, uint32_t e1, uint32_t e
   *n = nA + n2 + n3;
 }
 
-// Appends the n (8..104) bits m[0..3] to a lane's run of bits in region R: full words are stored, the partial
-// word stays in carry (nc < 32 bits of it valid).  wi = index of the word that carry will become.
-__device__ __forceinline__ void append_bits(uint32_t* R, uint32_t& wi, uint32_t& nc, uint32_t& carry, const uint32_t* m, uint32_t n) {
+// Appends the n (8..104) bits m[0..3] to a lane's run of bits in the region at shared address R: full words are
+// stored, the partial word stays in carry (nc < 32 bits of it valid).  wa = shared address of the word that carry
+// will become.
+__device__ __forceinline__ void append_bits(uint32_t& wa, uint32_t& nc, uint32_t& carry, const uint32_t* m, uint32_t n) {
   const uint32_t s0 = carry | (m[0] << nc);
   const uint32_t s1 = __funnelshift_l(m[0], m[1], nc);
   const uint32_t s2 = __funnelshift_l(m[1], m[2], nc);
@@ -50,12 +51,12 @@ __device__ __forceinline__ void append_bits(uint32_t* R, uint32_t& wi, uint32_t&
   const uint32_t tot = nc + n;
   const uint32_t nfull = tot >> 5;                                   // 0..4
   const bool p0 = nfull > 0u, p1 = nfull > 1u, p2 = nfull > 2u, p3 = nfull > 3u;
-  if (p0) R[wi] = s0;
-  if (p1) R[wi + 1] = s1;
-  if (p2) R[wi + 2] = s2;
-  if (p3) R[wi + 3] = s3;
+  if (p0) sts32(wa, s0);
+  if (p1) sts32(wa + 4u, s1);
+  if (p2) sts32(wa + 8u, s2);
+  if (p3) sts32(wa + 12u, s3);
   carry = p3 ? s4 : (p2 ? s3 : (p1 ? s2 : (p0 ? s1 : s0)));
-  wi += nfull;
+  wa += nfull << 2;
   nc = tot & 31u;
 }
 
@@ -77,16 +78,26 @@ __device__ __forceinline__ void tma_load_rows(void* dst, const CUtensorMap* map,
 }
 // orders this thread's earlier accesses to shared memory before later bulk copies into it
 __device__ __forceinline__ void fence_before_bulk_copy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// waits for the phase of the given parity to complete; false if the (bounded) wait ran out
+// Waits (one lane polls for its warp, backing off) for the phase of the given parity to complete; false if the
+// bounded wait ran out.  Called by whole warps.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity) {
   const unsigned addr = (unsigned)__cvta_generic_to_shared(bar);
-  for (int spin = 0; spin < kSpinLimit; ++spin) {
-    unsigned done;
-    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-    if (done) return true;
+  unsigned done = 0;
+  if ((threadIdx.x & 31u) == 0) {
+    for (int spin = 0; spin < kSpinLimit && !done; ++spin) {
+      asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                   : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+      if (!done && spin > 4) __nanosleep(100);
+    }
   }
-  return false;
+  done = __shfl_sync(0xffffffffu, done, 0);
+  if (done) {                                           // every lane observes the completed phase itself (and its data)
+    unsigned again;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(again) : "r"(addr), "r"(parity) : "memory");
+    done = again;
+  }
+  return __all_sync(0xffffffffu, done != 0);
 }
 __device__ __forceinline__ void team_sync(int team) {
   asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(kTeamThreads) : "memory");
@@ -95,27 +106,29 @@ __device__ __forceinline__ void team_sync(int team) {
 // where a warp keeps the 16-bit lengths of its sub-blocks: inside its part of the stage, past its region
 constexpr int kWarpHdrWord = 420;                        // a region has at most 1024 * 13 / 32 + 1 = 417 words
 
-// One segment of a bucket's stream for the copy-out: a region of T valid bits that starts at bit s of the bucket.
+// One segment of a bucket's stream for the copy-out: a region (shared address R) of T valid bits that starts at
+// bit s of the bucket.
 struct Segment {
-  const uint32_t* R;
+  uint32_t R;
   uint32_t s, T;
 };
 
 // Stores the words of the bucket's stream whose first bit lies in `seg` (a word that runs past the segment's end
-// takes its remaining bits from the first word of the following region; every following segment has >= 32 bits).
-__device__ __forceinline__ void copy_segment(const Segment seg, const uint32_t* next_R, uint32_t* dst, int lane) {
+// takes its remaining bits from the first word of the following region, at shared address next_R or 0 for none;
+// every following segment has >= 32 bits).
+__device__ __forceinline__ void copy_segment(const Segment seg, uint32_t next_R, uint32_t* dst, int lane) {
   const uint32_t m_lo = (seg.s + 31u) >> 5, m_hi = (seg.s + seg.T + 31u) >> 5;
   const uint32_t nw = (seg.T + 31u) >> 5;
   for (uint32_t m = m_lo + (uint32_t)lane; m < m_hi; m += 32u) {
     const uint32_t q = (m << 5) - seg.s;
     const uint32_t i = q >> 5;
-    const uint32_t lo = seg.R[i];
-    const uint32_t hi = (i + 1u < nw) ? seg.R[i + 1u] : 0u;
+    const uint32_t lo = lds32(seg.R + 4u * i);
+    const uint32_t hi = (i + 1u < nw) ? lds32(seg.R + 4u * i + 4u) : 0u;
     uint32_t v = __funnelshift_r(lo, hi, q & 31u);
     const uint32_t valid = seg.T - q;                                // > 0
     if (valid < 32u) {
       v &= (1u << valid) - 1u;
-      if (next_R != nullptr) v |= next_R[0] << valid;
+      if (next_R != 0u) v |= lds32(next_R) << valid;
     }
     dst[m] = v;
   }
@@ -124,12 +137,13 @@ __device__ __forceinline__ void copy_segment(const Segment seg, const uint32_t* 
 // Buckets [0, a.nb_whole) of every worker; G coordinates per sub-block; a.bucket a multiple of 1024 that divides
 // 16384; all sources 16-byte aligned, the workers' rows a multiple of 32 floats apart, and the vector's first
 // coordinate a multiple of 8 in the generator's counter space (the host checks).  tmap: the staged source as rows
-// of 32 floats.  Buckets are taken in the order b-major, k-minor, 16384 / bucket at a time, a group per ticket
-// drawn from a counter.  Group n of a CTA is worked on by team n & 1 in buffer n % 3; a team draws the ticket of
-// group n + 3 when it has finished group n, so each team's groups have increasing tickets.  A bucket waits
-// (look-back) only for buckets of groups with smaller tickets, and a group that has been drawn but not started
-// waits only for its own team's current group, whose ticket is smaller: the unfinished group with the smallest
-// ticket is always being worked on and waits for nothing, so every wait ends.
+// of 32 floats.  Buckets are taken in the order b-major, k-minor, 16384 / bucket at a time; group g belongs to CTA
+// g mod gridDim.x, which works on its groups in increasing order (its n-th group by team n & 1 in buffer n % 3).
+// All CTAs are resident and advance at the same pace, so the buckets a bucket looks back at (the same worker's
+// earlier buckets, which lie in groups before its own) have usually been counted when it asks.  A bucket waits
+// only for buckets of smaller groups, and a group that is staged but not started waits only for its own team's
+// current group, which is smaller: the smallest unfinished group is always being worked on and waits for
+// nothing, so every wait ends.
 template <int G, int RNG>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt, const __grid_constant__ CodeTable ct,
@@ -168,15 +182,14 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
   if (tid == 0) {
     for (int i = 0; i < kStageBuffers; ++i) {
       mbar_init(&s_full[i], 1);
-      s_group[i] = atomicAdd(a.ticket, 1u);                           // the CTA's first three groups, in order
+      s_group[i] = blockIdx.x + (unsigned)i * gridDim.x;              // the CTA's first three groups
     }
   }
   __syncthreads();
   fill_pair_lut_signed(s_pair, &s_lut);
   __syncthreads();
   const int nlev = lt.nlev;
-  const char* binz = reinterpret_cast<const char*>(s_bin) - kBinAddrBase;
-  const char* pairz = reinterpret_cast<const char*>(s_pair);
+  const uint32_t pair_sa = smem_addr(s_pair), stage_sa = smem_addr(s_stage);
   const float S = -rt.neg_qscale16 * 65536.0f, four_over_S = 4.0f / S;
   const size_t ld = a.src.ld ? a.src.ld : a.d;
   const unsigned long long total = (unsigned long long)a.nb_whole * (unsigned long long)a.K;
@@ -227,7 +240,8 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     const size_t b = active ? (size_t)(t / (unsigned long long)a.K) : 0, k = active ? (size_t)(t % (unsigned long long)a.K) : 0;
     const size_t lo = b * (size_t)a.bucket;
     float* stage = s_stage + buf * kStageCoords + slot * a.bucket;
-    uint32_t* region = reinterpret_cast<uint32_t*>(s_stage + buf * kStageCoords + tw * kWarpCoords);
+    const uint32_t region = stage_sa + 4u * (uint32_t)(buf * kStageCoords + tw * kWarpCoords);   // shared address of the warp's part
+    const uint32_t line_sa = stage_sa + 4u * (uint32_t)(buf * kStageCoords + slot * a.bucket + line * kLaneCoords);
 
     // ---- partial norm over this thread's chunks (chunk line, line + bthreads, ...: a warp reads contiguous
     //      memory of the second source); with two sources the stage receives their combination ----
@@ -276,7 +290,7 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     }
     const bool finite = (norm - norm) == 0.0f;
     const bool live = finite && norm != 0.0f;                         // otherwise every coordinate is level 0
-    const RoundK rc = round_k(rt, norm);
+    const RoundK rc = round_k(rt, norm, s_bin);
 
     // ---- rounding and pair codes of this lane's 32 coordinates: four octets ----
     uint32_t e[16];
@@ -287,16 +301,16 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
       for (int o = 0; o < 4; ++o) {
         float z[8];
         if (live) {
-          const float4 xa = *reinterpret_cast<const float4*>(stage + stage_at(line, 2 * o));
-          const float4 xb = *reinterpret_cast<const float4*>(stage + stage_at(line, 2 * o + 1));
-          octet_levels<RNG>(xa, xb, oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, binz, s_lev, nlev, z);
+          const float4 xa = lds128(line_sa + (uint32_t)(((2 * o) ^ (line & 7)) << 4));
+          const float4 xb = lds128(line_sa + (uint32_t)(((2 * o + 1) ^ (line & 7)) << 4));
+          octet_levels<RNG>(xa, xb, oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, s_lev, nlev, z);
         } else {
 #pragma unroll
           for (int i = 0; i < 8; ++i) z[i] = 0.0f;
         }
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
-          const uint32_t en = *reinterpret_cast<const uint32_t*>(pairz + pair_offset(z[2 * p], z[2 * p + 1], four_over_S));
+          const uint32_t en = pair_entry(pair_sa, z[2 * p], z[2 * p + 1], four_over_S);
           e[4 * o + p] = en;
           nbits_lane += en >> 26;
         }
@@ -336,23 +350,24 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
       constexpr int kSubLanes = G / kLaneCoords;                      // lanes per sub-block: 1, 2 or 4
       const uint32_t before = __shfl_up_sync(0xffffffffu, incl, kSubLanes);
       const uint32_t sub = incl - (lane >= kSubLanes ? before : 0u);
-      if ((lane + 1) % kSubLanes == 0) reinterpret_cast<uint16_t*>(region + kWarpHdrWord)[lane / kSubLanes] = (uint16_t)sub;
+      if ((lane + 1) % kSubLanes == 0)
+        asm volatile("st.shared.u16 [%0], %1;" ::"r"(region + 4u * kWarpHdrWord + 2u * (uint32_t)(lane / kSubLanes)), "h"((uint16_t)sub) : "memory");
     }
-    uint32_t wi = (incl - nbits_lane) >> 5, nc = (incl - nbits_lane) & 31u, carry = 0u;
-    const uint32_t wi0 = wi, nc0 = nc;
+    uint32_t wa = region + (((incl - nbits_lane) >> 5) << 2), nc = (incl - nbits_lane) & 31u, carry = 0u;
+    const uint32_t wa0 = wa, nc0 = nc;
     if (active) {
 #pragma unroll
       for (int o = 0; o < 4; ++o) {
         uint32_t m[4], n2;
         merge_octet(e[4 * o], e[4 * o + 1], e[4 * o + 2], e[4 * o + 3], m, &n2);
-        append_bits(region, wi, nc, carry, m, n2);
+        append_bits(wa, nc, carry, m, n2);
       }
     }
     {
       // the first word of a lane's run also holds the last bits of the lane before it
       const uint32_t prev = __shfl_up_sync(0xffffffffu, carry, 1);
-      if (active && lane > 0 && nc0 != 0u) region[wi0] |= prev;
-      if (active && lane == 31 && nc != 0u) region[wi] = carry;
+      if (active && lane > 0 && nc0 != 0u) sts32(wa0, lds32(wa0) | prev);
+      if (active && lane == 31 && nc != 0u) sts32(wa, carry);
     }
 
     unsigned int next_group = 0;
@@ -368,8 +383,7 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
         s_base[gslot] = excl;
         s_skip[gslot] = skip;
         s_cnt[gslot] = 0u;
-        // the group that will use this buffer next; the answer is not needed before the copy-out is over
-        if (slot == 0) next_group = atomicAdd(a.ticket, 1u);
+        if (slot == 0) next_group = (unsigned int)min(g + 3ull * gridDim.x, (unsigned long long)0xffffffffu);   // this buffer's next group
       }
     }
     team_sync(team);                                                  // all regions and stream offsets are in
@@ -384,13 +398,13 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
           uint32_t v = __float_as_uint(norm);
           if (m > 0u) {
             const uint32_t sb = 2u * (m - 1u);                        // the word's first sub-block
-            const uint32_t* wr = reinterpret_cast<const uint32_t*>(s_stage + buf * kStageCoords + (slot * wpb + (int)(sb / kSubPerWarp)) * kWarpCoords);
-            v = wr[kWarpHdrWord + (sb % kSubPerWarp) / 2u];
+            const uint32_t wr = stage_sa + 4u * (uint32_t)(buf * kStageCoords + (slot * wpb + (int)(sb / kSubPerWarp)) * kWarpCoords);
+            v = lds32(wr + 4u * (kWarpHdrWord + (sb % kSubPerWarp) / 2u));
           }
           dst[m] = v;
         }
       }
-      const uint32_t* next_R = wis + 1 < wpb ? region + kWarpCoords : nullptr;
+      const uint32_t next_R = wis + 1 < wpb ? region + 4u * kWarpCoords : 0u;
       copy_segment(Segment{region, hdr_bits + before, s_tot[warp]}, next_R, dst, lane);
     }
     if (last_of_bucket && slot == 0 && lane == 0) s_next[team] = next_group;

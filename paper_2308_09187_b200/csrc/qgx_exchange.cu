@@ -178,7 +178,7 @@ __device__ __forceinline__ void load_bucket_octets(BucketRegs<2 * P>& r, const D
 template <int RNG>
 static __device__ __noinline__ uint64_t redo_octet(const float4 xa, const float4 xb, const uint4 w0, const uint4 w1, uint64_t oct,
                                                    uint32_t k, uint32_t xid, const PhiloxKey* key, const RoundK rc, float norm,
-                                                   const char* binz, const float* lev, int nlev) {
+                                                   const float* lev, int nlev) {
   const float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
   const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
   const float inv_S = -1.0f / (rc.nqs * 65536.0f);
@@ -187,10 +187,10 @@ static __device__ __noinline__ uint64_t redo_octet(const float4 xa, const float4
   uint64_t out = 0;
   for (int i = 0; i < 8; ++i) {
     const uint32_t h = RNG == QGX_RNG_HALF32 ? ((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xffffu)) : (w[i] >> 16);
-    bool unsafe = false;
-    const float zi = round_signed(x[i], 0x4B000000u | h, rc, binz, &unsafe);
+    float worst = 0.0f;
+    const float zi = round_signed(x[i], 0x4B000000u | h, rc, &worst);
     int idx = (int)fabsf(__fmul_rn(zi, inv_S));
-    if (unsafe) {
+    if (!(worst <= rc.thr)) {
       uint32_t rb;
       if (RNG == QGX_RNG_HALF32) {
         if (!have2) { w2 = philox4x32_10((uint32_t)oct, (uint32_t)(oct >> 32), k | 0x80000000u, xid, *key); have2 = true; }
@@ -211,7 +211,7 @@ static __device__ __noinline__ uint64_t redo_octet(const float4 xa, const float4
 // space) of worker k.  S = the scale of the rounding table.
 template <int RNG>
 __device__ __forceinline__ void octet_levels(const float4 xa, const float4 xb, uint64_t oct, uint32_t k, uint32_t xid,
-                                             const PhiloxKey& key, const RoundK& rc, float norm, float S, const char* binz,
+                                             const PhiloxKey& key, const RoundK& rc, float norm, float S,
                                              const float* lev, int nlev, float* z) {
   constexpr uint32_t kTwo23 = 0x4B000000u;              // pattern of 2^23: its low mantissa bytes are replaced by h
   const float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
@@ -231,20 +231,21 @@ __device__ __forceinline__ void octet_levels(const float4 xa, const float4 xb, u
     hb[4] = prmt(w1.x, kTwo23, 0x7632u); hb[5] = prmt(w1.y, kTwo23, 0x7632u);
     hb[6] = prmt(w1.z, kTwo23, 0x7632u); hb[7] = prmt(w1.w, kTwo23, 0x7632u);
   }
-  bool unsafe = false;
+  float worst = 0.0f;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) z[i] = round_signed(x[i], hb[i], rc, binz, &unsafe);
-  if (unsafe) {                                         // some coordinate of the octet needs the exact routine
-    const uint64_t fixed = redo_octet<RNG>(xa, xb, w0, w1, oct, k, xid, &key, rc, norm, binz, lev, nlev);
+  for (int i = 0; i < 8; ++i) z[i] = round_signed(x[i], hb[i], rc, &worst);
+  if (!(worst <= rc.thr)) {                                      // some coordinate of the octet needs the exact routine
+    const uint64_t fixed = redo_octet<RNG>(xa, xb, w0, w1, oct, k, xid, &key, rc, norm, lev, nlev);
 #pragma unroll
     for (int i = 0; i < 8; ++i) z[i] = __fmul_rn((float)(int)(signed char)(uint8_t)(fixed >> (8 * i)), S);
   }
 }
 
-// the pair table's byte offset for two consecutive coordinates: 4 * ((first + 64 * second) mod 4096)
-__device__ __forceinline__ uint32_t pair_offset(float z_first, float z_second, float four_over_S) {
+// the pair table's entry for two consecutive coordinates, at byte 4 * ((first + 64 * second) mod 4096) of the
+// table at shared address `pair`
+__device__ __forceinline__ uint32_t pair_entry(uint32_t pair, float z_first, float z_second, float four_over_S) {
   const float t = fmaf(z_second, 64.0f * four_over_S, fmaf(z_first, four_over_S, 12582912.0f));   // 1.5 * 2^23 + 4 first + 256 second
-  return __float_as_uint(t) & 0x3ffcu;
+  return lds_table32(pair + (__float_as_uint(t) & 0x3ffcu));
 }
 
 // One persistent CTA per SM slot; each ticket is one bucket (k = ticket % K, b = ticket / K).
@@ -285,7 +286,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   fill_pair_lut_signed(s_pair, &s_lut);
   __syncthreads();
   const int nlev = lt.nlev;
-  const char* binz = reinterpret_cast<const char*>(s_bin) - kBinAddrBase;
+  const uint32_t pair_sa = smem_addr(s_pair);
   const float S = -rt.neg_qscale16 * 65536.0f, four_over_S = 4.0f / S;
   uint32_t used_words[2] = {0u, 0u};                    // words of each image that the last bucket in it dirtied
 
@@ -307,7 +308,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     }
     const float norm = bucket_norm_all<2 * P>(r, a.norm_type, s_red[par]);   // barrier inside: the image is zero
     const bool finite = (norm - norm) == 0.0f;
-    const RoundK rc = round_k(rt, norm);
+    const RoundK rc = round_k(rt, norm, s_bin);
     if (threadIdx.x == 0) {
       a.norms[k * a.nb + b] = norm;
       if (!finite) latch_error(a.st, QGX_ERR_NONFINITE);
@@ -327,12 +328,9 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
       for (int j = 0; j < P; ++j) {
         const int o = (warp * P + j) * 32 + lane;
         float z[8];
-        octet_levels<RNG>(r.x[2 * j], r.x[2 * j + 1], oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, binz, s_lev, nlev, z);
-        const char* pz = reinterpret_cast<const char*>(s_pair);
-        const uint32_t e01 = *reinterpret_cast<const uint32_t*>(pz + pair_offset(z[0], z[1], four_over_S));
-        const uint32_t e23 = *reinterpret_cast<const uint32_t*>(pz + pair_offset(z[2], z[3], four_over_S));
-        const uint32_t e45 = *reinterpret_cast<const uint32_t*>(pz + pair_offset(z[4], z[5], four_over_S));
-        const uint32_t e67 = *reinterpret_cast<const uint32_t*>(pz + pair_offset(z[6], z[7], four_over_S));
+        octet_levels<RNG>(r.x[2 * j], r.x[2 * j + 1], oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, s_lev, nlev, z);
+        const uint32_t e01 = pair_entry(pair_sa, z[0], z[1], four_over_S), e23 = pair_entry(pair_sa, z[2], z[3], four_over_S);
+        const uint32_t e45 = pair_entry(pair_sa, z[4], z[5], four_over_S), e67 = pair_entry(pair_sa, z[6], z[7], four_over_S);
         uint32_t n0, n1;
         pack_pair_entries(e01, e23, &qbits[2 * j], &n0);
         pack_pair_entries(e45, e67, &qbits[2 * j + 1], &n1);
