@@ -152,6 +152,28 @@ __device__ __forceinline__ void philox4x32_10_x2(uint64_t ctr_a, uint64_t ctr_b,
   *out_b = make_uint4(b0, b1, b2, b3);
 }
 
+// four blocks with consecutive counters ctr, ctr + 1, ctr + 2, ctr + 3 (same last two counter words), round by round
+__device__ __forceinline__ void philox4x32_10_x4(uint64_t ctr, uint32_t c2, uint32_t c3, const PhiloxKey& key, uint4* out) {
+  uint32_t s0[4], s1[4], s2[4], s3[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint64_t c = ctr + (uint64_t)j;
+    s0[j] = (uint32_t)c; s1[j] = (uint32_t)(c >> 32); s2[j] = c2; s3[j] = c3;
+  }
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t k0 = key.k0[r], k1 = key.k1[r];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)s0[j], p1 = (uint64_t)0xCD9E8D57u * (uint64_t)s2[j];
+      const uint32_t n0 = (uint32_t)(p1 >> 32) ^ s1[j] ^ k0, n2 = (uint32_t)(p0 >> 32) ^ s3[j] ^ k1;
+      s0[j] = n0; s1[j] = (uint32_t)p1; s2[j] = n2; s3[j] = (uint32_t)p0;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) out[j] = make_uint4(s0[j], s1[j], s2[j], s3[j]);
+}
+
 // ---- Definition 1 for one normalized coordinate, every operation one IEEE rounding ----------
 // returns the level index; lev points to the table in shared memory
 __device__ __forceinline__ int quantize_level(float absv, float norm, const float* lev, int nlev, uint32_t word) {
@@ -320,11 +342,12 @@ struct RoundK {
   float rn;                              // RN(1 / norm)
   float thr;                             // negative: every coordinate goes to the exact routine
   float nqs, magic;
-  uint32_t bin_mask;                     // keeps the bin part of pattern >> kBinAddrShift
-  uint32_t bin_base;                     // shared address of this lane's copy of bin 0, minus kBinAddrBase
+  uint32_t bin_mask;                     // clears the bits of pattern >> kBinAddrShift below a bin's copies
+  uint32_t bin_base;                     // shared address of the bin table (128-byte aligned) minus kBinAddrBase
+  uint32_t bin_lane;                     // byte offset of this lane's copy inside a bin
 };
 
-// bin = the bin table (entries with a16) in shared memory
+// bin = the bin table (entries with a16) in shared memory, aligned to 128 bytes
 __device__ __forceinline__ RoundK round_k(const RoundTable& rt, float norm, const float4* bin) {
   const bool ok = rt.usable && norm > 7.9e-31f && norm < 1.2e30f;
   RoundK c;
@@ -334,7 +357,8 @@ __device__ __forceinline__ RoundK round_k(const RoundTable& rt, float norm, cons
   c.magic = rt.magic;
   const uint32_t copy_bytes = 16u << (rt.key_shift - kKeyShiftMin);
   c.bin_mask = ~(copy_bytes - 1u);
-  c.bin_base = smem_addr(bin) - kBinAddrBase + (((threadIdx.x & 31u) << 4) & (copy_bytes - 1u));
+  c.bin_base = smem_addr(bin) - kBinAddrBase;           // a multiple of 128, like a bin's copies together
+  c.bin_lane = ((threadIdx.x & 31u) << 4) & (copy_bytes - 1u);
   return c;
 }
 
@@ -343,7 +367,8 @@ __device__ __forceinline__ RoundK round_k(const RoundTable& rt, float norm, cons
 // hbits = pattern of the float 2^23 + h.
 __device__ __forceinline__ float round_signed(float x, uint32_t hbits, const RoundK& c, float* worst) {
   const float u2 = fmaf(fabsf(x), c.rn, kRoundShift);
-  const float4 e = lds_table128(((__float_as_uint(u2) >> kBinAddrShift) & c.bin_mask) + c.bin_base);
+  // pattern >> 13 as the high word of pattern * 2^19, the table's address added in the same multiply-add
+  const float4 e = lds_table128(((__umulhi(__float_as_uint(u2), 1u << (32 - kBinAddrShift)) + c.bin_base) & c.bin_mask) | c.bin_lane);
   const float t1 = fmaf(__uint_as_float(hbits), c.nqs, e.x);                       // exact: both are multiples of S 2^-16
   float X = fmaf(u2, e.y, t1);
   X = fmaf(__saturatef(__fsub_rn(u2, e.z)), e.w, X);                               // S (F - r~) + S / 2

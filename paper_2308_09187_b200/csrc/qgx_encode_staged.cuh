@@ -113,24 +113,24 @@ struct Segment {
   uint32_t s, T;
 };
 
-// Stores the words of the bucket's stream whose first bit lies in `seg` (a word that runs past the segment's end
-// takes its remaining bits from the first word of the following region, at shared address next_R or 0 for none;
-// every following segment has >= 32 bits).
+// Stores the words of the bucket's stream whose first bit lies in `seg` (the last of them, when it runs past the
+// segment's end, takes its remaining bits from the first word of the following region, at shared address next_R
+// or 0 for none; every following segment has >= 32 bits).
 __device__ __forceinline__ void copy_segment(const Segment seg, uint32_t next_R, uint32_t* dst, int lane) {
   const uint32_t m_lo = (seg.s + 31u) >> 5, m_hi = (seg.s + seg.T + 31u) >> 5;
+  const uint32_t q0 = (m_lo << 5) - seg.s;                           // the region's bit that the first word starts at: 0..31
   const uint32_t nw = (seg.T + 31u) >> 5;
-  for (uint32_t m = m_lo + (uint32_t)lane; m < m_hi; m += 32u) {
-    const uint32_t q = (m << 5) - seg.s;
-    const uint32_t i = q >> 5;
-    const uint32_t lo = lds32(seg.R + 4u * i);
-    const uint32_t hi = (i + 1u < nw) ? lds32(seg.R + 4u * i + 4u) : 0u;
-    uint32_t v = __funnelshift_r(lo, hi, q & 31u);
-    const uint32_t valid = seg.T - q;                                // > 0
-    if (valid < 32u) {
-      v &= (1u << valid) - 1u;
-      if (next_R != 0u) v |= lds32(next_R) << valid;
+  const uint32_t count = m_hi - m_lo;
+  const uint32_t tail = (seg.T - q0) & 31u;                          // valid bits of the last word (0: all 32)
+  for (uint32_t j = (uint32_t)lane; j < count; j += 32u) {
+    const uint32_t lo = lds32(seg.R + 4u * j);
+    const uint32_t hi = (j + 1u < nw) ? lds32(seg.R + 4u * j + 4u) : 0u;
+    uint32_t v = __funnelshift_r(lo, hi, q0);
+    if (j + 1u == count && tail != 0u) {
+      v &= (1u << tail) - 1u;
+      if (next_R != 0u) v |= lds32(next_R) << tail;
     }
-    dst[m] = v;
+    dst[m_lo + j] = v;
   }
 }
 
@@ -149,12 +149,14 @@ __global__ void __launch_bounds__(kStagedThreads, 1)
 k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt, const __grid_constant__ CodeTable ct,
                 const __grid_constant__ PhiloxKey key, const __grid_constant__ RoundTable rt, const __grid_constant__ CUtensorMap tmap) {
   extern __shared__ __align__(1024) float s_stage[];                 // kStageBuffers * kStageCoords floats
-  __shared__ float4 s_bin[kBinEntries];
+  __shared__ __align__(128) float4 s_bin[kBinEntries];
   __shared__ uint32_t s_pair[kPairLutSize];
   __shared__ EncLut s_lut;
   __shared__ float s_lev[QGX_MAX_LEVELS];
   __shared__ double s_red[2 * kStagedWarps];
   __shared__ uint32_t s_tot[2 * kStagedWarps];
+  __shared__ uint32_t s_pre[2 * kStagedWarps];                        // bits of the bucket's warps before this one
+  __shared__ unsigned long long s_bk[kStageBuffers][kStagedWarps];   // bucket of a buffer's slot: b | k << 48, or ~0
   __shared__ unsigned int s_cnt[2 * kStagedWarps];                    // warps of a bucket that have their bit count
   __shared__ unsigned long long s_base[2 * kStagedWarps];             // word offset of the bucket in its worker's stream
   __shared__ int s_skip[2 * kStagedWarps];
@@ -203,10 +205,14 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     s_group[buf] = (unsigned int)min(g, (unsigned long long)0xffffffffu);
     const unsigned long long t0 = g * (unsigned long long)M;
     const int nslots = g < ngroups ? (int)min((unsigned long long)M, total - t0) : 0;
+    for (int sl = 0; sl < M; ++sl) {
+      const unsigned long long t = t0 + (unsigned long long)sl;
+      s_bk[buf][sl] = sl < nslots ? ((t / (unsigned long long)a.K) | ((t % (unsigned long long)a.K) << 48)) : ~0ull;
+    }
     mbar_arrive_expect(&s_full[buf], (unsigned)nslots * (unsigned)a.bucket * 4u);
     for (int sl = 0; sl < nslots; ++sl) {
-      const unsigned long long t = t0 + (unsigned long long)sl;
-      const size_t bb = (size_t)(t / (unsigned long long)a.K), kk = (size_t)(t % (unsigned long long)a.K);
+      const unsigned long long bk = s_bk[buf][sl];
+      const size_t bb = (size_t)(bk & 0xffffffffffffull), kk = (size_t)(bk >> 48);
       const size_t first = (a.src.v ? kk * ld : 0) + bb * (size_t)a.bucket;         // in floats from the map's base
       for (int r0 = 0; r0 < a.bucket / kLaneCoords; r0 += box_rows)
         tma_load_rows(s_stage + buf * kStageCoords + sl * a.bucket + r0 * kLaneCoords, &tmap, (int)(first / kLaneCoords) + r0, &s_full[buf]);
@@ -235,13 +241,13 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
       if (loader) issue_load(buf, ngroups);
       break;
     }
-    const unsigned long long t = g * (unsigned long long)M + (unsigned long long)slot;
-    const bool active = t < total;
-    const size_t b = active ? (size_t)(t / (unsigned long long)a.K) : 0, k = active ? (size_t)(t % (unsigned long long)a.K) : 0;
+    const unsigned long long bk = s_bk[buf][slot];
+    const bool active = bk != ~0ull;
+    const size_t b = active ? (size_t)(bk & 0xffffffffffffull) : 0, k = active ? (size_t)(bk >> 48) : 0;
     const size_t lo = b * (size_t)a.bucket;
-    float* stage = s_stage + buf * kStageCoords + slot * a.bucket;
-    const uint32_t region = stage_sa + 4u * (uint32_t)(buf * kStageCoords + tw * kWarpCoords);   // shared address of the warp's part
-    const uint32_t line_sa = stage_sa + 4u * (uint32_t)(buf * kStageCoords + slot * a.bucket + line * kLaneCoords);
+    const uint32_t slot_sa = stage_sa + 4u * (uint32_t)(buf * kStageCoords + slot * a.bucket);    // the bucket's stage
+    const uint32_t region = stage_sa + 4u * (uint32_t)(buf * kStageCoords + tw * kWarpCoords);    // the warp's part of it
+    const uint32_t line_sa = slot_sa + 4u * (uint32_t)(line * kLaneCoords);
 
     // ---- partial norm over this thread's chunks (chunk line, line + bthreads, ...: a warp reads contiguous
     //      memory of the second source); with two sources the stage receives their combination ----
@@ -254,12 +260,16 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
 #pragma unroll
         for (int r = 0; r < 8; ++r) av[r] = __ldg(reinterpret_cast<const float4*>(a.src.a + lo) + r * bthreads + line);
       }
+      const uint32_t l3 = (uint32_t)line >> 3, l7 = (uint32_t)line & 7u, step = (uint32_t)bthreads >> 3;
 #pragma unroll
       for (int r = 0; r < 8; ++r) {
-        const int c = r * bthreads + line;
-        float4* p = reinterpret_cast<float4*>(stage + stage_at(c >> 3, c & 7));
-        float4 x = *p;
-        if (two) { x = dual_combine(av[r], x, a.src.mul); *p = x; }
+        const uint32_t li = (uint32_t)r * step + l3;                  // chunk r * bthreads + line: chunk l7 of line li
+        const uint32_t pa = slot_sa + (li << 7) + ((l7 ^ (li & 7u)) << 4);
+        float4 x = lds128(pa);
+        if (two) {
+          x = dual_combine(av[r], x, a.src.mul);
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(pa), "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w) : "memory");
+        }
         if (a.norm_type == QGX_NORM_L2) {
           const double x0 = x.x, x1 = x.y, x2 = x.z, x3 = x.w;
           acc = fma(x0, x0, acc); acc = fma(x1, x1, acc); acc = fma(x2, x2, acc); acc = fma(x3, x3, acc);
@@ -292,28 +302,32 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     const bool live = finite && norm != 0.0f;                         // otherwise every coordinate is level 0
     const RoundK rc = round_k(rt, norm, s_bin);
 
-    // ---- rounding and pair codes of this lane's 32 coordinates: four octets ----
-    uint32_t e[16];
-    uint32_t nbits_lane = 0;
+    // ---- rounding, pair codes and stream bits of this lane's 32 coordinates: four octets ----
+    uint32_t mb[16];                                                  // the bits of the four octets, four words each
+    uint32_t npack = 0, nbits_lane = 0;                               // their bit counts, a byte each, and the sum
     if (active) {
       const uint64_t oct0 = ((a.quad_base + (uint64_t)(lo >> 2)) >> 1) + 4ull * (uint64_t)line;
+      const uint32_t l7 = (uint32_t)line & 7u;
+      uint4 W[4];
+      if (live && RNG == QGX_RNG_HALF32) philox4x32_10_x4(oct0, (uint32_t)k, a.xid, key, W);
 #pragma unroll
       for (int o = 0; o < 4; ++o) {
         float z[8];
         if (live) {
-          const float4 xa = lds128(line_sa + (uint32_t)(((2 * o) ^ (line & 7)) << 4));
-          const float4 xb = lds128(line_sa + (uint32_t)(((2 * o + 1) ^ (line & 7)) << 4));
-          octet_levels<RNG>(xa, xb, oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, s_lev, nlev, z);
+          if (RNG == QGX_RNG_WORD24 && (o & 1) == 0) philox4x32_10_x4(2ull * (oct0 + (uint64_t)o), (uint32_t)k, a.xid, key, W);
+          const float4 xa = lds128(line_sa + (((uint32_t)(2 * o) ^ l7) << 4));
+          const float4 xb = lds128(line_sa + (((uint32_t)(2 * o + 1) ^ l7) << 4));
+          const uint4 w0 = RNG == QGX_RNG_HALF32 ? W[o] : W[2 * (o & 1)], w1 = RNG == QGX_RNG_HALF32 ? W[o] : W[2 * (o & 1) + 1];
+          octet_levels_w<RNG>(xa, xb, w0, w1, oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, s_lev, nlev, z);
         } else {
 #pragma unroll
           for (int i = 0; i < 8; ++i) z[i] = 0.0f;
         }
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-          const uint32_t en = pair_entry(pair_sa, z[2 * p], z[2 * p + 1], four_over_S);
-          e[4 * o + p] = en;
-          nbits_lane += en >> 26;
-        }
+        uint32_t n2;
+        merge_octet(pair_entry(pair_sa, z[0], z[1], four_over_S), pair_entry(pair_sa, z[2], z[3], four_over_S),
+                    pair_entry(pair_sa, z[4], z[5], four_over_S), pair_entry(pair_sa, z[6], z[7], four_over_S), &mb[4 * o], &n2);
+        npack |= n2 << (8 * o);
+        nbits_lane += n2;
       }
     }
     // bit offsets inside the warp's region, the warp's total; the warp that completes the bucket's bit count
@@ -330,10 +344,10 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     unsigned long long* row = a.status + k * a.nb;
     uint32_t nbits = 0, nwords = 0;
     if (last_of_bucket) {
-      uint32_t payload = lane < wpb ? s_tot[team * kStagedWarps + slot * wpb + lane] : 0u;
-#pragma unroll
-      for (int o2 = 16; o2 > 0; o2 >>= 1) payload += __shfl_xor_sync(0xffffffffu, payload, o2);
-      nbits = hdr_bits + payload;
+      const uint32_t mine = lane < wpb ? s_tot[team * kStagedWarps + slot * wpb + lane] : 0u;
+      const uint32_t upto = warp_incl_scan(mine, lane);
+      if (lane < wpb) s_pre[team * kStagedWarps + slot * wpb + lane] = upto - mine;
+      nbits = hdr_bits + __shfl_sync(0xffffffffu, upto, 31);
       nwords = (nbits + 31u) >> 5;
       if (lane == 0) {
         st_status(row + b, kStAggregate | (unsigned long long)nwords);
@@ -357,11 +371,7 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     const uint32_t wa0 = wa, nc0 = nc;
     if (active) {
 #pragma unroll
-      for (int o = 0; o < 4; ++o) {
-        uint32_t m[4], n2;
-        merge_octet(e[4 * o], e[4 * o + 1], e[4 * o + 2], e[4 * o + 3], m, &n2);
-        append_bits(wa, nc, carry, m, n2);
-      }
+      for (int o = 0; o < 4; ++o) append_bits(wa, nc, carry, &mb[4 * o], (npack >> (8 * o)) & 0xffu);
     }
     {
       // the first word of a lane's run also holds the last bits of the lane before it
@@ -391,8 +401,7 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     // ---- copy out: the header (whole words) by the bucket's first warp, then every warp its own region ----
     if (active && !s_skip[gslot]) {
       uint32_t* dst = a.stream + k * a.cap_words + s_base[gslot];
-      uint32_t before = 0;
-      for (int w2 = 0; w2 < wis; ++w2) before += s_tot[team * kStagedWarps + slot * wpb + w2];
+      const uint32_t before = s_pre[warp];
       if (wis == 0) {
         for (uint32_t m = (uint32_t)lane; m < hdr_words; m += 32u) {
           uint32_t v = __float_as_uint(norm);

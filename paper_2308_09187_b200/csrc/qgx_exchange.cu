@@ -208,24 +208,21 @@ static __device__ __noinline__ uint64_t redo_octet(const float4 xa, const float4
 }
 
 // S * (signed level index) of the eight coordinates xa, xb of octet `oct` (its index in the generator's counter
-// space) of worker k.  S = the scale of the rounding table.
+// space) of worker k, given the octet's Philox words: w0 alone (QGX_RNG_HALF32: the block of counter oct) or w0, w1
+// (QGX_RNG_WORD24: the blocks of counters 2 oct and 2 oct + 1).  S = the scale of the rounding table.
 template <int RNG>
-__device__ __forceinline__ void octet_levels(const float4 xa, const float4 xb, uint64_t oct, uint32_t k, uint32_t xid,
-                                             const PhiloxKey& key, const RoundK& rc, float norm, float S,
-                                             const float* lev, int nlev, float* z) {
+__device__ __forceinline__ void octet_levels_w(const float4 xa, const float4 xb, const uint4 w0, const uint4 w1, uint64_t oct,
+                                               uint32_t k, uint32_t xid, const PhiloxKey& key, const RoundK& rc, float norm,
+                                               float S, const float* lev, int nlev, float* z) {
   constexpr uint32_t kTwo23 = 0x4B000000u;              // pattern of 2^23: its low mantissa bytes are replaced by h
   const float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-  uint4 w0, w1;
   uint32_t hb[8];
   if (RNG == QGX_RNG_HALF32) {
-    w0 = philox4x32_10((uint32_t)oct, (uint32_t)(oct >> 32), k, xid, key);
-    w1 = w0;
     hb[0] = prmt(w0.x, kTwo23, 0x7610u); hb[1] = prmt(w0.x, kTwo23, 0x7632u);
     hb[2] = prmt(w0.y, kTwo23, 0x7610u); hb[3] = prmt(w0.y, kTwo23, 0x7632u);
     hb[4] = prmt(w0.z, kTwo23, 0x7610u); hb[5] = prmt(w0.z, kTwo23, 0x7632u);
     hb[6] = prmt(w0.w, kTwo23, 0x7610u); hb[7] = prmt(w0.w, kTwo23, 0x7632u);
   } else {
-    philox4x32_10_x2(2ull * oct, 2ull * oct + 1ull, k, xid, key, &w0, &w1);
     hb[0] = prmt(w0.x, kTwo23, 0x7632u); hb[1] = prmt(w0.y, kTwo23, 0x7632u);
     hb[2] = prmt(w0.z, kTwo23, 0x7632u); hb[3] = prmt(w0.w, kTwo23, 0x7632u);
     hb[4] = prmt(w1.x, kTwo23, 0x7632u); hb[5] = prmt(w1.y, kTwo23, 0x7632u);
@@ -234,11 +231,25 @@ __device__ __forceinline__ void octet_levels(const float4 xa, const float4 xb, u
   float worst = 0.0f;
 #pragma unroll
   for (int i = 0; i < 8; ++i) z[i] = round_signed(x[i], hb[i], rc, &worst);
-  if (!(worst <= rc.thr)) {                                      // some coordinate of the octet needs the exact routine
+  if (!(worst <= rc.thr)) {                             // some coordinate of the octet needs the exact routine
     const uint64_t fixed = redo_octet<RNG>(xa, xb, w0, w1, oct, k, xid, &key, rc, norm, lev, nlev);
 #pragma unroll
     for (int i = 0; i < 8; ++i) z[i] = __fmul_rn((float)(int)(signed char)(uint8_t)(fixed >> (8 * i)), S);
   }
+}
+
+template <int RNG>
+__device__ __forceinline__ void octet_levels(const float4 xa, const float4 xb, uint64_t oct, uint32_t k, uint32_t xid,
+                                             const PhiloxKey& key, const RoundK& rc, float norm, float S,
+                                             const float* lev, int nlev, float* z) {
+  uint4 w0, w1;
+  if (RNG == QGX_RNG_HALF32) {
+    w0 = philox4x32_10((uint32_t)oct, (uint32_t)(oct >> 32), k, xid, key);
+    w1 = w0;
+  } else {
+    philox4x32_10_x2(2ull * oct, 2ull * oct + 1ull, k, xid, key, &w0, &w1);
+  }
+  octet_levels_w<RNG>(xa, xb, w0, w1, oct, k, xid, key, rc, norm, S, lev, nlev, z);
 }
 
 // the pair table's entry for two consecutive coordinates, at byte 4 * ((first + 64 * second) mod 4096) of the
@@ -259,7 +270,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
                   const __grid_constant__ RoundTable rt) {
   extern __shared__ __align__(16) uint32_t s_dyn[];
-  __shared__ float4 s_bin[kBinEntries];
+  __shared__ __align__(128) float4 s_bin[kBinEntries];
   __shared__ EncLut s_lut;
   __shared__ uint32_t s_pair[kPairLutSize];
   __shared__ float s_lev[QGX_MAX_LEVELS];
