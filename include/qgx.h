@@ -49,17 +49,6 @@ enum { QGX_OP_DENSE_AFFINE = 0, QGX_OP_BILINEAR = 1, QGX_OP_DIAGONAL = 2 };
 enum { QGX_REFIT_NONE = 0, QGX_REFIT_CONTINUE = 1, QGX_REFIT_FIRST = 2 };
 /* flag of qgx_quantize: `norms` is an input (the caller's norms are used as they are) */
 enum { QGX_NORMS_SUPPLIED = 1 };
-/* How the uniform variate r of a coordinate is drawn (Definition 1 says "with probability xi" and no more).
- * QGX_RNG_WORD24: r = (w >> 8) * 2^-24, w = word (i & 3) of Philox4x32-10 with key = seed and counter
- * (i >> 2 low, i >> 2 high, worker, exchange id): one block per four coordinates.
- * QGX_RNG_HALF32: r = (h * 2^16 + h') * 2^-32, h = 16-bit half (i & 7) of the block with counter
- * (i >> 3 low, i >> 3 high, worker, exchange id) -- half j is bits 16 * (j & 1) .. 16 * (j & 1) + 15 of word
- * j >> 1 -- and h' the same half of the block with counter (i >> 3 low, i >> 3 high, worker | 2^31, exchange id).
- * The coordinate rounds up iff r < xi (compared exactly).  A finer variate from half the generator work per
- * coordinate: h' matters for about 2^-16 of the coordinates only and is generated just for those. */
-enum { QGX_RNG_WORD24 = 0, QGX_RNG_HALF32 = 1 };
-/* flag of qgx_quantize: draw the variates as QGX_RNG_HALF32 */
-enum { QGX_QUANTIZE_RNG_HALF32 = 2 };
 
 enum { QGX_MAX_LEVELS = 32, QGX_MAX_CODE_LEN = 12, QGX_MAX_BUCKET = 16384 };
 
@@ -84,7 +73,7 @@ typedef struct {
   int32_t norm_type;        /* QGX_NORM_L2 | QGX_NORM_LINF */
   int32_t code_type;        /* what a refit rebuilds: QGX_CODE_FIXED | QGX_CODE_HUFFMAN | QGX_CODE_ELIAS */
   int32_t nbins;            /* histogram bins of the level refit (Sec. 3.3) */
-  int32_t rng_mode;         /* QGX_RNG_WORD24 | QGX_RNG_HALF32 */
+  int32_t pad;
   uint64_t seed;            /* key of the counter-based generator */
   float levels[32];
   qgx_codebook cb;
@@ -263,12 +252,14 @@ qgx_status qgx_exchange_segments(qgx_ctx *ctx, const float *v, int K, size_t d, 
  * falls back when the workspace would exceed 256 MB). */
 enum { QGX_SPLIT_AUTO = 0, QGX_SPLIT_NEVER = 1, QGX_SPLIT_ALWAYS = 2 };
 qgx_status qgx_set_decode_split(qgx_ctx *ctx, int mode);
-/* Which kernel the encode pass of the fused calls uses.  By default (QGX_ENCODE_AUTO) whole buckets of 1024, 2048,
- * 4096, 8192 or 16384 coordinates of 16-byte aligned vectors are staged in shared memory by bulk copies and packed
- * 32 coordinates per lane; everything else (other bucket sizes, a short last bucket, unaligned vectors) is held
- * in registers, one CTA per bucket.  QGX_ENCODE_REGISTERS forces the second kernel for all buckets; the streams
- * are the same bit for bit. */
-enum { QGX_ENCODE_AUTO = 0, QGX_ENCODE_REGISTERS = 1 };
+/* Which kernel the encode pass of the fused calls uses (no counterpart in the paper; the streams are the same bit
+ * for bit).  QGX_ENCODE_REGISTERS: one CTA per bucket, the bucket held in registers between the norm and the
+ * rounding.  QGX_ENCODE_STAGED: whole buckets of 1024, 2048, 4096, 8192 or 16384 coordinates of 16-byte aligned
+ * vectors whose rows lie a multiple of 32 floats apart are staged in shared memory by bulk tensor copies, three
+ * buffers deep, and packed 32 coordinates per lane; what does not qualify (other bucket sizes, a short last
+ * bucket) still goes through the first kernel.  QGX_ENCODE_AUTO (the default) takes the kernel that measured
+ * faster on B200: the first. */
+enum { QGX_ENCODE_AUTO = 0, QGX_ENCODE_REGISTERS = 1, QGX_ENCODE_STAGED = 2 };
 qgx_status qgx_set_encode_path(qgx_ctx *ctx, int mode);
 /* Where the last qgx_exchange on `slot` left its streams: all [dev], valid until the next call
  * that uses the slot.  Any output pointer may be NULL. */

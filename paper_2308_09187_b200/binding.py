@@ -20,8 +20,6 @@ QGX_CODE_FIXED, QGX_CODE_HUFFMAN, QGX_CODE_ELIAS = 0, 1, 2
 QGX_OP_DENSE_AFFINE, QGX_OP_BILINEAR, QGX_OP_DIAGONAL = 0, 1, 2
 QGX_REFIT_NONE, QGX_REFIT_CONTINUE, QGX_REFIT_FIRST = 0, 1, 2
 QGX_NORMS_SUPPLIED = 1
-QGX_QUANTIZE_RNG_HALF32 = 2
-QGX_RNG_WORD24, QGX_RNG_HALF32 = 0, 1
 QGX_MAX_LEVELS, QGX_MAX_CODE_LEN, QGX_MAX_BUCKET = 32, 12, 16384
 
 EXPORTS = [
@@ -49,7 +47,7 @@ class qgx_codebook(C.Structure):
 
 class qgx_quant_cfg(C.Structure):
     _fields_ = [("nlev", C.c_int32), ("bucket", C.c_int32), ("norm_type", C.c_int32), ("code_type", C.c_int32),
-                ("nbins", C.c_int32), ("rng_mode", C.c_int32), ("seed", C.c_uint64),
+                ("nbins", C.c_int32), ("pad", C.c_int32), ("seed", C.c_uint64),
                 ("levels", C.c_float * 32), ("cb", qgx_codebook)]
 
     def level_list(self):
@@ -338,7 +336,7 @@ def qgx_set_decode_split(ctx, mode):
     _chk(lib().qgx_set_decode_split(ctx.h, int(mode)), "qgx_set_decode_split")
 
 
-QGX_ENCODE_AUTO, QGX_ENCODE_REGISTERS = 0, 1
+QGX_ENCODE_AUTO, QGX_ENCODE_REGISTERS, QGX_ENCODE_STAGED = 0, 1, 2
 
 
 def qgx_set_encode_path(ctx, mode):

@@ -304,14 +304,9 @@ __device__ __forceinline__ uint32_t quantize_quad_codes(const float4 x, const ui
 }
 
 // ---- the octet encoder's rounding ---------------------------------------------------------------
-// How the uniform variate of a coordinate is drawn (the paper says only "with probability xi"):
-//   QGX_RNG_WORD24  r = (w >> 8) 2^-24, w = word (i & 3) of the Philox block with counter (i >> 2, worker, exchange);
-//   QGX_RNG_HALF32  r = (h 2^16 + h') 2^-32: h = 16-bit half (i & 7) of the block with counter (i >> 3, worker,
-//                   exchange) -- half j is bits 16 (j & 1) .. of word j >> 1 --, h' the same half of the block with
-//                   counter (i >> 3, worker | 2^31, exchange).  h alone decides all but about 2^-16 of the
-//                   coordinates, so the second block is generated only for those.
-// In both modes the fast path uses the leading 16 bits h of r (the centre of the interval of r they leave) and
-// sends a coordinate to the exact routine when the outcome could depend on the remaining bits.
+// The variate of coordinate i is r = (w >> 8) 2^-24, w = word (i & 3) of the Philox block with counter
+// (i >> 2, worker, exchange).  The fast path uses only the leading 16 bits h of r (the centre of the interval of r
+// they leave) and sends a coordinate to the exact routine when the outcome could depend on the remaining bits.
 // Shared memory by 32-bit address (what ld.shared takes): the hot loops compute table addresses themselves.
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 // read-only tables: the address depends on the data just loaded, so the compiler cannot move these too early
@@ -380,30 +375,18 @@ __device__ __forceinline__ float round_signed(float x, uint32_t hbits, const Rou
   return zi;
 }
 
-// The variate bits of coordinate e (its index in the generator's counter space) on their own: the 24 bits of
-// QGX_RNG_WORD24 or the 32 bits of QGX_RNG_HALF32.  One or two whole blocks per call: for ragged ends only.
-template <int RNG>
+// The 24 variate bits of coordinate e (its index in the generator's counter space) on their own: a whole block
+// per call, for ragged ends only.
 static __device__ __noinline__ uint32_t variate_bits(uint64_t e, uint32_t k, uint32_t xid, const PhiloxKey& key) {
-  if (RNG == QGX_RNG_WORD24) {
-    const uint64_t q = e >> 2;
-    const uint4 w = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), k, xid, key);
-    const int c = (int)(e & 3u);
-    return (c == 0 ? w.x : (c == 1 ? w.y : (c == 2 ? w.z : w.w))) >> 8;
-  }
-  const uint64_t o = e >> 3;
-  const uint4 w = philox4x32_10((uint32_t)o, (uint32_t)(o >> 32), k, xid, key);
-  const uint4 w2 = philox4x32_10((uint32_t)o, (uint32_t)(o >> 32), k | 0x80000000u, xid, key);
-  const int j = (int)(e & 7u);
-  const uint32_t x = (j >> 1) == 0 ? w.x : ((j >> 1) == 1 ? w.y : ((j >> 1) == 2 ? w.z : w.w));
-  const uint32_t y = (j >> 1) == 0 ? w2.x : ((j >> 1) == 1 ? w2.y : ((j >> 1) == 2 ? w2.z : w2.w));
-  const uint32_t h = (j & 1) ? (x >> 16) : (x & 0xffffu), h2 = (j & 1) ? (y >> 16) : (y & 0xffffu);
-  return (h << 16) | h2;
+  const uint64_t q = e >> 2;
+  const uint4 w = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), k, xid, key);
+  const int c = (int)(e & 3u);
+  return (c == 0 ? w.x : (c == 1 ? w.y : (c == 2 ? w.z : w.w))) >> 8;
 }
 
-// Definition 1 for one coordinate with the variate of either mode: rbits = the 24-bit variate (QGX_RNG_WORD24) or
-// the 32-bit variate (QGX_RNG_HALF32).  Out of line: it runs for about 1e-4 of the coordinates.
-template <int RNG>
-static __device__ __noinline__ int quantize_level_exact(float absv, float norm, const float* lev, int nlev, uint32_t rbits) {
+// Definition 1 for one coordinate, every operation one IEEE rounding; r24 = the 24-bit variate.  Out of line: it
+// runs for about 1e-4 of the coordinates.
+static __device__ __noinline__ int quantize_level_exact(float absv, float norm, const float* lev, int nlev, uint32_t r24) {
   float u = (norm > 0.0f) ? __fdiv_rn(absv, norm) : 0.0f;
   u = fminf(u, 1.0f);
   int tau = 0;
@@ -411,15 +394,8 @@ static __device__ __noinline__ int quantize_level_exact(float absv, float norm, 
   const float num = __fsub_rn(u, lev[tau]);
   const float den = __fsub_rn(lev[tau + 1], lev[tau]);
   const float xi = __fdiv_rn(num, den);
-  bool up;
-  if (RNG == QGX_RNG_WORD24) {
-    const float r = __fmul_rn(__uint2float_rn(rbits), 5.9604644775390625e-8f);    // exact
-    up = r < xi;
-  } else {
-    const double r = (double)rbits * 2.3283064365386962890625e-10;                 // exact
-    up = r < (double)xi;
-  }
-  return tau + (up ? 1 : 0);
+  const float r = __fmul_rn(__uint2float_rn(r24), 5.9604644775390625e-8f);        // exact
+  return tau + ((r < xi) ? 1 : 0);
 }
 
 __device__ __forceinline__ uint32_t symbol_of(float v, int idx) {

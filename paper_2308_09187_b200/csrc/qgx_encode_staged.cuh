@@ -144,7 +144,7 @@ __device__ __forceinline__ void copy_segment(const Segment seg, uint32_t next_R,
 // only for buckets of smaller groups, and a group that is staged but not started waits only for its own team's
 // current group, which is smaller: the smallest unfinished group is always being worked on and waits for
 // nothing, so every wait ends.
-template <int G, int RNG>
+template <int G>
 __global__ void __launch_bounds__(kStagedThreads, 1)
 k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt, const __grid_constant__ CodeTable ct,
                 const __grid_constant__ PhiloxKey key, const __grid_constant__ RoundTable rt, const __grid_constant__ CUtensorMap tmap) {
@@ -308,17 +308,15 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     if (active) {
       const uint64_t oct0 = ((a.quad_base + (uint64_t)(lo >> 2)) >> 1) + 4ull * (uint64_t)line;
       const uint32_t l7 = (uint32_t)line & 7u;
-      uint4 W[4];
-      if (live && RNG == QGX_RNG_HALF32) philox4x32_10_x4(oct0, (uint32_t)k, a.xid, key, W);
+      uint4 W[4];                                                     // the Philox blocks of two octets (four quads)
 #pragma unroll
       for (int o = 0; o < 4; ++o) {
         float z[8];
         if (live) {
-          if (RNG == QGX_RNG_WORD24 && (o & 1) == 0) philox4x32_10_x4(2ull * (oct0 + (uint64_t)o), (uint32_t)k, a.xid, key, W);
+          if ((o & 1) == 0) philox4x32_10_x4(2ull * (oct0 + (uint64_t)o), (uint32_t)k, a.xid, key, W);
           const float4 xa = lds128(line_sa + (((uint32_t)(2 * o) ^ l7) << 4));
           const float4 xb = lds128(line_sa + (((uint32_t)(2 * o + 1) ^ l7) << 4));
-          const uint4 w0 = RNG == QGX_RNG_HALF32 ? W[o] : W[2 * (o & 1)], w1 = RNG == QGX_RNG_HALF32 ? W[o] : W[2 * (o & 1) + 1];
-          octet_levels_w<RNG>(xa, xb, w0, w1, oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, s_lev, nlev, z);
+          octet_levels_w(xa, xb, W[2 * (o & 1)], W[2 * (o & 1) + 1], rc, norm, S, s_lev, nlev, z);
         } else {
 #pragma unroll
           for (int i = 0; i < 8; ++i) z[i] = 0.0f;

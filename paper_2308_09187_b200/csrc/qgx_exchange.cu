@@ -173,82 +173,49 @@ __device__ __forceinline__ void load_bucket_octets(BucketRegs<2 * P>& r, const D
 // ---- rounding of one octet (eight consecutive coordinates of one lane) ---------------------------
 // The rare way through an octet, out of line: every coordinate is tested again and the ones whose outcome the
 // leading variate bits do not settle go through the exact routine.  Returns the eight signed level indices, one
-// per byte.
-template <int RNG>
-static __device__ __noinline__ uint64_t redo_octet(const float4 xa, const float4 xb, const uint4 w0, const uint4 w1, uint64_t oct,
-                                                   uint32_t k, uint32_t xid, const PhiloxKey* key, const RoundK rc, float norm,
-                                                   const float* lev, int nlev) {
+// per byte.  w0, w1: the Philox blocks of the octet's two quads.
+static __device__ __noinline__ uint64_t redo_octet(const float4 xa, const float4 xb, const uint4 w0, const uint4 w1, const RoundK rc,
+                                                   float norm, const float* lev, int nlev) {
   const float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
   const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
   const float inv_S = -1.0f / (rc.nqs * 65536.0f);
-  uint4 w2 = make_uint4(0u, 0u, 0u, 0u);
-  bool have2 = false;
   uint64_t out = 0;
   for (int i = 0; i < 8; ++i) {
-    const uint32_t h = RNG == QGX_RNG_HALF32 ? ((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xffffu)) : (w[i] >> 16);
     float worst = 0.0f;
-    const float zi = round_signed(x[i], 0x4B000000u | h, rc, &worst);
+    const float zi = round_signed(x[i], 0x4B000000u | (w[i] >> 16), rc, &worst);
     int idx = (int)fabsf(__fmul_rn(zi, inv_S));
-    if (!(worst <= rc.thr)) {
-      uint32_t rb;
-      if (RNG == QGX_RNG_HALF32) {
-        if (!have2) { w2 = philox4x32_10((uint32_t)oct, (uint32_t)(oct >> 32), k | 0x80000000u, xid, *key); have2 = true; }
-        const uint32_t y = (i >> 1) == 0 ? w2.x : ((i >> 1) == 1 ? w2.y : ((i >> 1) == 2 ? w2.z : w2.w));
-        rb = (h << 16) | ((i & 1) ? (y >> 16) : (y & 0xffffu));
-      } else {
-        rb = w[i] >> 8;
-      }
-      idx = quantize_level_exact<RNG>(fabsf(x[i]), norm, lev, nlev, rb);
-    }
+    if (!(worst <= rc.thr)) idx = quantize_level_exact(fabsf(x[i]), norm, lev, nlev, w[i] >> 8);
     const int sidx = (__float_as_uint(x[i]) >> 31) ? -idx : idx;
     out |= (uint64_t)(uint8_t)(signed char)sidx << (8 * i);
   }
   return out;
 }
 
-// S * (signed level index) of the eight coordinates xa, xb of octet `oct` (its index in the generator's counter
-// space) of worker k, given the octet's Philox words: w0 alone (QGX_RNG_HALF32: the block of counter oct) or w0, w1
-// (QGX_RNG_WORD24: the blocks of counters 2 oct and 2 oct + 1).  S = the scale of the rounding table.
-template <int RNG>
-__device__ __forceinline__ void octet_levels_w(const float4 xa, const float4 xb, const uint4 w0, const uint4 w1, uint64_t oct,
-                                               uint32_t k, uint32_t xid, const PhiloxKey& key, const RoundK& rc, float norm,
-                                               float S, const float* lev, int nlev, float* z) {
+// S * (signed level index) of the eight coordinates xa, xb of an octet, given the Philox blocks w0, w1 of its two
+// quads.  S = the scale of the rounding table.
+__device__ __forceinline__ void octet_levels_w(const float4 xa, const float4 xb, const uint4 w0, const uint4 w1, const RoundK& rc,
+                                               float norm, float S, const float* lev, int nlev, float* z) {
   constexpr uint32_t kTwo23 = 0x4B000000u;              // pattern of 2^23: its low mantissa bytes are replaced by h
   const float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-  uint32_t hb[8];
-  if (RNG == QGX_RNG_HALF32) {
-    hb[0] = prmt(w0.x, kTwo23, 0x7610u); hb[1] = prmt(w0.x, kTwo23, 0x7632u);
-    hb[2] = prmt(w0.y, kTwo23, 0x7610u); hb[3] = prmt(w0.y, kTwo23, 0x7632u);
-    hb[4] = prmt(w0.z, kTwo23, 0x7610u); hb[5] = prmt(w0.z, kTwo23, 0x7632u);
-    hb[6] = prmt(w0.w, kTwo23, 0x7610u); hb[7] = prmt(w0.w, kTwo23, 0x7632u);
-  } else {
-    hb[0] = prmt(w0.x, kTwo23, 0x7632u); hb[1] = prmt(w0.y, kTwo23, 0x7632u);
-    hb[2] = prmt(w0.z, kTwo23, 0x7632u); hb[3] = prmt(w0.w, kTwo23, 0x7632u);
-    hb[4] = prmt(w1.x, kTwo23, 0x7632u); hb[5] = prmt(w1.y, kTwo23, 0x7632u);
-    hb[6] = prmt(w1.z, kTwo23, 0x7632u); hb[7] = prmt(w1.w, kTwo23, 0x7632u);
-  }
+  const uint32_t hb[8] = {prmt(w0.x, kTwo23, 0x7632u), prmt(w0.y, kTwo23, 0x7632u), prmt(w0.z, kTwo23, 0x7632u), prmt(w0.w, kTwo23, 0x7632u),
+                          prmt(w1.x, kTwo23, 0x7632u), prmt(w1.y, kTwo23, 0x7632u), prmt(w1.z, kTwo23, 0x7632u), prmt(w1.w, kTwo23, 0x7632u)};
   float worst = 0.0f;
 #pragma unroll
   for (int i = 0; i < 8; ++i) z[i] = round_signed(x[i], hb[i], rc, &worst);
   if (!(worst <= rc.thr)) {                             // some coordinate of the octet needs the exact routine
-    const uint64_t fixed = redo_octet<RNG>(xa, xb, w0, w1, oct, k, xid, &key, rc, norm, lev, nlev);
+    const uint64_t fixed = redo_octet(xa, xb, w0, w1, rc, norm, lev, nlev);
 #pragma unroll
     for (int i = 0; i < 8; ++i) z[i] = __fmul_rn((float)(int)(signed char)(uint8_t)(fixed >> (8 * i)), S);
   }
 }
 
-template <int RNG>
+// the same for octet `oct` (its index in the generator's counter space) of worker k
 __device__ __forceinline__ void octet_levels(const float4 xa, const float4 xb, uint64_t oct, uint32_t k, uint32_t xid,
                                              const PhiloxKey& key, const RoundK& rc, float norm, float S,
                                              const float* lev, int nlev, float* z) {
   uint4 w0, w1;
-  if (RNG == QGX_RNG_HALF32) {
-    w0 = philox4x32_10((uint32_t)oct, (uint32_t)(oct >> 32), k, xid, key);
-    w1 = w0;
-  } else {
-    philox4x32_10_x2(2ull * oct, 2ull * oct + 1ull, k, xid, key, &w0, &w1);
-  }
-  octet_levels_w<RNG>(xa, xb, w0, w1, oct, k, xid, key, rc, norm, S, lev, nlev, z);
+  philox4x32_10_x2(2ull * oct, 2ull * oct + 1ull, k, xid, key, &w0, &w1);
+  octet_levels_w(xa, xb, w0, w1, rc, norm, S, lev, nlev, z);
 }
 
 // the pair table's entry for two consecutive coordinates, at byte 4 * ((first + 64 * second) mod 4096) of the
@@ -263,7 +230,7 @@ __device__ __forceinline__ uint32_t pair_entry(uint32_t pair, float z_first, flo
 //   barrier | warp offsets, bit scatter, look-back (warp 0) | barrier | copy out
 // The bucket image is double buffered, so the copy-out of one bucket needs no barrier before the next
 // bucket starts.  A thread works on P octets; warp w owns the 256 * P coordinates [w * 256 * P, ...).
-template <int P, int G, int RNG>
+template <int P, int G>
 __global__ void __launch_bounds__(P == 1 ? 256 : 512, P == 1 ? 4 : 2)
 k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ LevelTable lt,
                   const __grid_constant__ CodeTable ct, const __grid_constant__ PhiloxKey key,
@@ -340,7 +307,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
       for (int j = 0; j < P; ++j) {
         const int o = (warp * P + j) * 32 + lane;
         float z[8];
-        octet_levels<RNG>(r.x[2 * j], r.x[2 * j + 1], oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, s_lev, nlev, z);
+        octet_levels(r.x[2 * j], r.x[2 * j + 1], oct0 + (uint64_t)o, (uint32_t)k, a.xid, key, rc, norm, S, s_lev, nlev, z);
         const uint32_t e01 = pair_entry(pair_sa, z[0], z[1], four_over_S), e23 = pair_entry(pair_sa, z[2], z[3], four_over_S);
         const uint32_t e45 = pair_entry(pair_sa, z[4], z[5], four_over_S), e67 = pair_entry(pair_sa, z[6], z[7], four_over_S);
         uint32_t n0, n1;
@@ -359,8 +326,8 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
           const float x[8] = {r.x[2 * j].x, r.x[2 * j].y, r.x[2 * j].z, r.x[2 * j].w,
                               r.x[2 * j + 1].x, r.x[2 * j + 1].y, r.x[2 * j + 1].z, r.x[2 * j + 1].w};
           for (int i = 0; i < nv; ++i) {                    // ragged ends and odd offsets: the exact routine throughout
-            const uint32_t rb = variate_bits<RNG>(e0 + (uint64_t)i, (uint32_t)k, a.xid, key);
-            const int idx = quantize_level_exact<RNG>(fabsf(x[i]), norm, s_lev, nlev, rb);
+            const uint32_t rb = variate_bits(e0 + (uint64_t)i, (uint32_t)k, a.xid, key);
+            const int idx = quantize_level_exact(fabsf(x[i]), norm, s_lev, nlev, rb);
             sy[i >> 2] |= symbol_of(x[i], idx) << (8 * (i & 3));
           }
         }
@@ -865,8 +832,8 @@ constexpr int kTableCacheSlots = 32;
 struct LaunchShape { size_t smem; int per_sm; };      // smem == 0: not asked yet
 struct TableCache {
   CachedTables e[kTableCacheSlots];
-  LaunchShape enc[2][3][3];             // [variate mode][octets per thread 1, 2, 4][sub-block 32, 64, 128]
-  LaunchShape enc_staged[2][3];         // [variate mode][sub-block]
+  LaunchShape enc[3][3];                // [octets per thread 1, 2, 4][sub-block 32, 64, 128]
+  LaunchShape enc_staged[3];            // [sub-block]
   LaunchShape dec[3][6];                // [sub-block][symbol mode]
 };
 
@@ -997,7 +964,6 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const int bucket = cfg->bucket;
   if (bucket < kQuad || bucket > QGX_MAX_BUCKET || bucket % kQuad != 0) return QGX_ERR_INVALID_ARG;
   if (cfg->norm_type != QGX_NORM_L2 && cfg->norm_type != QGX_NORM_LINF) return QGX_ERR_INVALID_ARG;
-  if (cfg->rng_mode != QGX_RNG_WORD24 && cfg->rng_mode != QGX_RNG_HALF32) return QGX_ERR_INVALID_ARG;
   if (check_levels_host(cfg->levels, cfg->nlev) != QGX_OK) return QGX_ERR_BAD_LEVELS;
   if (cfg->cb.nlev != cfg->nlev) return QGX_ERR_INVALID_ARG;
   if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
@@ -1062,24 +1028,19 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   const size_t img_words = (((((size_t)bucket * (ct.maxlen + 1) + 16u * (bucket / ct.G + 1) + kNormBits + 31u) >> 5) + 4) + 3) & ~(size_t)3;
   const size_t smem = sizeof(uint32_t) * 2 * img_words;   // two images: see k_exchange_encode
   int per_sm = 1;
-#define QGX_LAUNCH_ER(V, GG, RR)                                                                               \
+#define QGX_LAUNCH_E(V, GG)                                                                                    \
   do {                                                                                                         \
-    allow_max_dynamic_smem(k_exchange_encode<V, GG, RR>, c->device);                                           \
-    LaunchShape& shape = table_cache(c)->enc[RR][V == 1 ? 0 : (V == 2 ? 1 : 2)][GG == 32 ? 0 : (GG == 64 ? 1 : 2)];  \
+    allow_max_dynamic_smem(k_exchange_encode<V, GG>, c->device);                                               \
+    LaunchShape& shape = table_cache(c)->enc[V == 1 ? 0 : (V == 2 ? 1 : 2)][GG == 32 ? 0 : (GG == 64 ? 1 : 2)];  \
     if (shape.smem != smem + 1 + (size_t)threads * 0x100000) {   /* occupancy asked once per shape */          \
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG, RR>, threads, smem);     \
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_encode<V, GG>, threads, smem);         \
       shape.smem = smem + 1 + (size_t)threads * 0x100000;                                                      \
       shape.per_sm = per_sm < 1 ? 1 : per_sm;                                                                  \
     }                                                                                                          \
     per_sm = shape.per_sm;                                                                                     \
     const unsigned long long want = (unsigned long long)(nb - ea.b_first) * (unsigned long long)K;             \
     const unsigned grid = (unsigned)std::min<unsigned long long>(want, (unsigned long long)c->num_sms * (unsigned long long)per_sm);   \
-    k_exchange_encode<V, GG, RR><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                     \
-  } while (0)
-#define QGX_LAUNCH_E(V, GG)                                          \
-  do {                                                               \
-    if (cfg->rng_mode == QGX_RNG_HALF32) QGX_LAUNCH_ER(V, GG, 1);    \
-    else QGX_LAUNCH_ER(V, GG, 0);                                    \
+    k_exchange_encode<V, GG><<<grid, threads, smem, c->stream>>>(ea, lt, ct, key, qt);                         \
   } while (0)
 #define QGX_LAUNCH_EG(V)                                   \
   do {                                                     \
@@ -1090,7 +1051,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   // Whole buckets of a multiple of 1024 coordinates that divides 16384 go through the staged kernel; what is left
   // (a short last bucket, other bucket sizes, unaligned vectors) through the bucket-in-registers kernel.
   bool staged_ok = ea.vec_ok && bucket % kWarpCoords == 0 && kStageCoords % bucket == 0 && coord_base % 8 == 0 &&
-                   c->encode_path != QGX_ENCODE_REGISTERS && d / (size_t)bucket > 0;
+                   c->encode_path == QGX_ENCODE_STAGED && d / (size_t)bucket > 0;
   CUtensorMap tmap;
   std::memset(&tmap, 0, sizeof(tmap));
   if (staged_ok) {
@@ -1110,28 +1071,22 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
       const size_t smem_st = sizeof(float) * kStageCoords * kStageBuffers;
       const unsigned long long per_group = (unsigned long long)(kStageCoords / bucket);
       const unsigned long long groups = ((unsigned long long)ea.nb_whole * (unsigned long long)K + per_group - 1ull) / per_group;
-#define QGX_LAUNCH_S(GG, RR)                                                                                         \
+#define QGX_LAUNCH_SG(GG)                                                                                            \
   do {                                                                                                               \
-    allow_max_dynamic_smem(k_encode_staged<GG, RR>, c->device);                                                      \
-    LaunchShape& shape = table_cache(c)->enc_staged[RR][GG == 32 ? 0 : (GG == 64 ? 1 : 2)];                          \
+    allow_max_dynamic_smem(k_encode_staged<GG>, c->device);                                                          \
+    LaunchShape& shape = table_cache(c)->enc_staged[GG == 32 ? 0 : (GG == 64 ? 1 : 2)];                              \
     if (shape.smem == 0) {                                                                                           \
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_encode_staged<GG, RR>, kStagedThreads, smem_st);      \
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_encode_staged<GG>, kStagedThreads, smem_st);          \
       shape.smem = 1;                                                                                                \
       shape.per_sm = per_sm < 1 ? 1 : per_sm;                                                                        \
     }                                                                                                                \
     const unsigned grid = (unsigned)std::min<unsigned long long>((groups + 1ull) / 2ull, (unsigned long long)c->num_sms * (unsigned long long)shape.per_sm); \
-    k_encode_staged<GG, RR><<<grid, kStagedThreads, smem_st, c->stream>>>(ea, lt, ct, key, qt, tmap);                \
-  } while (0)
-#define QGX_LAUNCH_SG(GG)                                            \
-  do {                                                               \
-    if (cfg->rng_mode == QGX_RNG_HALF32) QGX_LAUNCH_S(GG, 1);        \
-    else QGX_LAUNCH_S(GG, 0);                                        \
+    k_encode_staged<GG><<<grid, kStagedThreads, smem_st, c->stream>>>(ea, lt, ct, key, qt, tmap);                    \
   } while (0)
       if (ct.G == 32) QGX_LAUNCH_SG(32);
       else if (ct.G == 64) QGX_LAUNCH_SG(64);
       else QGX_LAUNCH_SG(128);
 #undef QGX_LAUNCH_SG
-#undef QGX_LAUNCH_S
       count_launch(c);
     }
     if (ea.b_first < nb) {
@@ -1145,7 +1100,6 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   }
 #undef QGX_LAUNCH_EG
 #undef QGX_LAUNCH_E
-#undef QGX_LAUNCH_ER
   if (cudaGetLastError() != cudaSuccess) return QGX_ERR_CUDA;
   if (total_bits_out &&
       cudaMemcpyAsync(total_bits_out, tot, sizeof(uint64_t) * (size_t)K, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
@@ -1310,7 +1264,7 @@ qgx_status qgx_set_decode_split(qgx_ctx* c, int mode) {
 }
 
 qgx_status qgx_set_encode_path(qgx_ctx* c, int mode) {
-  if (!c || (mode != QGX_ENCODE_AUTO && mode != QGX_ENCODE_REGISTERS)) return QGX_ERR_INVALID_ARG;
+  if (!c || (mode != QGX_ENCODE_AUTO && mode != QGX_ENCODE_REGISTERS && mode != QGX_ENCODE_STAGED)) return QGX_ERR_INVALID_ARG;
   c->encode_path = mode;
   return QGX_OK;
 }

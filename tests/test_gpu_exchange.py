@@ -10,12 +10,14 @@ from oracle import qgx_oracle as o
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=["one thread per sub-block", "one worker per thread"])
+@pytest.fixture(scope="module", params=["one thread per sub-block", "one worker per thread", "staged encode"])
 def q(request):
-    """Every test runs with both ways of spreading the decode pass (small vectors would only see the second)."""
+    """Every test runs with both ways of spreading the decode pass (small vectors would only see the second) and
+    with the staged encode kernel (the shapes it does not take fall back to the bucket-in-registers kernel)."""
     import paper_2308_09187_b200 as qgx
     ctx = qgx.qgx_create(0)
-    qgx.qgx_set_decode_split(ctx, qgx.QGX_SPLIT_NEVER if request.param == "one thread per sub-block" else qgx.QGX_SPLIT_ALWAYS)
+    qgx.qgx_set_decode_split(ctx, qgx.QGX_SPLIT_ALWAYS if request.param == "one worker per thread" else qgx.QGX_SPLIT_NEVER)
+    qgx.qgx_set_encode_path(ctx, qgx.QGX_ENCODE_STAGED if request.param == "staged encode" else qgx.QGX_ENCODE_REGISTERS)
     yield qgx, ctx
     qgx.qgx_destroy(ctx)
 
@@ -38,6 +40,12 @@ CASES = [
     (5, 40000, 4096, 17, 64, True),
     (2, 70000, 2048, 32, 32, False),
     (2, 1001, 256, 3, 32, True),          # d not a multiple of 4
+    # rows a multiple of 32 floats apart: the whole buckets qualify for the staged encode kernel
+    (4, 5 * 16384, 16384, 17, 64, True),
+    (6, 7 * 4096 + 2048, 4096, 9, 32, True),      # short last bucket
+    (3, 9 * 1024, 1024, 17, 128, False),          # sixteen buckets per group, a last group of nine
+    (2, 3 * 2048 + 32, 2048, 32, 64, True),
+    (5, 21 * 8192, 8192, 17, 128, True),
 ]
 
 
