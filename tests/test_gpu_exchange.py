@@ -206,5 +206,5 @@ def test_elias_recursive_code(q, K, d, bucket, nlev, sub):
     # a refit moves the levels and leaves this code in place
     qgx.qgx_update_levels(ctx, v, cfg, qgx.QGX_REFIT_FIRST)
     lev_ref, _ = o.refit(vh, bucket, 1024, lev.copy(), cbo, True, o.CODE_ELIAS)
-    assert np.max(np.abs(np.array(cfg.level_list(), dtype=np.float32) - lev_ref)) < 5e-5
+    assert np.max(np.abs(np.array(cfg.level_list(), dtype=np.float32) - lev_ref)) <= 1e-6
     assert cfg.cb.codes() == cbo.codes() and cfg.cb.lengths() == cbo.lengths() and cfg.cb.subblock == sub

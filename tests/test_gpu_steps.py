@@ -89,6 +89,24 @@ def test_quantize_encode_decode_average(q, K, d, bucket, nlev, sub):
     assert np.array_equal(out.cpu().numpy(), o.average(n_gpu, s_ref, bucket, lev))
 
 
+def test_supplied_norms_smaller_than_the_coordinates(q):
+    """Norms handed in by the caller are used as they are: where one is smaller than a coordinate's magnitude the
+    normalized coordinate is clamped to 1 (the top level), as in the oracle; nothing is read out of range."""
+    qgx, ctx = q
+    K, d, bucket, nlev = 3, 5 * 2048 + 100, 2048, 17
+    v = gen.gaussian_mixture((K, d), seed=5, device="cuda")
+    vh = v.cpu().numpy()
+    lev = np.r_[0.0, np.sort(np.random.default_rng(5).uniform(0.001, 0.3, nlev - 2)), 1.0].astype(np.float32)
+    for factor in (0.5, 0.01):
+        n_small = (o.bucket_norms(vh, bucket) * np.float32(factor)).astype(np.float32)
+        _, sym = qgx.qgx_quantize(ctx, v, bucket, lev, qgx.QGX_NORM_L2, 17, 4, flags=qgx.QGX_NORMS_SUPPLIED,
+                                  norms=torch.from_numpy(n_small).cuda())
+        qgx.qgx_sync_status(ctx)
+        s_ref = o.quantize(vh, bucket, lev, n_small, 17, 4)
+        assert np.array_equal(sym.cpu().numpy(), s_ref)
+        assert np.count_nonzero((s_ref & 31) == nlev - 1) > 0          # some coordinates did exceed their norm
+
+
 LEVEL_SETS = {
     "uniform17": np.linspace(0, 1, 17),
     "uniform32": np.linspace(0, 1, 32),

@@ -5,14 +5,15 @@ is being recorded into a CUDA stream capture, or a service whose GPU memory is h
 start-up.  For them the library has a second encode entry point whose scratch (bucket offsets and
 overflow flags) is a fixed array inside the library instead of a cudaMalloc'ed workspace.  This test
 calls it through the C ABI twice in a row, on different shapes so that the second call finds the
-first call's leftovers in the shared scratch, and expects exactly what qgx_encode writes (the stream is
-integer work: bit for bit).  The file sorts last on purpose: a run that stops at the first failure has
+first call's leftovers in the shared scratch, and expects exactly what qgx_encode writes -- and what the
+oracle's encoder writes -- (the stream is integer work: bit for bit).  The file sorts last on purpose: a run that stops at the first failure has
 then already run every other test."""
 import numpy as np
 import pytest
 import torch
 
 import qgx_inputs as gen
+from oracle import qgx_oracle as o
 
 pytestmark = pytest.mark.gpu
 
@@ -35,6 +36,14 @@ def _case(qgx, ctx, K, d, bucket, nlev, sub, seed):
     assert torch.equal(bbits, want[1])
     assert torch.equal(total, want[2])
     assert torch.equal(stream, want[0])
+    # and against the oracle's encoder: lengths, totals and the used words of every worker's stream
+    st_ref, bb_ref, tot_ref = o.encode(norms.cpu().numpy(), sym.cpu().numpy(), bucket, o.codebook_from(cb.lengths(), cb.codes(), subblock=sub))
+    assert np.array_equal(bbits.cpu().numpy().view(np.uint32), bb_ref)
+    assert np.array_equal(total.cpu().numpy().astype(np.uint64), tot_ref)
+    used = ((bb_ref.astype(np.int64) + 31) // 32).sum(axis=1)
+    got = stream.cpu().numpy().view(np.uint32)
+    for k in range(K):
+        assert np.array_equal(got[k, :used[k]], st_ref[k, :used[k]])
     return norms, sym, cb
 
 
