@@ -424,6 +424,57 @@ int qgxo_codebook_huffman(const double* p, int nlev, int subblock, qgxo_codebook
   return OK;
 }
 
+// ------------------------------- choice of the code (App. J) -----------------------
+// App. J names two families of codes: Huffman's when the frequencies of the levels are known or can be estimated,
+// Elias' recursive code when they are not.  What decides between candidate codes here is what an exchange would
+// have cost under each: counts[j] = how many coordinates of the last exchange were sent as level j; a code costs
+// sum_j counts[j] * (len_j + [j != 0]) bits on them (codeword, plus the sign bit of a nonzero level; the bucket
+// headers are the same under every code).
+int qgxo_level_counts(const uint8_t* sym, int K, uint64_t d, int nlev, uint64_t* counts) {
+  if (K < 1 || nlev < 2 || nlev > kMaxLevels) return INVALID_ARG;
+  for (int j = 0; j < kMaxLevels; ++j) counts[j] = 0;
+  for (uint64_t i = 0; i < (uint64_t)K * d; ++i) {
+    const int idx = sym[i] & 31;
+    if (idx >= nlev) return CORRUPT;
+    counts[idx] += 1;
+  }
+  return OK;
+}
+
+uint64_t qgxo_code_bits(const uint64_t* counts, const qgxo_codebook* cb) {
+  uint64_t bits = 0;
+  for (int j = 0; j < cb->nlev; ++j) bits += counts[j] * (uint64_t)(cb->len[j] + (j != 0 ? 1 : 0));
+  return bits;
+}
+
+// Candidates, in this order: 0 the code in use; 1 a Huffman code built from the counts themselves (only if
+// allow_rebuild); 2 Elias' recursive code; 3 the fixed-length code.  bits[c] receives each candidate's cost
+// (~0 for a candidate that is not allowed); the cheapest wins, the earlier candidate on ties; *chosen receives
+// its codebook.  Returns the winner's number, or a negative status.
+int qgxo_choose_code(const uint64_t* counts, int nlev, const qgxo_codebook* current, int allow_rebuild, uint64_t* bits,
+                     qgxo_codebook* chosen) {
+  if (nlev < 2 || nlev > kMaxLevels || current->nlev != nlev) return -INVALID_ARG;
+  qgxo_codebook cand[4];
+  cand[0] = *current;
+  uint64_t total = 0;
+  for (int j = 0; j < nlev; ++j) total += counts[j];
+  bool have[4] = {true, allow_rebuild != 0 && total > 0, true, true};
+  if (have[1]) {
+    std::vector<double> p(nlev);
+    for (int j = 0; j < nlev; ++j) p[j] = (double)counts[j] / (double)total;
+    if (qgxo_codebook_huffman(p.data(), nlev, current->subblock, &cand[1]) != OK) have[1] = false;
+  }
+  if (qgxo_codebook_elias(nlev, current->subblock, &cand[2]) != OK) have[2] = false;
+  if (qgxo_codebook_fixed(nlev, current->subblock, &cand[3]) != OK) have[3] = false;
+  int best = 0;
+  for (int c = 0; c < 4; ++c) {
+    bits[c] = have[c] ? qgxo_code_bits(counts, &cand[c]) : ~(uint64_t)0;
+    if (have[c] && bits[c] < bits[best]) best = c;
+  }
+  *chosen = cand[best];
+  return best;
+}
+
 // ------------------------------- stream geometry -----------------------------------
 static inline int eff_subblock(int bucket, int subblock) { return (subblock <= 0 || subblock >= bucket) ? bucket : subblock; }
 

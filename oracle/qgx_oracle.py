@@ -204,6 +204,32 @@ def codebook_huffman(p, subblock=0):
     return cb
 
 
+def level_counts(sym, nlev):
+    """How many coordinates carry each level index (32 counters)."""
+    sym = np.ascontiguousarray(sym, dtype=np.uint8)
+    K, d = sym.shape
+    counts = np.zeros(32, dtype=np.uint64)
+    _chk(lib().qgxo_level_counts(_p(sym), K, C.c_uint64(d), nlev, _p(counts)), "level_counts")
+    return counts
+
+
+def code_bits(counts, cb):
+    lib().qgxo_code_bits.restype = C.c_uint64
+    counts = np.ascontiguousarray(counts, dtype=np.uint64)
+    return int(lib().qgxo_code_bits(_p(counts), C.byref(cb)))
+
+
+def choose_code(counts, cb, allow_rebuild=True):
+    """(winner 0..3, bits of the four candidates, the winner's codebook): current, Huffman from the counts, Elias, fixed."""
+    counts = np.ascontiguousarray(counts, dtype=np.uint64)
+    bits = np.zeros(4, dtype=np.uint64)
+    out = Codebook()
+    r = lib().qgxo_choose_code(_p(counts), cb.nlev, C.byref(cb), int(allow_rebuild), _p(bits), C.byref(out))
+    if r < 0:
+        raise OracleError(-r, "choose_code")
+    return r, bits, out
+
+
 def codebook_from(lengths, codes, subblock=0):
     """A hand-made prefix code (tests)."""
     cb = Codebook()

@@ -221,3 +221,38 @@ def test_corrupt_and_short_streams_are_reported():
     with pytest.raises(o.OracleError) as e:
         o.decode(stream, huge, d, bucket, cb)
     assert e.value.status == o.CORRUPT
+
+
+def test_choice_of_code_by_measured_bits():
+    """App. J: Huffman when the level frequencies are known or estimated, Elias' recursive code when they are not.
+    The cost of a code on an exchange's level counts is pinned to the encoder itself (bits of the streams minus
+    the bucket headers), the choice to cases whose winner is known beforehand."""
+    rng = np.random.default_rng(21)
+    K, d, bucket, nlev, sub = 3, 5 * 256 + 77, 256, 17, 64
+    # small levels frequent, as after quantizing a dual vector
+    p_true = np.array([2.0 ** -(j + 1) for j in range(nlev)]); p_true /= p_true.sum()
+    idx = rng.choice(nlev, size=(K, d), p=p_true).astype(np.uint8)
+    sym = idx | ((rng.integers(0, 2, size=(K, d)).astype(np.uint8) << 7) * (idx != 0))
+    norms = rng.uniform(0.5, 2.0, size=(K, o.nbuckets(d, bucket))).astype(np.float32)
+    counts = o.level_counts(sym, nlev)
+    assert counts.sum() == K * d and np.array_equal(counts[:nlev], np.bincount(idx.ravel(), minlength=nlev).astype(np.uint64))
+    nsub = sum(-(-min(bucket, d - b * bucket) // sub) for b in range(o.nbuckets(d, bucket)))
+    for cb in (o.codebook_fixed(nlev, sub), o.codebook_elias(nlev, sub), o.codebook_huffman(p_true, sub)):
+        _, bb, _ = o.encode(norms, sym, bucket, cb)
+        payload = int(bb.astype(np.int64).sum()) - K * (32 * o.nbuckets(d, bucket) + 16 * nsub)
+        assert o.code_bits(counts, cb) == payload                     # the cost formula is what the encoder spends
+    # a Huffman code fitted to frequencies that no longer hold (large levels frequent) loses to Elias' code ...
+    stale = o.codebook_huffman(p_true[::-1].copy(), sub)
+    win, bits, chosen = o.choose_code(counts, stale, allow_rebuild=False)
+    assert win == 2 and bits[2] < bits[0] and bits[2] < bits[3]
+    assert chosen.lengths() == o.codebook_elias(nlev, sub).lengths() and chosen.subblock == sub
+    # ... and to a Huffman code built from the counts themselves, which no prefix code beats on those counts
+    win, bits, chosen = o.choose_code(counts, stale, allow_rebuild=True)
+    assert win == 1 and bits[1] <= min(bits[0], bits[2], bits[3])
+    # a current code that is already the best stays (ties go to the earlier candidate)
+    win, bits2, _ = o.choose_code(counts, chosen, allow_rebuild=True)
+    assert win == 0 and bits2[0] == bits[1]
+    # uniform levels: nothing beats the fixed-length code by more than Huffman's rounding, and Elias is worst
+    flat = np.zeros(32, dtype=np.uint64); flat[:16] = 1000
+    win, bits, _ = o.choose_code(flat, o.codebook_elias(16, 0), allow_rebuild=False)
+    assert win == 3 and bits[3] == 16 * 1000 * 4 + 15 * 1000
