@@ -266,6 +266,30 @@ qgx_status qgx_set_encode_path(qgx_ctx *ctx, int mode);
 qgx_status qgx_exchange_streams(qgx_ctx *ctx, int slot, const uint32_t **stream, size_t *cap_words,
                                 const uint32_t **bucket_bits, const uint64_t **total_bits);
 
+/* ---- choice of the code by measured bits (App. J) -------------------------------------------- */
+
+/* App. J gives two kinds of prefix code: Huffman's when the frequencies of the levels are known or can be
+ * estimated, Elias' recursive code when they are not.  Between refits the frequencies drift, so the library can
+ * measure instead of assuming: counts[j] = coordinates of an exchange that were sent as level j, and a code costs
+ * sum_j counts[j] * (len[j] + [j != 0]) bits on them (the bucket headers cost the same under every code).
+ *
+ * qgx_set_keep_symbols: qgx_exchange keeps its decoded symbols in the workspace too (one byte per coordinate
+ * and worker), as the iteration calls always do for their last exchange but one.
+ * qgx_level_counts: counts [dev] uint64[32] of the exchange whose symbols the context keeps (asynchronous);
+ * QGX_ERR_INVALID_ARG if it keeps none.
+ * qgx_code_bits: the cost of a code on counts [host].
+ * qgx_choose_code_host: candidates 0 the code in *cb, 1 a Huffman code built from the counts (only if
+ * allow_rebuild), 2 Elias' recursive code, 3 the fixed-length code; bits [host] uint64[4] receives their costs
+ * (all ones for a candidate that is not allowed), *cb the cheapest (the earlier one on ties), *winner its number.
+ * qgx_choose_code: qgx_level_counts into counts [dev] uint64[32], then qgx_choose_code_host on cfg->cb, for
+ * the exchanges that follow; synchronizes the stream.  cfg->code_type (what a refit builds) is left as it is. */
+qgx_status qgx_set_keep_symbols(qgx_ctx *ctx, int on);
+qgx_status qgx_level_counts(qgx_ctx *ctx, uint64_t *counts);
+qgx_status qgx_code_bits(const uint64_t *counts, const qgx_codebook *cb, uint64_t *bits);
+qgx_status qgx_choose_code_host(const uint64_t *counts, qgx_codebook *cb, int allow_rebuild, uint64_t *bits, int *winner);
+qgx_status qgx_choose_code(qgx_ctx *ctx, qgx_quant_cfg *cfg /*[host] in/out*/, int allow_rebuild, uint64_t *counts,
+                           uint64_t *bits, int *winner);
+
 /* ---- level adaptation (Sec. 3.3; Algorithm 1, "t in U") ------------------------------------- */
 
 /* Sufficient statistics and refit in one call: hist [dev] double[nbins] receives the histogram of

@@ -28,7 +28,8 @@ EXPORTS = [
     "qgx_build_codebook_huffman", "qgx_fit_levels", "qgx_symbol_pmf",
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
-    "qgx_set_decode_split", "qgx_set_encode_path", "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
+    "qgx_set_decode_split", "qgx_set_encode_path", "qgx_set_keep_symbols", "qgx_level_counts", "qgx_code_bits",
+    "qgx_choose_code_host", "qgx_choose_code", "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
     "qgx_encode_noalloc", "qgx_exchange_segments",
 ]
 QGX_KERNEL_ENCODE, QGX_KERNEL_DECODE, QGX_KERNEL_HISTOGRAM, QGX_KERNEL_OPERATOR, QGX_KERNEL_FINISH = range(5)
@@ -350,6 +351,42 @@ def qgx_exchange_streams(ctx, slot, K, nb):
     _chk(lib().qgx_exchange_streams(ctx.h, slot, C.byref(sp), C.byref(cap), C.byref(bp), C.byref(tp)),
          "qgx_exchange_streams")
     return sp.value, int(cap.value), bp.value, tp.value
+
+
+# ---------------------------------------------------------------- choice of the code
+def qgx_set_keep_symbols(ctx, on):
+    _chk(lib().qgx_set_keep_symbols(ctx.h, int(bool(on))), "qgx_set_keep_symbols")
+
+
+def qgx_level_counts(ctx, counts=None):
+    if counts is None:
+        counts = torch.empty((32,), dtype=torch.int64, device="cuda:%d" % ctx.device)
+    _chk(lib().qgx_level_counts(ctx.h, _ptr(counts)), "qgx_level_counts")
+    return counts
+
+
+def qgx_code_bits(counts, cb):
+    arr = (C.c_uint64 * 32)(*[int(x) for x in counts])
+    bits = C.c_uint64(0)
+    _chk(lib().qgx_code_bits(arr, C.byref(cb), C.byref(bits)), "qgx_code_bits")
+    return int(bits.value)
+
+
+def qgx_choose_code_host(counts, cb, allow_rebuild=True):
+    """(winner, [bits of the four candidates]); cb is replaced by the winner."""
+    arr = (C.c_uint64 * 32)(*[int(x) for x in counts])
+    bits, win = (C.c_uint64 * 4)(), C.c_int(0)
+    _chk(lib().qgx_choose_code_host(arr, C.byref(cb), int(allow_rebuild), bits, C.byref(win)), "qgx_choose_code_host")
+    return win.value, [int(b) for b in bits]
+
+
+def qgx_choose_code(ctx, cfg, allow_rebuild=True, counts=None):
+    """(winner, [bits of the four candidates], counts tensor); cfg.cb is replaced by the winner."""
+    if counts is None:
+        counts = torch.empty((32,), dtype=torch.int64, device="cuda:%d" % ctx.device)
+    bits, win = (C.c_uint64 * 4)(), C.c_int(0)
+    _chk(lib().qgx_choose_code(ctx.h, C.byref(cfg), int(allow_rebuild), _ptr(counts), bits, C.byref(win)), "qgx_choose_code")
+    return win.value, [int(b) for b in bits], counts
 
 
 # ---------------------------------------------------------------- level adaptation

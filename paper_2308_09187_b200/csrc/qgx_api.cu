@@ -427,6 +427,54 @@ struct BinnedCdf {
 
 }  // namespace
 
+qgx_status qgx_code_bits(const uint64_t* counts, const qgx_codebook* cb, uint64_t* bits) {
+  if (!counts || !cb || !bits || cb->nlev < 2 || cb->nlev > QGX_MAX_LEVELS) return QGX_ERR_INVALID_ARG;
+  uint64_t total = 0;
+  for (int j = 0; j < cb->nlev; ++j) total += counts[j] * (uint64_t)(cb->len[j] + (j ? 1u : 0u));   // codeword, and a sign bit unless level 0
+  *bits = total;
+  return QGX_OK;
+}
+
+qgx_status qgx_choose_code_host(const uint64_t* counts, qgx_codebook* cb, int allow_rebuild, uint64_t* bits, int* winner) {
+  if (!counts || !cb || !bits || !winner || cb->nlev < 2 || cb->nlev > QGX_MAX_LEVELS) return QGX_ERR_INVALID_ARG;
+  const int nlev = cb->nlev, sub = cb->subblock;
+  qgx_codebook cand[4];
+  bool have[4] = {true, false, false, false};
+  cand[0] = *cb;
+  uint64_t sent = 0;
+  for (int j = 0; j < nlev; ++j) sent += counts[j];
+  if (allow_rebuild && sent > 0) {                      // the code that the counts themselves call for
+    double w[QGX_MAX_LEVELS];
+    for (int j = 0; j < nlev; ++j) w[j] = (double)counts[j] / (double)sent;
+    have[1] = qgx_build_codebook_huffman(w, nlev, sub, &cand[1]) == QGX_OK;
+  }
+  have[2] = qgx_build_codebook_elias(nlev, sub, &cand[2]) == QGX_OK;
+  have[3] = qgx_build_codebook_fixed(nlev, sub, &cand[3]) == QGX_OK;
+  int best = 0;
+  for (int cnd = 0; cnd < 4; ++cnd) {
+    bits[cnd] = ~(uint64_t)0;
+    if (have[cnd]) qgx_code_bits(counts, &cand[cnd], &bits[cnd]);
+    if (have[cnd] && bits[cnd] < bits[best]) best = cnd;   // ties keep the earlier candidate
+  }
+  *cb = cand[best];
+  *winner = best;
+  return QGX_OK;
+}
+
+qgx_status qgx_choose_code(qgx_ctx* c, qgx_quant_cfg* cfg, int allow_rebuild, uint64_t* counts_dev, uint64_t* bits, int* winner) {
+  if (!c || !cfg || !counts_dev || !bits || !winner) return QGX_ERR_INVALID_ARG;
+  if (cfg->cb.nlev != cfg->nlev || c->sym_nlev != cfg->nlev) return QGX_ERR_INVALID_ARG;
+  qgx_status rc = qgx_level_counts(c, counts_dev);
+  if (rc != QGX_OK) return rc;
+  uint64_t host[QGX_MAX_LEVELS];
+  if (cudaMemcpyAsync(host, counts_dev, sizeof(host), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+      cudaStreamSynchronize(c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return QGX_ERR_CUDA;
+  }
+  return qgx_choose_code_host(host, &cfg->cb, allow_rebuild, bits, winner);
+}
+
 qgx_status qgx_fit_levels(const double* hist, int nbins, float* levels, int nlev, int first_fit) {
   if (hist == nullptr || levels == nullptr || nbins < 1 || nlev < 2 || nlev > QGX_MAX_LEVELS) return QGX_ERR_INVALID_ARG;
   for (int j = 0; j < nbins; ++j)

@@ -40,6 +40,8 @@ struct qgx_ctx {
   int sym_K;
   size_t sym_d;
   size_t sym_ld;                         // bytes per worker in the kept-symbol layout
+  int sym_bucket, sym_G;                 // bucket and sub-block sizes of that layout
+  int keep_symbols;                      // qgx_exchange keeps its decoded symbols too (qgx_set_keep_symbols)
   int sym_nlev;                          // the level table those symbols were quantized with
   float sym_levels[QGX_MAX_LEVELS];
   int decode_split;                      // QGX_SPLIT_AUTO / NEVER / ALWAYS: see qgx_set_decode_split

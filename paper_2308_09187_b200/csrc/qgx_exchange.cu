@@ -1015,7 +1015,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   if (sym_mode & 1) {
     sym_out = (uint8_t*)ws_get(c, WS_SYM, (size_t)K * sym_ld + 16);
     if (!sym_out) return QGX_ERR_CUDA;
-    c->sym_slot = slot; c->sym_K = K; c->sym_d = d; c->sym_ld = sym_ld;
+    c->sym_slot = slot; c->sym_K = K; c->sym_d = d; c->sym_ld = sym_ld; c->sym_bucket = bucket; c->sym_G = ct.G;
     c->sym_nlev = cfg->nlev;
     for (int j = 0; j < cfg->nlev; ++j) c->sym_levels[j] = cfg->levels[j];
   }
@@ -1245,6 +1245,31 @@ static SegChildren* seg_children(qgx_ctx* c) {
   return sc;
 }
 
+// counts[j] += coordinates of the kept symbols (layout: DecodeArgs::sym_out) that carry level j
+__global__ void __launch_bounds__(256) k_level_counts(const uint8_t* __restrict__ sym, int K, size_t d, size_t sym_ld, int bucket, int G,
+                                                      unsigned long long* counts) {
+  __shared__ unsigned int s_cnt[8][QGX_MAX_LEVELS];                  // one set per warp
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) < QGX_MAX_LEVELS) s_cnt[warp][threadIdx.x & 31] = 0u;
+  __syncwarp();
+  const size_t wpw = sym_ld / 4;                                      // words per worker
+  const size_t spb = (size_t)(bucket / G);
+  const size_t total_sub = ((d + (size_t)bucket - 1) / (size_t)bucket) * spb;
+  for (size_t w = (size_t)blockIdx.x * blockDim.x + threadIdx.x; w < (size_t)K * wpw; w += (size_t)gridDim.x * blockDim.x) {
+    const size_t at = (w % wpw) * 4;                                  // byte inside the worker's symbols
+    const size_t gs = (at / (size_t)(32 * G)) * 32 + (at % 128) / 4;  // the sub-block
+    const size_t i0 = ((at % (size_t)(32 * G)) / 128) * 4;            // first of the word's four coordinates in it
+    if (gs >= total_sub) continue;
+    const size_t e0 = (gs / spb) * (size_t)bucket + (gs % spb) * (size_t)G + i0;
+    const uint32_t four = *reinterpret_cast<const uint32_t*>(sym + w * 4);
+    for (int cc = 0; cc < 4; ++cc)
+      if (e0 + cc < d && e0 + cc < (gs / spb + 1) * (size_t)bucket) atomicAdd(&s_cnt[warp][(four >> (8 * cc)) & 31u], 1u);
+  }
+  __syncwarp();
+  const unsigned int mine = (threadIdx.x & 31) < QGX_MAX_LEVELS ? s_cnt[warp][threadIdx.x & 31] : 0u;
+  if (mine) atomicAdd(counts + (threadIdx.x & 31), (unsigned long long)mine);
+}
+
 // acc[i] += x[i]; several streams may add into the same totals
 __global__ void k_add_u64_atomic(unsigned long long* acc, const unsigned long long* x, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -1273,7 +1298,7 @@ qgx_status qgx_exchange(qgx_ctx* c, const float* v, int K, size_t d, const qgx_q
                         int slot, float* mean_out, uint64_t* total_bits) {
   if (!v) return QGX_ERR_INVALID_ARG;
   DualSource src{v, nullptr, 0, 0};
-  return exchange_impl(c, src, K, d, cfg, exchange_id, slot, mean_out, total_bits, nullptr, 0, nullptr, 0);
+  return exchange_impl(c, src, K, d, cfg, exchange_id, slot, mean_out, total_bits, nullptr, (c && c->keep_symbols) ? 1 : 0, nullptr, 0);
 }
 
 qgx_status qgx_exchange_segments(qgx_ctx* c, const float* v, int K, size_t d, const qgx_segment* segs, int nseg,
@@ -1323,6 +1348,24 @@ qgx_status qgx_exchange_segments(qgx_ctx* c, const float* v, int K, size_t d, co
         rc = rc == QGX_OK ? QGX_ERR_CUDA : rc;
   }
   if (rc != QGX_OK) return rc;
+  return cuda_status(cudaGetLastError());
+}
+
+qgx_status qgx_set_keep_symbols(qgx_ctx* c, int on) {
+  if (!c) return QGX_ERR_INVALID_ARG;
+  c->keep_symbols = on ? 1 : 0;
+  return QGX_OK;
+}
+
+qgx_status qgx_level_counts(qgx_ctx* c, uint64_t* counts) {
+  if (!c || !counts || c->sym_slot < 0 || !c->ws[WS_SYM] || c->sym_G <= 0) return QGX_ERR_INVALID_ARG;
+  if (cudaSetDevice(c->device) != cudaSuccess) return QGX_ERR_CUDA;
+  if (cudaMemsetAsync(counts, 0, sizeof(uint64_t) * QGX_MAX_LEVELS, c->stream) != cudaSuccess) return QGX_ERR_CUDA;
+  const size_t words = (size_t)c->sym_K * (c->sym_ld / 4);
+  const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>((words + 255) / 256, (size_t)c->num_sms * 8));
+  k_level_counts<<<grid, 256, 0, c->stream>>>((const uint8_t*)c->ws[WS_SYM], c->sym_K, c->sym_d, c->sym_ld, c->sym_bucket, c->sym_G,
+                                               reinterpret_cast<unsigned long long*>(counts));
+  count_launch(c);
   return cuda_status(cudaGetLastError());
 }
 

@@ -208,3 +208,41 @@ def test_elias_recursive_code(q, K, d, bucket, nlev, sub):
     lev_ref, _ = o.refit(vh, bucket, 1024, lev.copy(), cbo, True, o.CODE_ELIAS)
     assert np.max(np.abs(np.array(cfg.level_list(), dtype=np.float32) - lev_ref)) <= 1e-6
     assert cfg.cb.codes() == cbo.codes() and cfg.cb.lengths() == cbo.lengths() and cfg.cb.subblock == sub
+
+
+def test_choice_of_code_by_measured_bits(q):
+    """App. J: the level counts of an exchange decide the code of the next ones.  Counts, costs and winner agree
+    with the oracle, and the next exchange spends exactly the predicted bits."""
+    qgx, ctx = q
+    K, d, bucket, nlev, sub = 4, 6 * 4096 + 1000, 4096, 17, 64
+    v = gen.gaussian_mixture((K, d), seed=31, device="cuda")
+    vh = v.cpu().numpy()
+    lev = np.r_[0.0, np.geomspace(2e-3, 0.2, nlev - 2), 1.0].astype(np.float32)
+    # a code fitted to frequencies that do not hold: the large levels frequent
+    stale_p = np.array([2.0 ** -(nlev - j) for j in range(nlev)])
+    cb = qgx.qgx_build_codebook_huffman(list(stale_p / stale_p.sum()), sub)
+    cbo = o.codebook_from(cb.lengths(), cb.codes(), subblock=sub)
+    cfg = qgx.make_quant_cfg(lev, bucket, cb, 5)
+    qgx.qgx_set_keep_symbols(ctx, True)
+    try:
+        _, total0 = qgx.qgx_exchange(ctx, v, cfg, 6, slot=0)
+        counts = qgx.qgx_level_counts(ctx)
+        qgx.qgx_sync_status(ctx)
+        sym_ref = o.quantize(vh, bucket, lev, o.bucket_norms(vh, bucket), 5, 6)
+        counts_ref = o.level_counts(sym_ref, nlev)
+        got = counts.cpu().numpy().astype(np.uint64)
+        flips = int(np.abs(got.astype(np.int64) - counts_ref.astype(np.int64)).sum())
+        assert got.sum() == K * d and flips <= 2 * max(1, int(1e-6 * K * d))
+        nsub = sum(-(-min(bucket, d - b * bucket) // sub) for b in range(o.nbuckets(d, bucket)))
+        headers = K * (32 * o.nbuckets(d, bucket) + 16 * nsub)
+        assert int(total0.sum().item()) == headers + qgx.qgx_code_bits(got, cfg.cb)
+        for allow, want in ((False, 2), (True, 1)):          # Elias beats the stale code; a code from the counts beats both
+            cfg2 = qgx.make_quant_cfg(lev, bucket, cb, 5)
+            win, bits, _ = qgx.qgx_choose_code(ctx, cfg2, allow)
+            win_o, bits_o, _ = o.choose_code(got, cbo, allow)
+            assert win == want == win_o and bits == [int(x) for x in bits_o]
+            _, total1 = qgx.qgx_exchange(ctx, v, cfg2, 6, slot=1)
+            qgx.qgx_sync_status(ctx)
+            assert int(total1.sum().item()) == headers + bits[win] < int(total0.sum().item())
+    finally:
+        qgx.qgx_set_keep_symbols(ctx, False)

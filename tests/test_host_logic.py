@@ -90,3 +90,27 @@ def test_level_fit_and_symbol_weights_match_oracle(qgx):
             assert np.max(np.abs(p - o.symbol_pmf(hist, ref))) < 1e-12
     # an empty histogram keeps the table
     assert qgx.qgx_fit_levels([0.0] * 64, levels=[0.0, 0.25, 1.0]) == [0.0, 0.25, 1.0]
+
+
+def test_choice_of_code_matches_oracle(qgx):
+    """Cost of a code on level counts and the choice between the four candidates (App. J), host side."""
+    rng = np.random.default_rng(8)
+    for nlev in (3, 9, 17, 32):
+        for trial in range(6):
+            counts = np.zeros(32, dtype=np.uint64)
+            counts[:nlev] = rng.integers(0, 10 ** rng.integers(1, 7), size=nlev)
+            if trial == 0:
+                counts[:] = 0
+            cur_o = [o.codebook_fixed(nlev, 64), o.codebook_elias(nlev, 64), o.codebook_huffman(rng.dirichlet(np.ones(nlev)), 64)][trial % 3]
+            cur = qgx.qgx_codebook()
+            cur.nlev, cur.maxlen, cur.subblock = cur_o.nlev, cur_o.maxlen, cur_o.subblock
+            for j in range(nlev):
+                cur.len[j], cur.code[j] = cur_o.len[j], cur_o.code[j]
+            assert qgx.qgx_code_bits(counts, cur) == o.code_bits(counts, cur_o)
+            for allow in (False, True):
+                cb = qgx.qgx_codebook.from_buffer_copy(cur)
+                win, bits = qgx.qgx_choose_code_host(counts, cb, allow)
+                win_o, bits_o, cb_o = o.choose_code(counts, cur_o, allow)
+                # the two Huffman builders may break ties differently: equal costs, not necessarily equal codes
+                assert bits == [int(b) for b in bits_o] and win == win_o
+                assert qgx.qgx_code_bits(counts, cb) == min(bits) and cb.subblock == 64
