@@ -261,6 +261,20 @@ qgx_status qgx_set_decode_split(qgx_ctx *ctx, int mode);
  * faster on B200: the first. */
 enum { QGX_ENCODE_AUTO = 0, QGX_ENCODE_REGISTERS = 1, QGX_ENCODE_STAGED = 2 };
 qgx_status qgx_set_encode_path(qgx_ctx *ctx, int mode);
+/* The receiving side alone (Algorithm 1: decode, aggregate): decodes the streams that the last qgx_exchange with
+ * the same K, d and bucket left in `slot` -- as they are now, so also after the caller has changed them -- and writes
+ * their mean to mean_out [dev] float[d].  cfg [host] must carry the level table and code they were made with.
+ * Device-side error: QGX_ERR_CORRUPT for streams that no encoder could have produced (every read stays inside
+ * the slot's buffers). */
+qgx_status qgx_exchange_decode(qgx_ctx *ctx, int K, size_t d, const qgx_quant_cfg *cfg, int slot, float *mean_out);
+/* How many times a device-side wait (one bucket waiting for the word count of an earlier bucket of its worker)
+ * polls before it gives up with QGX_ERR_TIMEOUT; the default, 2^22, is seconds.  No counterpart in the paper. */
+qgx_status qgx_set_wait_limit(qgx_ctx *ctx, int polls);
+/* Diagnostic (no counterpart in the paper): the next fused exchange on this context leaves the first `buckets`
+ * buckets of every worker unencoded, so that the buckets after them wait for word counts that never come.  With a
+ * small wait limit this shows the bounded wait at work: the waiting buckets give up, QGX_ERR_TIMEOUT is latched,
+ * nothing is written for them, the kernel ends, and the context stays usable. */
+qgx_status qgx_debug_skip_buckets(qgx_ctx *ctx, size_t buckets);
 /* Where the last qgx_exchange on `slot` left its streams: all [dev], valid until the next call
  * that uses the slot.  Any output pointer may be NULL. */
 qgx_status qgx_exchange_streams(qgx_ctx *ctx, int slot, const uint32_t **stream, size_t *cap_words,

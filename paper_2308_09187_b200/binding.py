@@ -29,7 +29,7 @@ EXPORTS = [
     "qgx_quantize", "qgx_encode", "qgx_decode", "qgx_average",
     "qgx_exchange", "qgx_exchange_streams", "qgx_update_levels", "qgx_histogram",
     "qgx_set_decode_split", "qgx_set_encode_path", "qgx_set_keep_symbols", "qgx_level_counts", "qgx_code_bits",
-    "qgx_choose_code_host", "qgx_choose_code", "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
+    "qgx_choose_code_host", "qgx_choose_code", "qgx_exchange_decode", "qgx_set_wait_limit", "qgx_debug_skip_buckets", "qgx_eg_init", "qgx_eg_step", "qgx_eg_step_two_tables", "qgx_family_step", "qgx_apply_operator", "qgx_timing_enable", "qgx_timing_read",
     "qgx_encode_noalloc", "qgx_exchange_segments",
 ]
 QGX_KERNEL_ENCODE, QGX_KERNEL_DECODE, QGX_KERNEL_HISTOGRAM, QGX_KERNEL_OPERATOR, QGX_KERNEL_FINISH = range(5)
@@ -307,6 +307,21 @@ def qgx_exchange(ctx, v, cfg, exchange_id, slot=0, mean_out=None, total_bits=Non
     _chk(lib().qgx_exchange(ctx.h, _ptr(v), K, C.c_size_t(d), C.byref(cfg), C.c_uint32(exchange_id), slot,
                             _ptr(mean_out), _ptr(total_bits)), "qgx_exchange")
     return mean_out, total_bits
+
+
+def qgx_exchange_decode(ctx, K, d, cfg, slot=0, mean_out=None):
+    if mean_out is None:
+        mean_out = torch.empty((d,), dtype=torch.float32, device="cuda:%d" % ctx.device)
+    _chk(lib().qgx_exchange_decode(ctx.h, K, C.c_size_t(d), C.byref(cfg), slot, _ptr(mean_out)), "qgx_exchange_decode")
+    return mean_out
+
+
+def qgx_set_wait_limit(ctx, polls):
+    _chk(lib().qgx_set_wait_limit(ctx.h, int(polls)), "qgx_set_wait_limit")
+
+
+def qgx_debug_skip_buckets(ctx, buckets):
+    _chk(lib().qgx_debug_skip_buckets(ctx.h, C.c_size_t(buckets)), "qgx_debug_skip_buckets")
 
 
 class qgx_segment(C.Structure):

@@ -164,6 +164,7 @@ qgx_status qgx_create(qgx_ctx** out, int device, void* cuda_stream) {
   std::memset(c, 0, sizeof(*c));
   c->device = device;
   c->sym_slot = -1;
+  c->wait_limit = kSpinLimit;
   c->num_sms = 1;
   if (cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->num_sms < 1) { cudaGetLastError(); c->num_sms = 1; }
   c->stream = (cudaStream_t)cuda_stream;

@@ -42,6 +42,9 @@ struct qgx_ctx {
   size_t sym_ld;                         // bytes per worker in the kept-symbol layout
   int sym_bucket, sym_G;                 // bucket and sub-block sizes of that layout
   int keep_symbols;                      // qgx_exchange keeps its decoded symbols too (qgx_set_keep_symbols)
+  int wait_limit;                        // polls of a device-side wait before it gives up (qgx_set_wait_limit)
+  size_t skip_buckets;                   // diagnostic: the next exchange leaves these first buckets unencoded
+  int decode_only;                       // set around the decode-only entry point
   int sym_nlev;                          // the level table those symbols were quantized with
   float sym_levels[QGX_MAX_LEVELS];
   int decode_split;                      // QGX_SPLIT_AUTO / NEVER / ALWAYS: see qgx_set_decode_split

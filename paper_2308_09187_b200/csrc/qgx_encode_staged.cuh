@@ -381,7 +381,7 @@ k_encode_staged(const __grid_constant__ EncodeArgs a, const __grid_constant__ Le
     unsigned int next_group = 0;
     if (last_of_bucket) {                                             // where the bucket goes in its worker's stream
       bool timed_out = false;
-      const unsigned long long excl = lookback_prefix(row, (long long)b, lane, &timed_out);
+      const unsigned long long excl = lookback_prefix(row, (long long)b, lane, a.spin_limit, &timed_out);
       if (lane == 0) {
         st_status(row + b, kStPrefix | (excl + (unsigned long long)nwords));
         int skip = 0;

@@ -31,7 +31,7 @@ __device__ __forceinline__ void st_status(unsigned long long* p, unsigned long l
 // bucket waits only for buckets with smaller t, and the unfinished bucket with the smallest t waits for nothing,
 // so the wait below always ends; it is bounded all the same, and *timed_out reports a wait that ran out.
 __device__ __forceinline__ unsigned long long lookback_prefix(unsigned long long* row /* status of worker k */, long long b,
-                                                              int lane, bool* timed_out) {
+                                                              int lane, int spin_limit, bool* timed_out) {
   unsigned long long prefix = 0;
   long long hi = b - 1;                                 // nearest predecessor not yet accounted for
   int spins = 0;
@@ -46,7 +46,7 @@ __device__ __forceinline__ unsigned long long lookback_prefix(unsigned long long
     const int first_pref = pref ? __ffs(pref) - 1 : 32;
     const int first_empty = empty ? __ffs(empty) - 1 : 32;
     if (first_empty < first_pref) {                     // a predecessor has not published yet
-      if (++spins > kSpinLimit) fail = true;
+      if (++spins > spin_limit) fail = true;
       __nanosleep(64);
       continue;
     }
@@ -82,6 +82,7 @@ struct EncodeArgs {
   DevStatus* st;
   size_t nb_whole;              // buckets [0, nb_whole) of every worker belong to k_encode_staged ...
   size_t b_first;               // ... and buckets [b_first, nb) to k_exchange_encode
+  int spin_limit;               // polls of a wait for another bucket's count before it gives up
 };
 
 // Norm of the bucket held by the CTA, one barrier: per-warp partials go to shared memory and every
@@ -385,7 +386,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
     for (int j = 0; j < P; ++j) put_bits2(s_img, base + qoff[j], qbits[2 * j], qn[j] & 0xffu, qbits[2 * j + 1], qn[j] >> 8);
     if (warp == 0) {
       bool timed_out = false;
-      const unsigned long long excl = lookback_prefix(row, (long long)b, lane, &timed_out);
+      const unsigned long long excl = lookback_prefix(row, (long long)b, lane, a.spin_limit, &timed_out);
       if (lane == 0) {
         st_status(row + b, kStPrefix | (excl + (unsigned long long)nwords));
         int skip = 0;
@@ -845,6 +846,8 @@ static void allow_max_dynamic_smem(Kernel kernel, int device) {
   struct Seen { const void* fn; int device; };
   static Seen seen[256];                                // all template instances of a kernel share this function
   static int nseen = 0;
+  static std::mutex guard;                              // contexts may be driven from different host threads
+  std::lock_guard<std::mutex> lock(guard);
   const void* fn = reinterpret_cast<const void*>(kernel);
   for (int i = 0; i < nseen; ++i)
     if (seen[i].fn == fn && seen[i].device == device) return;
@@ -991,7 +994,8 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   c->slot_K[slot] = K;
   c->slot_nb[slot] = nb;
 
-  if (cudaMemsetAsync(tot, 0, sizeof(uint64_t) * ((size_t)K + 2 + (size_t)K * nb), c->stream) != cudaSuccess) return QGX_ERR_CUDA;
+  const bool do_encode = !c->decode_only;               // the decode-only entry point works on the streams that are there
+  if (do_encode && cudaMemsetAsync(tot, 0, sizeof(uint64_t) * ((size_t)K + 2 + (size_t)K * nb), c->stream) != cudaSuccess) return QGX_ERR_CUDA;
 
   EncodeArgs ea;
   ea.src = src; ea.d = d; ea.bucket = bucket; ea.K = K; ea.nb = nb; ea.norm_type = cfg->norm_type; ea.xid = xid; ea.quad_base = coord_base / kQuad;
@@ -1051,7 +1055,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   // Whole buckets of a multiple of 1024 coordinates that divides 16384 go through the staged kernel; what is left
   // (a short last bucket, other bucket sizes, unaligned vectors) through the bucket-in-registers kernel.
   bool staged_ok = ea.vec_ok && bucket % kWarpCoords == 0 && kStageCoords % bucket == 0 && coord_base % 8 == 0 &&
-                   c->encode_path == QGX_ENCODE_STAGED && d / (size_t)bucket > 0;
+                   c->encode_path == QGX_ENCODE_STAGED && d / (size_t)bucket > 0 && c->skip_buckets == 0;
   CUtensorMap tmap;
   std::memset(&tmap, 0, sizeof(tmap));
   if (staged_ok) {
@@ -1064,8 +1068,10 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
                 make_rows_map(base, floats / kLaneCoords, (unsigned)std::min(256, bucket / kLaneCoords), &tmap);
   }
   ea.nb_whole = staged_ok ? d / (size_t)bucket : 0;
-  ea.b_first = ea.nb_whole;
-  {
+  ea.b_first = staged_ok ? ea.nb_whole : std::min(c->skip_buckets, nb);
+  c->skip_buckets = 0;
+  ea.spin_limit = c->wait_limit;
+  if (do_encode) {
     ScopedKernelTimer timer(c, QGX_KERNEL_ENCODE);
     if (ea.nb_whole > 0) {
       const size_t smem_st = sizeof(float) * kStageCoords * kStageBuffers;
@@ -1228,6 +1234,7 @@ static SegChildren* seg_children(qgx_ctx* c) {
     std::memset(h, 0, sizeof(*h));
     h->device = c->device;
     h->sym_slot = -1;
+    h->wait_limit = c->wait_limit;
     h->decode_split = c->decode_split;
     h->encode_path = c->encode_path;
     h->num_sms = c->num_sms;
@@ -1349,6 +1356,29 @@ qgx_status qgx_exchange_segments(qgx_ctx* c, const float* v, int K, size_t d, co
   }
   if (rc != QGX_OK) return rc;
   return cuda_status(cudaGetLastError());
+}
+
+qgx_status qgx_exchange_decode(qgx_ctx* c, int K, size_t d, const qgx_quant_cfg* cfg, int slot, float* mean_out) {
+  if (!c || slot < 0 || slot > 1 || !cfg || c->slot_K[slot] != K || K < 1 || d < 1 || cfg->bucket < kQuad ||
+      c->slot_nb[slot] != (d + (size_t)cfg->bucket - 1) / (size_t)cfg->bucket)
+    return QGX_ERR_INVALID_ARG;
+  DualSource none{nullptr, nullptr, 0, 0};
+  c->decode_only = 1;
+  const qgx_status rc = exchange_impl(c, none, K, d, cfg, 0, slot, mean_out, nullptr, nullptr, 0, nullptr, 0);
+  c->decode_only = 0;
+  return rc;
+}
+
+qgx_status qgx_set_wait_limit(qgx_ctx* c, int polls) {
+  if (!c || polls < 1) return QGX_ERR_INVALID_ARG;
+  c->wait_limit = polls;
+  return QGX_OK;
+}
+
+qgx_status qgx_debug_skip_buckets(qgx_ctx* c, size_t buckets) {
+  if (!c) return QGX_ERR_INVALID_ARG;
+  c->skip_buckets = buckets;
+  return QGX_OK;
 }
 
 qgx_status qgx_set_keep_symbols(qgx_ctx* c, int on) {

@@ -246,3 +246,62 @@ def test_choice_of_code_by_measured_bits(q):
             assert int(total1.sum().item()) == headers + bits[win] < int(total0.sum().item())
     finally:
         qgx.qgx_set_keep_symbols(ctx, False)
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable(q):
+    """A bucket waits for the word counts of its worker's earlier buckets; the wait is bounded.  With the first
+    buckets left unencoded on purpose and a small limit the waiting buckets give up: QGX_ERR_TIMEOUT comes back, the
+    kernel ends by itself, and the next exchange on the same context is exact again."""
+    qgx, ctx = q
+    K, d, bucket = 3, 12 * 1024, 1024
+    v = gen.gaussian((K, d), seed=4, device="cuda")
+    lev = np.linspace(0, 1, 9, dtype=np.float32)
+    cfg = qgx.make_quant_cfg(lev, bucket, qgx.qgx_build_codebook_fixed(9, 64), 3)
+    want, tot = qgx.qgx_exchange(ctx, v, cfg, 1, slot=0)
+    qgx.qgx_sync_status(ctx)
+    want, tot = want.clone(), tot.clone()
+    qgx.qgx_set_wait_limit(ctx, 50)
+    qgx.qgx_debug_skip_buckets(ctx, 2)
+    qgx.qgx_exchange(ctx, v, cfg, 1, slot=0)
+    assert qgx.qgx_sync_status(ctx, check=False) == qgx.QGX_ERR_TIMEOUT
+    qgx.qgx_set_wait_limit(ctx, 1 << 22)
+    again, tot2 = qgx.qgx_exchange(ctx, v, cfg, 1, slot=0)
+    qgx.qgx_sync_status(ctx)
+    assert torch.equal(again, want) and torch.equal(tot2, tot)
+
+
+def test_decode_pass_alone_and_corrupt_streams(q):
+    """The receiving side on its own reproduces the mean; streams changed behind its back are reported as corrupt
+    (or decode to something else where the change happens to be a valid stream), never read out of range."""
+    qgx, ctx = q
+    K, d, bucket, sub = 4, 9 * 2048 + 600, 2048, 64
+    v = gen.gaussian_mixture((K, d), seed=8, device="cuda")
+    lev = np.r_[0.0, np.geomspace(1e-3, 0.3, 15), 1.0].astype(np.float32)
+    p = np.array([2.0 ** -(j + 1) for j in range(17)])
+    cfg = qgx.make_quant_cfg(lev, bucket, qgx.qgx_build_codebook_huffman(list(p / p.sum()), sub), 21)
+    nb = o.nbuckets(d, bucket)
+    mean, _ = qgx.qgx_exchange(ctx, v, cfg, 2, slot=1)
+    qgx.qgx_sync_status(ctx)
+    mean = mean.clone()
+    assert torch.equal(qgx.qgx_exchange_decode(ctx, K, d, cfg, slot=1), mean)
+    qgx.qgx_sync_status(ctx)
+    stream, bbits, _ = qgx.exchange_stream_tensors(ctx, 1, K, nb)
+    keep_s, keep_b = stream.clone(), bbits.clone()
+    # 1. a sub-block length in a bucket header that disagrees with the bits that follow
+    stream[1, 1] ^= 0x0004
+    qgx.qgx_exchange_decode(ctx, K, d, cfg, slot=1)
+    assert qgx.qgx_sync_status(ctx, check=False) == qgx.QGX_ERR_CORRUPT
+    stream.copy_(keep_s)
+    # 2. a bucket length beyond anything the buffers hold
+    bbits[2, 3] = 0x7fffffff
+    qgx.qgx_exchange_decode(ctx, K, d, cfg, slot=1)
+    assert qgx.qgx_sync_status(ctx, check=False) == qgx.QGX_ERR_CORRUPT
+    bbits.copy_(keep_b)
+    # 3. random bits flipped all over the payload
+    noise = torch.randint(0, 2 ** 31 - 1, stream.shape, dtype=torch.int32, device="cuda", generator=torch.Generator("cuda").manual_seed(1))
+    stream ^= noise
+    qgx.qgx_exchange_decode(ctx, K, d, cfg, slot=1)
+    assert qgx.qgx_sync_status(ctx, check=False) == qgx.QGX_ERR_CORRUPT
+    stream.copy_(keep_s)
+    assert torch.equal(qgx.qgx_exchange_decode(ctx, K, d, cfg, slot=1), mean)
+    qgx.qgx_sync_status(ctx)
