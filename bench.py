@@ -35,10 +35,18 @@ METRIC = "Q-GenX quantize->code->decode->average GB/s (% of HBM peak); EG iterat
 WORKLOAD = "c5-scale: K=32, d=2^26, mixture noise, diagonal operator, bucket 16384, 17 adaptive levels"
 
 
-# measured DRAM traffic of k_exchange_encode per coordinate (ncu, current kernel); None once the kernel has changed
-ENCODE_DRAM_BYTES_PER_COORDINATE = 4.882
-# executed thread instructions of k_exchange_encode per coordinate (ncu, same capture); None once the kernel has changed
-ENCODE_INSTRUCTIONS_PER_COORDINATE = 60.7
+def profile_constants():
+    """DRAM bytes and executed thread instructions per coordinate of the encode kernel, as counted by ncu on the
+    small case: read from the line "bench: ..." of the committed summary, so that they change together with it.
+    (None, None) when the summary does not carry them, e.g. after the kernel changed and before a new capture."""
+    import re
+    try:
+        text = open(os.path.join(ROOT, "profiles", "exchange_kernels_K8_d16M.txt")).read()
+        m = re.search(r"^bench: dram_bytes_per_coordinate=([0-9.]+) instructions_per_coordinate=([0-9.]+)", text, re.M)
+        return (float(m.group(1)), float(m.group(2))) if m else (None, None)
+    except OSError:
+        return None, None
+
 
 def exchange_bytes(K, d, nb, stream_words):
     """Algorithmic bytes of one exchange: read V, write + read the streams and their length words, write the mean."""
@@ -205,17 +213,18 @@ def run_ours(args):
     # DRAM bytes per launch of that kernel: counted by ncu on a smaller case of the same kernel (see
     # profiles/exchange_kernels_K8_d16M.txt: 655.2 MB read + written for K * d = 2^27 coordinates) and scaled by
     # the coordinates of a launch, which the traffic is proportional to.  Set to None when the kernel changes.
+    dram_per_coord, instr_per_coord = profile_constants()
     traffic = args.traffic_bytes
-    if traffic is None and ENCODE_DRAM_BYTES_PER_COORDINATE is not None:
-        traffic = ENCODE_DRAM_BYTES_PER_COORDINATE * K * d
+    if traffic is None and dram_per_coord is not None:
+        traffic = dram_per_coord * K * d
     # The same kernel against the issue ceiling that actually binds it: executed thread instructions per second
     # (ncu's count per coordinate x coordinates per launch / the event time) over 148 SMs x 128 lanes x the SM clock
     # seen during the timed region.
     alu = None
-    if n_enc and ENCODE_INSTRUCTIONS_PER_COORDINATE is not None:
+    if n_enc and instr_per_coord is not None:
         sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
         alu_peak = 148 * 128 * sm_mhz * 1e6 / 1e12
-        alu_ach = ENCODE_INSTRUCTIONS_PER_COORDINATE * K * d / (enc_ms * 1e-3) / 1e12
+        alu_ach = instr_per_coord * K * d / (enc_ms * 1e-3) / 1e12
         alu = {"achieved": alu_ach, "peak": alu_peak, "unit": "T thread-instructions/s", "frac": alu_ach / alu_peak}
     roofline = {"bound": "hbm", "kernel": "k_exchange_encode", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None, "peak_kind": "of " + peak_kind,
@@ -336,13 +345,15 @@ def other_configs(qgx, ctx):
 
 def run_e2e(args, qgx, ctx, st, op, cfg, prob, world, bytes_step):
     """The same step through the public call with HOST inputs: the step's noise is copied from pinned host
-    memory to the device and the step's scalars (sum of squared differences, step size) are read back."""
+    memory to the device and the step's result (the new iterate, with the sum of squared differences and the step
+    size) is read back."""
     import torch
     import torch.distributed as dist
     K, d = args.workers, args.d
     host_noise = torch.empty((2, K, d), dtype=torch.float32, pin_memory=True)
     host_noise.copy_(prob.noise)
     host_out = torch.empty(2, dtype=torch.float64, pin_memory=True)
+    host_x = torch.empty((d,), dtype=torch.float32, pin_memory=True)      # the step's result: the new iterate
     dev_noise = prob.noise                       # destination of the per-step copy
     steps = max(1, min(args.steps, args.e2e_steps))
 
@@ -350,6 +361,7 @@ def run_e2e(args, qgx, ctx, st, op, cfg, prob, world, bytes_step):
         dev_noise.copy_(host_noise, non_blocking=True)
         qgx.qgx_eg_step(ctx, st, op, dev_noise[0], dev_noise[1], cfg, refit=qgx.QGX_REFIT_NONE)
         host_out.copy_(st.scalars, non_blocking=True)
+        host_x.copy_(st.X, non_blocking=True)
 
     step()
     torch.cuda.synchronize()
@@ -364,7 +376,7 @@ def run_e2e(args, qgx, ctx, st, op, cfg, prob, world, bytes_step):
     ms = max_over_ranks(e0.elapsed_time(e1), world)
     qgx.qgx_sync_status(ctx)
     return {"value": world * bytes_step * steps / (ms * 1e-3) / 1e9, "unit": "GB/s", "steps": steps,
-            "ms_per_step": ms / steps, "h2d_bytes_per_step": 2 * K * d * 4, "d2h_bytes_per_step": 16,
+            "ms_per_step": ms / steps, "h2d_bytes_per_step": 2 * K * d * 4, "d2h_bytes_per_step": 4 * d + 16,
             "eg_iterations_per_s": world * steps / (ms * 1e-3)}
 
 
@@ -375,9 +387,38 @@ def oracle_sample_problem(args, seed=1005):
     return gen.c5_diagonal(K=args.workers, d=d_s, device="cpu", seed=seed, bucket=args.bucket), d_s
 
 
+def cpu_model():
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+class pinned_to_one_core:
+    """Runs the enclosed code on one host core (where the system allows it)."""
+
+    def __enter__(self):
+        self.before = None
+        try:
+            self.before = os.sched_getaffinity(0)
+            os.sched_setaffinity(0, {min(self.before)})
+        except (AttributeError, OSError):
+            self.before = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.before is not None:
+            os.sched_setaffinity(0, self.before)
+
+
 def cpu_baseline(args, cfg, prob):
-    """The oracle, as it stands, on one host core, on a bounded sample of the same workload."""
+    """The oracle, as it stands, on a bounded sample of the same workload: pinned to one host core, and again
+    with one thread per worker (each thread runs one worker's quantize -> encode -> decode; timing only)."""
     import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
     from oracle import qgx_oracle as o
     K, bucket = args.workers, args.bucket
     d_s = args.cpu_buckets * bucket
@@ -385,15 +426,25 @@ def cpu_baseline(args, cfg, prob):
     V = (prob.noise[0, :, :d_s].cpu().numpy() + a[None, :]).astype(np.float32)
     lev = np.array(cfg.level_list(), dtype=np.float32)
     cbo = o.codebook_from(cfg.cb.lengths(), cfg.cb.codes(), subblock=cfg.cb.subblock)
-    t0 = time.perf_counter()
-    mean, total = o.exchange(V, bucket, lev, cbo, int(cfg.seed), 2)
-    dt = time.perf_counter() - t0
+    with pinned_to_one_core():
+        t0 = time.perf_counter()
+        mean, total = o.exchange(V, bucket, lev, cbo, int(cfg.seed), 2)
+        dt = time.perf_counter() - t0
     nb = d_s // bucket
     words = int(np.sum((total.astype(np.int64) + 31) // 32)) + K * nb      # upper estimate of padded words
     by = exchange_bytes(K, d_s, nb, words)
+    threads = max(1, min(K, os.cpu_count() or 1))
+    slices = [np.ascontiguousarray(V[k:k + 1]) for k in range(K)]
+    with ThreadPoolExecutor(max_workers=threads) as pool:               # the C calls release the interpreter lock
+        t0 = time.perf_counter()
+        list(pool.map(lambda vk: o.exchange(vk, bucket, lev, cbo, int(cfg.seed), 2), slices))
+        dt_threads = time.perf_counter() - t0
     return {"value": by / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
-            "sample": "one exchange of K=%d workers x %d buckets of %d coordinates (%.1f M coordinates), %.1f s"
-                      % (K, args.cpu_buckets, bucket, K * d_s / 1e6, dt)}
+            "cpu": cpu_model(), "host_cores": os.cpu_count(),
+            "threads_value": by / dt_threads / 1e9, "threads": threads,
+            "sample": "one exchange of K=%d workers x %d buckets of %d coordinates (%.1f M coordinates): %.1f s on one "
+                      "core, %.1f s with %d threads (one worker per thread)"
+                      % (K, args.cpu_buckets, bucket, K * d_s / 1e6, dt, dt_threads, threads)}
 
 
 def run_reference(args):
@@ -420,12 +471,13 @@ def run_reference(args):
         refit = 2 if t == 1 else (1 if (t - 1) % args.refit_every == 0 else 0)
         return o.eg_step(st, opo, n0, n1, bucket, lev, cbo, prob.seed, refit=refit, code_type=o.CODE_HUFFMAN, nbins=1024)
 
-    for _ in range(max(args.warmup, 1)):
-        step()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        bits = step()
-    dt = time.perf_counter() - t0
+    with pinned_to_one_core():
+        for _ in range(max(args.warmup, 1)):
+            step()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            bits = step()
+        dt = time.perf_counter() - t0
     words = bits // 32 + 2 * K * nbk                      # both exchanges, padded estimate
     by = 2 * (4 * K * d_s + 4 * d_s) + 2 * (4 * words + 2 * 4 * K * nbk)
     value = by * args.steps / dt / 1e9
@@ -437,7 +489,8 @@ def run_reference(args):
         "config": {"workload": WORKLOAD + " (bounded sample)", "K": K, "d": d_s, "bucket": bucket, "nlev": nlev,
                    "subblock": args.subblock, "code": "huffman", "refit_every": args.refit_every},
         "eg_iterations_per_s": args.steps / dt,
-        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample, "cpu": cpu_model(),
+                         "host_cores": os.cpu_count()},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
