@@ -139,8 +139,9 @@ __device__ __forceinline__ void copy_segment(const Segment seg, uint32_t next_R,
 // coordinate a multiple of 8 in the generator's counter space (the host checks).  tmap: the staged source as rows
 // of 32 floats.  Buckets are taken in the order b-major, k-minor, 16384 / bucket at a time; group g belongs to CTA
 // g mod gridDim.x, which works on its groups in increasing order (its n-th group by team n & 1 in buffer n % 3).
-// All CTAs are resident and advance at the same pace, so the buckets a bucket looks back at (the same worker's
-// earlier buckets, which lie in groups before its own) have usually been counted when it asks.  A bucket waits
+// The launch is cooperative, so all CTAs are resident whatever else runs on the device, and they advance at the
+// same pace: the buckets a bucket looks back at (the same worker's earlier buckets, which lie in groups before
+// its own) have usually been counted when it asks.  A bucket waits
 // only for buckets of smaller groups, and a group that is staged but not started waits only for its own team's
 // current group, which is smaller: the smallest unfinished group is always being worked on and waits for
 // nothing, so every wait ends.

@@ -26,10 +26,10 @@ __device__ __forceinline__ void st_status(unsigned long long* p, unsigned long l
   *reinterpret_cast<volatile unsigned long long*>(p) = v;
 }
 
-// Exclusive prefix (in words) of bucket b of one worker, by one warp.  Buckets are taken in the order b-major,
-// k-minor, bucket t by CTA t mod gridDim.x, every CTA is resident and takes its buckets in increasing order: a
-// bucket waits only for buckets with smaller t, and the unfinished bucket with the smallest t waits for nothing,
-// so the wait below always ends; it is bounded all the same, and *timed_out reports a wait that ran out.
+// Exclusive prefix (in words) of bucket b of one worker, by warp 0 of the CTA.  Buckets are handed
+// out by a ticket counter in the order b-major, k-minor, so every predecessor (k, b') with b' < b
+// belongs to a CTA that is already running or done: the wait below always ends; it is bounded all
+// the same, and *timed_out reports a wait that ran out.
 __device__ __forceinline__ unsigned long long lookback_prefix(unsigned long long* row /* status of worker k */, long long b,
                                                               int lane, int spin_limit, bool* timed_out) {
   unsigned long long prefix = 0;
@@ -79,6 +79,7 @@ struct EncodeArgs {
   unsigned long long* total_bits;   // [K], zeroed before the launch
   float* norms;                 // [K][nb] (kept for the caller; the streams carry them too)
   unsigned long long* status;   // [K][nb], zeroed before the launch
+  unsigned int* ticket;         // zeroed before the launch
   DevStatus* st;
   size_t nb_whole;              // buckets [0, nb_whole) of every worker belong to k_encode_staged ...
   size_t b_first;               // ... and buckets [b_first, nb) to k_exchange_encode
@@ -226,7 +227,7 @@ __device__ __forceinline__ uint32_t pair_entry(uint32_t pair, float z_first, flo
   return lds_table32(pair + (__float_as_uint(t) & 0x3ffcu));
 }
 
-// One persistent CTA per SM slot; bucket t of the launch is (k = t % K, b = t / K).
+// One persistent CTA per SM slot; each ticket is one bucket (k = ticket % K, b = ticket / K).
 //   loads, zero the image | barrier | norm, Philox, rounding, packing, sub-block lengths, warp scans |
 //   barrier | warp offsets, bit scatter, look-back (warp 0) | barrier | copy out
 // The bucket image is double buffered, so the copy-out of one bucket needs no barrier before the next
@@ -243,6 +244,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   __shared__ float s_lev[QGX_MAX_LEVELS];
   __shared__ double s_red[2][32];
   __shared__ uint32_t s_wtot[2][32];
+  __shared__ unsigned int s_ticket[2];
   __shared__ unsigned long long s_prefix[2];
   __shared__ int s_skip[2];
 
@@ -257,6 +259,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   fill_enc_lut(&s_lut, ct);
   fill_bin_table(s_bin, rt, true);
   if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 1.0f;
+  if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
   for (int i = threadIdx.x; i < 2 * img_words; i += blockDim.x) s_dyn[i] = 0;
   __syncthreads();
   fill_pair_lut_signed(s_pair, &s_lut);
@@ -266,14 +269,10 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   const float S = -rt.neg_qscale16 * 65536.0f, four_over_S = 4.0f / S;
   uint32_t used_words[2] = {0u, 0u};                    // words of each image that the last bucket in it dirtied
 
-  // bucket t of the launch (b-major, k-minor) belongs to CTA t mod gridDim.x, which takes its buckets in increasing
-  // order; (b, k) advance by (gridDim.x / K, gridDim.x mod K) from one bucket of a CTA to its next
-  const unsigned long long step_b = (unsigned long long)gridDim.x / (unsigned long long)a.K;
-  const unsigned int step_k = gridDim.x % (unsigned int)a.K;
-  size_t b = a.b_first + (size_t)(blockIdx.x / (unsigned int)a.K), k = (size_t)(blockIdx.x % (unsigned int)a.K);
-  unsigned long long t = blockIdx.x;
-  for (int par = 0; t < total; par ^= 1, t += gridDim.x, b += (size_t)step_b, k += step_k) {
-    if (k >= (size_t)a.K) { k -= (size_t)a.K; ++b; }
+  for (int par = 0;; par ^= 1) {
+    const unsigned long long t = s_ticket[par];
+    if (t >= total) break;
+    const size_t b = a.b_first + (size_t)(t / (unsigned long long)a.K), k = (size_t)(t % (unsigned long long)a.K);
     const size_t lo = b * (size_t)a.bucket;
     const int len = (int)min((size_t)a.bucket, a.d - lo);
     uint32_t* s_img = s_dyn + par * img_words;
@@ -395,6 +394,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
         a.offsets[k * a.nb + b] = (uint32_t)min(excl, (unsigned long long)0xffffffffu);
         s_prefix[par] = excl;
         s_skip[par] = skip;
+        s_ticket[par ^ 1] = atomicAdd(a.ticket, 1u);
       }
     }
     __syncthreads();
@@ -984,7 +984,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   uint32_t* stream = (uint32_t*)ws_get(c, base + 0, sizeof(uint32_t) * ((size_t)K * cap + 64));   // slack: see Window
   uint32_t* bbits = (uint32_t*)ws_get(c, base + 1, sizeof(uint32_t) * (size_t)K * nb);
   uint32_t* offs = (uint32_t*)ws_get(c, base + 2, sizeof(uint32_t) * (size_t)K * nb);
-  // one block per slot, zeroed by one memset: the per-worker bit totals, the status words of the scan
+  // one block per slot, zeroed by one memset: the per-worker bit totals, the ticket counter, the status words of the scan
   unsigned long long* tot = (unsigned long long*)ws_get(c, base + 3, sizeof(uint64_t) * ((size_t)K + 2 + (size_t)K * nb));
   unsigned long long* status = tot ? tot + K + 2 : nullptr;
   float* norms = (float*)ws_get(c, slot == 0 ? WS_NORMS : WS_NORMS2, sizeof(float) * (size_t)K * nb);
@@ -1001,7 +1001,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   ea.src = src; ea.d = d; ea.bucket = bucket; ea.K = K; ea.nb = nb; ea.norm_type = cfg->norm_type; ea.xid = xid; ea.quad_base = coord_base / kQuad;
   ea.vec_ok = (d % kQuad == 0) && (src.ld % kQuad == 0) && ((reinterpret_cast<uintptr_t>(src.v) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
   ea.stream = stream; ea.cap_words = cap; ea.bucket_bits = bbits; ea.offsets = offs; ea.total_bits = tot; ea.norms = norms;
-  ea.status = status; ea.st = c->dstatus;
+  ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(tot + K); ea.st = c->dstatus;
   uint8_t* sym_out = nullptr;
   const uint8_t* sym_prev = nullptr;
   const size_t sym_ld = ((nb * (size_t)(bucket / ct.G) + 31) / 32) * 32 * (size_t)ct.G;   // see DecodeArgs::sym_out
@@ -1087,7 +1087,10 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
       shape.per_sm = per_sm < 1 ? 1 : per_sm;                                                                        \
     }                                                                                                                \
     const unsigned grid = (unsigned)std::min<unsigned long long>((groups + 1ull) / 2ull, (unsigned long long)c->num_sms * (unsigned long long)shape.per_sm); \
-    k_encode_staged<GG><<<grid, kStagedThreads, smem_st, c->stream>>>(ea, lt, ct, key, qt, tmap);                    \
+    /* a cooperative launch: the static assignment of groups needs every CTA of the grid resident at once, */       \
+    /* also when other kernels (another exchange on a helper stream) share the device                      */       \
+    void* kargs[] = {(void*)&ea, (void*)&lt, (void*)&ct, (void*)&key, (void*)&qt, (void*)&tmap};                     \
+    cudaLaunchCooperativeKernel((const void*)k_encode_staged<GG>, dim3(grid), dim3(kStagedThreads), kargs, smem_st, c->stream); \
   } while (0)
       if (ct.G == 32) QGX_LAUNCH_SG(32);
       else if (ct.G == 64) QGX_LAUNCH_SG(64);

@@ -125,12 +125,17 @@ def test_microbench_config_on_sampled_buckets():
         qgx.qgx_destroy(ctx)
 
 
-def test_layerwise_config_on_sampled_buckets():
+@pytest.mark.parametrize("staged", [False, True], ids=["bucket in registers", "staged encode"])
+def test_layerwise_config_on_sampled_buckets(staged):
     """The 16 layer-shaped tensors at their full sizes (each size twice), K = 16, bucket 4096, per-tensor tables and
-    codes: first, last (the smallest tensors are one partial bucket) and one inner bucket of every tensor."""
+    codes: first, last (the smallest tensors are one partial bucket) and one inner bucket of every tensor.  The
+    tensors' exchanges run side by side on helper streams, so no encode kernel has the device to itself: every
+    wait of the offset scan must still end (a wait that ran out would latch QGX_ERR_TIMEOUT)."""
     import paper_2308_09187_b200 as qgx
     ctx = qgx.qgx_create(0)
     try:
+        if staged:
+            qgx.qgx_set_encode_path(ctx, qgx.QGX_ENCODE_STAGED)
         lw = gen.c3_layerwise(K=16, device="cuda")
         K, d = lw.v.shape
         assert len(lw.sizes) == 16 and d == 2 * sum(gen.C3_TENSOR_SIZES)
