@@ -3,51 +3,113 @@
 // qgx_update_levels, which feeds it to the host-side fit and code builders.
 #include "qgx_bucket.cuh"
 
+#include <algorithm>
 #include <vector>
 
 namespace qgx {
 
 constexpr int kMaxBins = 4096;
 
-// One CTA per (bucket, worker): counts per bin in shared memory, then one fp64 atomic per
-// occupied bin adds count * weight to the global histogram.
-template <int V4>
-__global__ void __launch_bounds__(512) k_histogram(DualSource src, size_t d, int bucket, int norm_type, int nbins, int weighted,
-                                                   bool vec_ok, double* __restrict__ hist, DevStatus* st) {
-  extern __shared__ uint32_t s_cnt[];
-  __shared__ double s_red[34];
-  const size_t b = blockIdx.x, k = blockIdx.y;
-  const size_t lo = b * (size_t)bucket;
-  const int len = (int)min((size_t)bucket, d - lo);
-  for (int i = threadIdx.x; i < nbins; i += blockDim.x) s_cnt[i] = 0;
+// Bin of one coordinate: floor(fl(fl(|x| / norm) * nbins)), clamped to the last bin -- the definition, in IEEE
+// operations.
+__device__ __forceinline__ int bin_exact(float x, float norm, float nbf, int nbins) {
+  float u = (norm > 0.0f) ? __fdiv_rn(fabsf(x), norm) : 0.0f;
+  u = fminf(u, 1.0f);
+  return min((int)floorf(__fmul_rn(u, nbf)), nbins - 1);
+}
 
-  BucketRegs<V4> r;
-  load_bucket<V4>(r, src, k, d, lo, len, vec_ok);
-  const float norm = bucket_norm<V4>(r, norm_type, s_red);     // contains __syncthreads
-  if (!((norm - norm) == 0.0f)) {
-    if (threadIdx.x == 0) latch_error(st, QGX_ERR_NONFINITE);
-    return;
-  }
+// floor(t) of t = min(|x| * c, nbins), c = fl(nbins / norm), read from the mantissa of t + (2^23 - 1/2) -- one exact
+// rounding to the nearest integer of t - 1/2 (which is -1/2, read as bin 0, while t < 1/4) -- and whether it is
+// safely the bin of x: t differs from the defining product T by less than 4.0001 * 2^-24 * T < 2^-21.9 * t (four
+// roundings), so floor(t) = floor(T) whenever t keeps a distance of 2^-21 * t from the integers.  A t that is not
+// finite, or that reaches nbins, is never safe.
+struct FastBin { int bin; bool safe; };
+__device__ __forceinline__ FastBin fast_bin(float x, float c, float nbf) {
+  const float kMagic = 8388607.5f;                                    // 2^23 - 1/2
+  const float tt = fminf(__fmul_rn(fabsf(x), c), nbf);
+  const float m = __fadd_rn(tt, kMagic);
+  FastBin f;
+  f.bin = max((int)__float_as_uint(m) - 0x4B000000, 0);
+  const float dist = __fsub_rn(tt, __fsub_rn(m, kMagic));             // t - (floor(t) + 1/2)
+  f.safe = fabsf(dist) <= __fmaf_rn(tt, -4.76837158203125e-07f, 0.5f);
+  return f;
+}
+
+// Persistent CTAs: bucket t of the launch (b = t / K, k = t % K, so that CTAs working side by side share the
+// operator's bucket in L2) belongs to CTA t mod gridDim.x.  Counts per bin of one bucket in shared memory, folded
+// after each bucket into the CTA's own fp64 histogram (count * weight); one fp64 atomic per occupied bin and CTA at
+// the end.
+//
+// A coordinate whose bin fast_bin cannot vouch for (a few in a million for bins of small index) takes the defining
+// operations after the thread's other coordinates.
+template <int V4>
+__global__ void __launch_bounds__(512, 2) k_histogram(DualSource src, size_t d, int bucket, size_t nb, int K, int norm_type,
+                                                      int nbins, int weighted, bool vec_ok, double* __restrict__ hist,
+                                                      DevStatus* st) {
+  extern __shared__ __align__(8) unsigned char s_raw[];
+  double* s_hist = reinterpret_cast<double*>(s_raw);                 // [nbins]
+  uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_hist + nbins);      // [nbins + 1]
+  __shared__ double s_red[34];
+  for (int i = threadIdx.x; i < nbins; i += blockDim.x) { s_hist[i] = 0.0; s_cnt[i] = 0u; }
   const float nbf = (float)nbins;
+  const unsigned long long total = (unsigned long long)nb * (unsigned long long)K;
+  for (unsigned long long t = blockIdx.x; t < total; t += gridDim.x) {
+    const size_t b = (size_t)(t / (unsigned long long)K), k = (size_t)(t % (unsigned long long)K);
+    const size_t lo = b * (size_t)bucket;
+    const int len = (int)min((size_t)bucket, d - lo);
+    BucketRegs<V4> r;
+    load_bucket<V4>(r, src, k, d, lo, len, vec_ok);
+    const float norm = bucket_norm<V4>(r, norm_type, s_red);   // contains __syncthreads: the fold of the last bucket is done
+    const bool finite = (norm - norm) == 0.0f;
+    if (!finite) {
+      if (threadIdx.x == 0) latch_error(st, QGX_ERR_NONFINITE);
+    } else {
+      if (len == (int)blockDim.x * V4 * kQuad) {                   // every thread's quads lie inside the bucket
+        const float c = (norm > 0.0f) ? __fdiv_rn(nbf, norm) : 0.0f;
+        bool redo = false;                                         // one of this thread's coordinates is not safe
 #pragma unroll
-  for (int j = 0; j < V4; ++j) {
-    const int e = (j * (int)blockDim.x + (int)threadIdx.x) * kQuad;
-    const float x[kQuad] = {r.x[j].x, r.x[j].y, r.x[j].z, r.x[j].w};
+        for (int j = 0; j < V4; ++j) {
+          const float x[kQuad] = {r.x[j].x, r.x[j].y, r.x[j].z, r.x[j].w};
 #pragma unroll
-    for (int c = 0; c < kQuad; ++c) {
-      if (e + c < len) {
-        float u = (norm > 0.0f) ? __fdiv_rn(fabsf(x[c]), norm) : 0.0f;
-        u = fminf(u, 1.0f);
-        const int bin = min((int)floorf(__fmul_rn(u, nbf)), nbins - 1);
-        atomicAdd(&s_cnt[bin], 1u);
+          for (int q = 0; q < kQuad; ++q) {
+            const FastBin f = fast_bin(x[q], c, nbf);
+            redo = redo || !f.safe;
+            atomicAdd(&s_cnt[f.safe ? f.bin : nbins], 1u);         // entry nbins collects the unsafe ones and is never read
+          }
+        }
+        if (redo) {                                                // rare: the thread's coordinates are read again
+          for (int j = 0; j < V4; ++j) {
+            const size_t e = lo + (size_t)(j * (int)blockDim.x + (int)threadIdx.x) * kQuad;
+            for (int q = 0; q < kQuad; ++q) {
+              const float xq = dual_value(src, k, d, e + q);
+              if (!fast_bin(xq, c, nbf).safe) atomicAdd(&s_cnt[bin_exact(xq, norm, nbf, nbins)], 1u);
+            }
+          }
+        }
+      } else {                                                     // a short last bucket: the defining operations
+#pragma unroll
+        for (int j = 0; j < V4; ++j) {
+          const int e = (j * (int)blockDim.x + (int)threadIdx.x) * kQuad;
+          const float x[kQuad] = {r.x[j].x, r.x[j].y, r.x[j].z, r.x[j].w};
+#pragma unroll
+          for (int q = 0; q < kQuad; ++q)
+            if (e + q < len) atomicAdd(&s_cnt[bin_exact(x[q], norm, nbf, nbins)], 1u);
+        }
+      }
+    }
+    __syncthreads();
+    if (finite) {
+      const double wgt = weighted ? (double)norm * (double)norm : 1.0;
+      for (int i = threadIdx.x; i < nbins; i += blockDim.x) {
+        const uint32_t n = s_cnt[i];
+        if (n) { s_hist[i] += (double)n * wgt; s_cnt[i] = 0u; }
       }
     }
   }
   __syncthreads();
-  const double wgt = weighted ? (double)norm * (double)norm : 1.0;
   for (int i = threadIdx.x; i < nbins; i += blockDim.x) {
-    const uint32_t n = s_cnt[i];
-    if (n) atomicAdd(&hist[i], (double)n * wgt);
+    const double h = s_hist[i];
+    if (h != 0.0) atomicAdd(&hist[i], h);
   }
 }
 
@@ -63,15 +125,24 @@ qgx_status launch_histogram(qgx_ctx* c, DualSource src, int K, size_t d, int buc
                       ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
   const int v4 = bucket_v4(bucket);
   const int threads = bucket_threads(bucket, v4);
-  const dim3 grid((unsigned)nb, (unsigned)K);
-  const size_t smem = sizeof(uint32_t) * (size_t)nbins;
+  const size_t smem = (sizeof(double) + sizeof(uint32_t)) * (size_t)nbins + 16;
+  const unsigned long long total = (unsigned long long)nb * (unsigned long long)K;
   ScopedKernelTimer timer(c, QGX_KERNEL_HISTOGRAM);
+#define QGX_LAUNCH_H(V)                                                                                              \
+  do {                                                                                                               \
+    int per_sm = 1;                                                                                                  \
+    if (smem > 40u * 1024u) cudaFuncSetAttribute(k_histogram<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_histogram<V>, threads, smem);                           \
+    const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)c->num_sms * (unsigned long long)std::max(per_sm, 1)); \
+    k_histogram<V><<<grid, threads, smem, c->stream>>>(src, d, bucket, nb, K, norm_type, nbins, weighted, vec_ok, hist, c->dstatus); \
+  } while (0)
   switch (v4) {
-    case 1: k_histogram<1><<<grid, threads, smem, c->stream>>>(src, d, bucket, norm_type, nbins, weighted, vec_ok, hist, c->dstatus); break;
-    case 2: k_histogram<2><<<grid, threads, smem, c->stream>>>(src, d, bucket, norm_type, nbins, weighted, vec_ok, hist, c->dstatus); break;
-    case 4: k_histogram<4><<<grid, threads, smem, c->stream>>>(src, d, bucket, norm_type, nbins, weighted, vec_ok, hist, c->dstatus); break;
-    default: k_histogram<8><<<grid, threads, smem, c->stream>>>(src, d, bucket, norm_type, nbins, weighted, vec_ok, hist, c->dstatus); break;
+    case 1: QGX_LAUNCH_H(1); break;
+    case 2: QGX_LAUNCH_H(2); break;
+    case 4: QGX_LAUNCH_H(4); break;
+    default: QGX_LAUNCH_H(8); break;
   }
+#undef QGX_LAUNCH_H
   count_launch(c);
   return cuda_status(cudaGetLastError());
 }

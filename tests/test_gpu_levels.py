@@ -1,6 +1,7 @@
 """Parity of the histogram kernel and of qgx_update_levels with the oracle."""
 import numpy as np
 import pytest
+import torch
 
 import qgx_inputs as gen
 from oracle import qgx_oracle as o
@@ -38,6 +39,32 @@ def test_histogram(q, K, d, bucket, nbins):
     qgx.qgx_sync_status(ctx)
     assert np.array_equal(hl.cpu().numpy(), o.histogram(vh, bucket, nbins, o.LINF, False))
     assert n_ref.shape == (K, o.nbuckets(d, bucket))
+
+
+def test_histogram_on_bin_edges(q):
+    """Coordinates that sit on, just below and just above the bin edges (u * nbins an integer, or one fp32 step
+    away from one), tiny and zero coordinates, and an all-zero bucket, under the max-norm (the bucket's largest
+    entry is 1, so u = |v| exactly): the counts must equal the oracle's, which takes the division and the product."""
+    qgx, ctx = q
+    K, bucket, nbins = 2, 4096, 64
+    rng = np.random.default_rng(11)
+    edges = (rng.integers(0, nbins + 1, size=(K, 2 * bucket)) / nbins).astype(np.float32)
+    step = rng.integers(-2, 3, size=edges.shape)
+    v = edges.copy()
+    for s_ in (-2, -1, 1, 2):
+        for _ in range(abs(s_)):
+            v = np.where(step == s_, np.nextafter(v, np.float32(2.0 if s_ > 0 else -1.0), dtype=np.float32), v)
+    v = np.clip(v, 0.0, 1.0).astype(np.float32)
+    v[:, 0] = 1.0
+    v[:, bucket] = 1.0
+    v[:, 1:9] = [0.0, 1e-45, 1e-30, 1e-10, 0.2499 / nbins, 0.25 / nbins, 0.9999999 / nbins, 1.0 / nbins]
+    v *= np.where(rng.random(v.shape) < 0.5, -1.0, 1.0).astype(np.float32)
+    v = np.concatenate([v, np.zeros((K, bucket), dtype=np.float32)], axis=1)
+    got = qgx.qgx_histogram(ctx, torch.from_numpy(v).cuda(), bucket, nbins, norm_type=qgx.QGX_NORM_LINF, weighted=False)
+    qgx.qgx_sync_status(ctx)
+    ref = o.histogram(v, bucket, nbins, o.LINF, False)
+    assert ref[0] >= K * bucket and ref[nbins - 1] >= 2 * K
+    assert np.array_equal(got.cpu().numpy(), ref)
 
 
 def test_update_levels_matches_oracle_refit(q):
