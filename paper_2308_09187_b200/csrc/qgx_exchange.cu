@@ -8,8 +8,10 @@
 
 #include <algorithm>
 #include <cstring>
+#include <limits>
 #include <mutex>
 #include <new>
+#include <type_traits>
 #include <vector>
 
 namespace qgx {
@@ -415,8 +417,9 @@ namespace qgx {
 
 // ---- decode + average ------------------------------------------------------------------------
 // Decoder table of the fused path: index = the next maxlen + 1 stream bits (codeword, then the sign
-// bit of a nonzero level); entry = the signed level value and the bits consumed (bit 7 set: no
-// codeword starts like this, one bit is consumed so that the walk goes on and the lengths disagree).
+// bit of a nonzero level); entry = the signed level value and, in `len`, the bits consumed (bits 0..4) and the
+// symbol byte (bits 8..15).  Where no codeword starts like the index the value is NaN -- it stays in the running
+// sum of its coordinate, where the kernel looks for it -- and one bit is consumed so that the walk goes on.
 struct DecEntry {
   float val;
   uint32_t len;
@@ -459,24 +462,38 @@ constexpr int kDecThreads = 128;
 
 // Bits not yet consumed of one sub-block: a 64-bit window refilled 32 bits at a time.  The streams
 // of the fused path lie in the context's workspace, which extends past every bucket, so a read a
-// few words beyond a (corrupt) sub-block stays inside allocated memory.
+// few words beyond a (corrupt) sub-block stays inside allocated memory.  SH: the words are read from the warp's
+// staged row by shared-memory loads (the address is a 32-bit shared address); otherwise from wherever p points.
+template <bool SH>
 struct Window {
-  const uint32_t* next;   // address of `ahead`
+  using Addr = typename std::conditional<SH, uint32_t, const uint32_t*>::type;
+  Addr next;              // address of `ahead`
+  Addr first;             // address of the word that held the first bit
   uint32_t lo, hi;
   uint32_t ahead;         // the word after the window, fetched one refill early
   int avail;
-  // p = address of the word that holds the first bit (shared or global memory), sh = first bit within it
+  uint32_t sh0;
+  static __device__ __forceinline__ uint32_t word(uint32_t a) { return lds32(a); }
+  static __device__ __forceinline__ uint32_t word(const uint32_t* a) { return *a; }
+  static __device__ __forceinline__ Addr at(const uint32_t* p, std::true_type) { return smem_addr(p); }
+  static __device__ __forceinline__ Addr at(const uint32_t* p, std::false_type) { return p; }
+  static __device__ __forceinline__ uint32_t step(uint32_t a, int words) { return a + 4u * (uint32_t)words; }
+  static __device__ __forceinline__ const uint32_t* step(const uint32_t* a, int words) { return a + words; }
+  // p = address of the word that holds the first bit, sh = first bit within it
   __device__ __forceinline__ void open(const uint32_t* p, uint32_t sh) {
-    const uint32_t w0 = p[0], w1 = p[1], w2 = p[2];
+    first = at(p, std::integral_constant<bool, SH>());
+    const uint32_t w0 = word(first), w1 = word(step(first, 1)), w2 = word(step(first, 2));
     lo = __funnelshift_r(w0, w1, sh);
     hi = w1 >> sh;
     avail = 64 - (int)sh;                               // the window ends on a word boundary
+    sh0 = sh;
     ahead = w2;
-    next = p + 2;
+    next = step(first, 2);
   }
   __device__ __forceinline__ void refill() {            // needs avail <= 32
     const uint32_t w = ahead;
-    ahead = *++next;                                    // not needed before the next refill
+    next = step(next, 1);
+    ahead = word(next);                                 // not needed before the next refill
     lo |= __funnelshift_lc(0u, w, (uint32_t)avail);     // w << avail, nothing when avail == 32
     hi |= __funnelshift_lc(w, 0u, (uint32_t)avail);     // the bits of w that do not fit the low word
     avail += 32;
@@ -486,6 +503,10 @@ struct Window {
     hi >>= n;
     avail -= (int)n;
   }
+  static __device__ __forceinline__ uint32_t words_from(uint32_t a, uint32_t b) { return (a - b) >> 2; }
+  static __device__ __forceinline__ uint32_t words_from(const uint32_t* a, const uint32_t* b) { return (uint32_t)(a - b); }
+  // bits consumed since open(): the words taken in so far, less what is still in the window
+  __device__ __forceinline__ uint32_t used() const { return 32u * words_from(next, first) - sh0 - (uint32_t)avail; }
 };
 
 // start of sub-block `s` (bits after the header) = sum of the 16-bit lengths before it; all lanes of
@@ -550,6 +571,7 @@ struct SubBlockAt {
   float norm;
   float norm_prev;        // norm of the same bucket in the other exchange (when comparing)
   bool ok;
+  bool staged;            // p points into the warp's staged row
 };
 
 // Words that a thread may read past the first word of its sub-block: G symbols of at most 13 bits, the
@@ -576,6 +598,7 @@ __device__ __forceinline__ SubBlockAt find_subblock(const DecodeArgs& a, int k, 
   r.sh = st & 31u;
   // bucket-level validity is the same for all lanes; the lengths are bounded, so the row is at most 2^19 bits
   const bool stage = uniform && __all_sync(0xffffffffu, r.ok) && row_bits < (1u << 19);
+  r.staged = false;
   if (stage) {
     const size_t first = (size_t)(w - a.stream) + ((hdr_bits + row_before) >> 5);       // word index in the whole buffer
     const size_t first_al = first & ~(size_t)3;                                          // 16-byte aligned
@@ -586,7 +609,7 @@ __device__ __forceinline__ SubBlockAt find_subblock(const DecodeArgs& a, int k, 
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(a.stream + first_al + 4 * (size_t)c) : "memory");
     }
     const size_t mine = (size_t)(r.p - a.stream) - first_al;
-    if (mine + DecodeReach<G>::kWords <= (size_t)nwords) r.p = row + mine;
+    if (mine + DecodeReach<G>::kWords <= (size_t)nwords) { r.p = row + mine; r.staged = true; }
   }
   r.norm_prev = a.norms_prev ? a.norms_prev[(size_t)k * a.nb + b] : 0.0f;
   return r;
@@ -688,60 +711,69 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
       asm volatile("cp.async.wait_group 1;" ::: "memory");       // worker k's rows have landed
       __syncwarp();
       bad = bad || !cur.ok;
-      Window win;
-      win.open(cur.p, cur.sh);
-      uint32_t flags = 0, used = 0;
-      if (count == G) {
-        uint32_t pack = 0, prev4 = 0;
+      uint32_t used = 0;
+      // the walk over the sub-block's symbols, with the window's words read from the staged row (every lane's
+      // words are there) or from wherever they are
+      auto walk = [&](auto shared_tag) {
+        Window<decltype(shared_tag)::value> win;
+        win.open(cur.p, cur.sh);
+        if (count == G) {
+          uint32_t pack = 0, prev4 = 0;
 #pragma unroll
-        for (int i = 0; i < G; ++i) {
-          if ((i & 1) == 0) {                              // two symbols use at most 26 bits
-            if (win.avail <= 32) win.refill();
-          }
-          if (kCompare && (i & 3) == 0) prev4 = prev_row[(i >> 2) * 32];
-          const DecEntry e = s_lut[win.lo & mask];
-          const uint32_t L = e.len & 31u;
-          flags |= e.len;
-          win.skip(L);
-          used += L;
-          const float val = __fmul_rn(cur.norm, e.val);
-          acc[i] = __fadd_rn(acc[i], val);
-          if (kCompare) {
-            const float dlt = __fsub_rn(dequantize_symbol((prev4 >> (8 * (i & 3))) & 0xffu, cur.norm_prev, s_lev), val);
-            sq = fma((double)dlt, (double)dlt, sq);
-          }
-          if (kSquare) sq = fma((double)val, (double)val, sq);
-          if (kStore) {
-            pack |= ((e.len >> 8) & 0xffu) << (8 * (i & 3));
-            if ((i & 3) == 3) { *reinterpret_cast<uint32_t*>(a.sym_out + (size_t)k * a.sym_ld + sbase + (i >> 2) * 128) = pack; pack = 0; }
-          }
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < G; ++i) {
-          if ((i & 1) == 0) {
-            if (win.avail <= 32) win.refill();
-          }
-          if (i < count) {
+          for (int i = 0; i < G; ++i) {
+            if ((i & 1) == 0) {                              // two symbols use at most 26 bits
+              if (win.avail <= 32) win.refill();
+            }
+            if (kCompare && (i & 3) == 0) prev4 = prev_row[(i >> 2) * 32];
             const DecEntry e = s_lut[win.lo & mask];
-            const uint32_t L = e.len & 31u;
-            flags |= e.len;
-            win.skip(L);
-            used += L;
+            win.skip(e.len & 31u);
             const float val = __fmul_rn(cur.norm, e.val);
             acc[i] = __fadd_rn(acc[i], val);
             if (kCompare) {
-              const float dlt = __fsub_rn(dequantize_symbol(a.sym_prev[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)], cur.norm_prev, s_lev), val);
+              const float dlt = __fsub_rn(dequantize_symbol((prev4 >> (8 * (i & 3))) & 0xffu, cur.norm_prev, s_lev), val);
               sq = fma((double)dlt, (double)dlt, sq);
             }
             if (kSquare) sq = fma((double)val, (double)val, sq);
-            if (kStore) a.sym_out[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)] = (uint8_t)((e.len >> 8) & 0xffu);
+            if (kStore) {
+              // byte 1 of e.len, the symbol byte, becomes byte i % 4 of the word
+              pack = prmt(pack, e.len, (i & 3) == 0 ? 0x3215u : ((i & 3) == 1 ? 0x3250u : ((i & 3) == 2 ? 0x3510u : 0x5210u)));
+              if ((i & 3) == 3) *reinterpret_cast<uint32_t*>(a.sym_out + (size_t)k * a.sym_ld + sbase + (i >> 2) * 128) = pack;
+            }
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < G; ++i) {
+            if ((i & 1) == 0) {
+              if (win.avail <= 32) win.refill();
+            }
+            if (i < count) {
+              const DecEntry e = s_lut[win.lo & mask];
+              win.skip(e.len & 31u);
+              const float val = __fmul_rn(cur.norm, e.val);
+              acc[i] = __fadd_rn(acc[i], val);
+              if (kCompare) {
+                const float dlt = __fsub_rn(dequantize_symbol(a.sym_prev[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)], cur.norm_prev, s_lev), val);
+                sq = fma((double)dlt, (double)dlt, sq);
+              }
+              if (kSquare) sq = fma((double)val, (double)val, sq);
+              if (kStore) a.sym_out[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)] = (uint8_t)((e.len >> 8) & 0xffu);
+            }
           }
         }
-      }
-      bad = bad || (flags & 0x80u) || (count > 0 && used != cur.want);   // every sub-block uses exactly its length
+        used = win.used();
+      };
+      if (__all_sync(0xffffffffu, cur.staged)) walk(std::true_type());
+      else walk(std::false_type());
+      bad = bad || (count > 0 && used != cur.want);          // every sub-block uses exactly its length
     }
     if (count <= 0) continue;
+    {
+      // an index that no codeword starts like left a NaN in its coordinate's sum (as a norm that is not finite does)
+      bool marked = false;
+#pragma unroll
+      for (int i = 0; i < G; ++i) marked = marked || (acc[i] != acc[i]);
+      bad = bad || marked;
+    }
     if (wide) {                                         // the worker's values; summed by k_sum_workers
       float* out = a.values + (size_t)kbeg * a.d + e0;
       if (count == G && a.vec_out) {
@@ -910,7 +942,7 @@ static qgx_status cached_tables(qgx_ctx* c, const qgx_quant_cfg* cfg, const Cach
     for (size_t i = 0; i < h_lut.size(); ++i) {
       const uint16_t w = by_code[i & (((size_t)1 << ct.maxlen) - 1)];
       const uint32_t L = w >> 8, idx = w & 0xffu;
-      if (L == 0) { h_lut[i].val = 0.0f; h_lut[i].len = 1u | 0x80u; continue; }
+      if (L == 0) { h_lut[i].val = std::numeric_limits<float>::quiet_NaN(); h_lut[i].len = 1u; continue; }   // no codeword starts like this
       if (idx == 0) { h_lut[i].val = 0.0f; h_lut[i].len = L; continue; }       // symbol byte 0
       const bool neg = (i >> L) & 1u;
       h_lut[i].val = neg ? -cfg->levels[idx] : cfg->levels[idx];
