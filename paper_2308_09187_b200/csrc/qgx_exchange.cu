@@ -665,6 +665,9 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
   const size_t total_sub = a.nb * spb;
   const bool uniform = (spb % 32 == 0);
   const float Kf = (float)a.K;
+  // the mean is sum / K, one fp32 division; for K a power of two the product with 1 / K is the same number
+  const bool k_pow2 = (a.K & (a.K - 1)) == 0;
+  const float Kinv = 1.0f / Kf;
   bool bad = false;
   double sq = 0.0;
 
@@ -790,18 +793,23 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
     float gam = 1.0f;
     if (a.update == 1) gam = (float)a.scalars[1];
     if (count == G && a.vec_out) {
+      auto emit = [&](auto pow2_tag) {
+        auto mean_of = [&](float sum) { return decltype(pow2_tag)::value ? __fmul_rn(sum, Kinv) : __fdiv_rn(sum, Kf); };
 #pragma unroll
-      for (int i = 0; i < G; i += 4) {
-        const float4 m = make_float4(__fdiv_rn(acc[i], Kf), __fdiv_rn(acc[i + 1], Kf), __fdiv_rn(acc[i + 2], Kf), __fdiv_rn(acc[i + 3], Kf));
-        *reinterpret_cast<float4*>(a.mean + e0 + i) = m;
-        if (a.update != 0) {
-          const float4 x = *reinterpret_cast<const float4*>(a.xin + e0 + i);
-          const float g = a.update == 1 ? gam : 1.0f;      // update 2 subtracts the mean itself (1 * m is exact)
-          *reinterpret_cast<float4*>(a.xout + e0 + i) =
-              make_float4(__fsub_rn(x.x, __fmul_rn(g, m.x)), __fsub_rn(x.y, __fmul_rn(g, m.y)),
-                          __fsub_rn(x.z, __fmul_rn(g, m.z)), __fsub_rn(x.w, __fmul_rn(g, m.w)));
+        for (int i = 0; i < G; i += 4) {
+          const float4 m = make_float4(mean_of(acc[i]), mean_of(acc[i + 1]), mean_of(acc[i + 2]), mean_of(acc[i + 3]));
+          *reinterpret_cast<float4*>(a.mean + e0 + i) = m;
+          if (a.update != 0) {
+            const float4 x = *reinterpret_cast<const float4*>(a.xin + e0 + i);
+            const float g = a.update == 1 ? gam : 1.0f;      // update 2 subtracts the mean itself (1 * m is exact)
+            *reinterpret_cast<float4*>(a.xout + e0 + i) =
+                make_float4(__fsub_rn(x.x, __fmul_rn(g, m.x)), __fsub_rn(x.y, __fmul_rn(g, m.y)),
+                            __fsub_rn(x.z, __fmul_rn(g, m.z)), __fsub_rn(x.w, __fmul_rn(g, m.w)));
+          }
         }
-      }
+      };
+      if (k_pow2) emit(std::true_type());
+      else emit(std::false_type());
     } else {
 #pragma unroll
       for (int i = 0; i < G; ++i) {
