@@ -66,7 +66,10 @@ typedef struct {
 } qgx_codebook;
 
 /* Quantizer configuration (Definition 1 + Sec. 3.2).  levels[0] = 0 < ... < levels[nlev-1] = 1.
- * In the paper's counting "s levels" means nlev = s + 2. */
+ * nlev counts every entry of the table, the end points 0 and 1 among them.  Definition 1 writes the table as
+ * 0 = l_0 < l_1 < ... < l_s < l_{s+1} = 1, so its s (the free levels between the end points) is nlev - 2; where the
+ * paper's experiments speak of "s levels" of a uniform quantizer with s quantization intervals, the table has
+ * nlev = s + 1 entries (the convention of the benchmark's configurations). */
 typedef struct {
   int32_t nlev;
   int32_t bucket;           /* multiple of 4, <= QGX_MAX_BUCKET */
