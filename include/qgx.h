@@ -253,7 +253,7 @@ qgx_status qgx_exchange_segments(qgx_ctx *ctx, const float *v, int K, size_t d, 
  * order (same results, K times more threads, K * d floats of workspace, at most 256 MB); large vectors are decoded
  * by one thread per sub-block over all workers.  QGX_SPLIT_NEVER / QGX_SPLIT_ALWAYS force one way (ALWAYS still
  * falls back when the workspace would exceed 256 MB). */
-enum { QGX_SPLIT_AUTO = 0, QGX_SPLIT_NEVER = 1, QGX_SPLIT_ALWAYS = 2 };
+enum { QGX_SPLIT_AUTO = 0, QGX_SPLIT_NEVER = 1, QGX_SPLIT_ALWAYS = 2, QGX_SPLIT_SYMBOLS = 3 };
 qgx_status qgx_set_decode_split(qgx_ctx *ctx, int mode);
 /* Which kernel the encode pass of the fused calls uses (no counterpart in the paper; the streams are the same bit
  * for bit).  QGX_ENCODE_REGISTERS: one CTA per bucket, the bucket held in registers between the norm and the

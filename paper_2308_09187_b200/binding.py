@@ -345,7 +345,7 @@ def qgx_exchange_segments(ctx, v, sizes, cfgs, exchange_id, mean_out=None, total
     return mean_out, total_bits
 
 
-QGX_SPLIT_AUTO, QGX_SPLIT_NEVER, QGX_SPLIT_ALWAYS = 0, 1, 2
+QGX_SPLIT_AUTO, QGX_SPLIT_NEVER, QGX_SPLIT_ALWAYS, QGX_SPLIT_SYMBOLS = 0, 1, 2, 3
 
 
 def qgx_set_decode_split(ctx, mode):

@@ -445,6 +445,9 @@ struct DecodeArgs {
   // small vectors: a thread decodes its sub-block of ONE worker and stores the values to values[K][d]; the
   // ordered sum over the workers, the division and the state update follow in k_sum_workers
   float* values;                // [K][d] or null
+  // large vectors: the walk alone (one worker per thread, VAL = false) writes every worker's symbol bytes to sym_out
+  // and the norms it read from the streams to norms_out; k_symbols_mean forms the ordered sums from them
+  float* norms_out;             // [K][nb] or null
   // optional: keep the decoded symbols (1 byte per coordinate and worker) ...
   // Symbol bytes are kept transposed, so that a warp's accesses coalesce: worker k, sub-block gs, coordinate i of the
   // sub-block -> byte k * sym_ld + (gs / 32) * 32 * G + (i / 4) * 128 + (gs % 32) * 4 + i % 4.
@@ -459,6 +462,8 @@ struct DecodeArgs {
 };
 
 constexpr int kDecThreads = 128;
+constexpr bool kTwoPassByDefault = false;   // large vectors decode in two passes (walk, then sums) unless told otherwise
+constexpr uint32_t kBadSymbol = 0x40u;      // symbol byte of an index that no codeword starts like (no level has bit 6)
 
 // Bits not yet consumed of one sub-block: a 64-bit window refilled 32 bits at a time.  The streams
 // of the fused path lie in the context's workspace, which extends past every bucket, so a read a
@@ -626,36 +631,47 @@ __device__ __forceinline__ void stage_symbol_row(uint32_t* dst, const uint8_t* s
   }
 }
 
-// shared memory of the decode kernel after its table: two stream rows and (when comparing) two symbol rows per warp
-template <int G, int SYM>
+// shared memory of the decode kernel after its table: per warp two stream rows and (when comparing) two symbol rows --
+// one of each when a thread walks a single worker and nothing is fetched a worker ahead (VAL = false)
+template <int G, int SYM, bool VAL>
 struct DecodeSmem {
   static constexpr int kStreamRow = 9 * G + 64;         // words, a multiple of 4
-  static constexpr size_t kBytes = sizeof(uint32_t) * 2 * (128 / 32) * (size_t)(kStreamRow + ((SYM & 2) ? G * 8 : 0));
+  static constexpr int kBufs = VAL ? 2 : 1;
+  static constexpr size_t kBytes = sizeof(uint32_t) * kBufs * (128 / 32) * (size_t)(kStreamRow + ((SYM & 2) ? G * 8 : 0));
 };
 
 // SYM, a set of bits: 1 keeps the decoded symbols; 2 adds the squared differences between the vectors kept by an
 // earlier exchange (whose level table is `lt`) and the ones decoded now to *sum_sq; 4 adds the squared decoded values
 // themselves (an earlier vector of zero).  1 | 2 compares first and then overwrites the kept symbols in place.
-template <int G, int SYM>
-__global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6)) k_exchange_decode(const __grid_constant__ DecodeArgs a,
+// VAL = false: the walk alone, one worker per thread -- no running sums, so half the registers and twice the warps;
+// symbols always go to a.sym_out, the norms read from the streams to a.norms_out.
+template <int G, int SYM, bool VAL>
+__global__ void __launch_bounds__(kDecThreads, VAL ? (G == 128 ? 3 : (G == 64 ? 4 : 6)) : 10) k_exchange_decode(const __grid_constant__ DecodeArgs a,
                                                                       const __grid_constant__ CodeTable ct,
                                                                       const __grid_constant__ LevelTable lt) {
-  constexpr bool kStore = (SYM & 1) != 0, kCompare = (SYM & 2) != 0, kSquare = (SYM & 4) != 0;
+  constexpr bool kStore = (SYM & 1) != 0 || !VAL, kCompare = VAL && (SYM & 2) != 0, kSquare = VAL && (SYM & 4) != 0;
+  constexpr int kBufs = DecodeSmem<G, SYM, VAL>::kBufs;
   extern __shared__ __align__(16) unsigned char s_raw[];
   __shared__ float s_lev[QGX_MAX_LEVELS];            // the table of the kept symbols (comparing)
   // comparing: the kept symbol words of the warp's 32 sub-blocks, one worker ahead (asynchronous copies)
   constexpr int kRowWords = G * 8;                      // 32 sub-blocks x G bytes
   // the stream words of the warp's 32 sub-blocks, one worker ahead (asynchronous copies): room for 8 bits per
   // symbol and sign on average; longer rows are partly read from the stream itself
-  constexpr int kStreamRow = DecodeSmem<G, SYM>::kStreamRow;
+  constexpr int kStreamRow = DecodeSmem<G, SYM, VAL>::kStreamRow;
   const int lut_n = 2 << ct.maxlen;
-  DecEntry* s_lut = reinterpret_cast<DecEntry*>(s_raw);                       // dynamic shared memory: table, stream rows, symbol rows
-  uint32_t* s_rows = reinterpret_cast<uint32_t*>(s_raw + sizeof(DecEntry) * (size_t)lut_n);
-  uint32_t* s_prev = s_rows + 2 * (kDecThreads / 32) * kStreamRow;
+  // dynamic shared memory: table, stream rows, symbol rows.  The walk alone needs only the entries' second word
+  // (bits consumed, symbol byte).
+  DecEntry* s_lut = reinterpret_cast<DecEntry*>(s_raw);
+  uint32_t* s_len = reinterpret_cast<uint32_t*>(s_raw);
+  uint32_t* s_rows = reinterpret_cast<uint32_t*>(s_raw + (VAL ? sizeof(DecEntry) : sizeof(uint32_t)) * (size_t)lut_n);
+  uint32_t* s_prev = s_rows + kBufs * (kDecThreads / 32) * kStreamRow;
   {
     const uint2* src = reinterpret_cast<const uint2*>(a.lut);
     uint2* dst = reinterpret_cast<uint2*>(s_lut);
-    for (int i = threadIdx.x; i < lut_n; i += blockDim.x) dst[i] = src[i];
+    for (int i = threadIdx.x; i < lut_n; i += blockDim.x) {
+      if constexpr (VAL) dst[i] = src[i];
+      else s_len[i] = src[i].y;
+    }
   }
   if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 0.0f;
   __syncthreads();
@@ -671,7 +687,7 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
   bool bad = false;
   double sq = 0.0;
 
-  const bool wide = a.values != nullptr;
+  const bool wide = !VAL || a.values != nullptr;
   const size_t sub_pad = (total_sub + 31) & ~(size_t)31;                // whole warps per worker
   const size_t items = wide ? sub_pad * (size_t)a.K : total_sub;
   for (size_t item = (size_t)blockIdx.x * blockDim.x + tid; item - lane < items; item += (size_t)gridDim.x * blockDim.x) {
@@ -690,24 +706,24 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
     const size_t e0 = lo + (size_t)first;
     const size_t sbase = (gs >> 5) * (size_t)(32 * G) + (size_t)(gs & 31) * 4;   // see DecodeArgs::sym_out
 
-    float acc[G];
+    float acc[VAL ? G : 1];
 #pragma unroll
-    for (int i = 0; i < G; ++i) acc[i] = 0.0f;
-    uint32_t* my_rows = s_prev + (kCompare ? (tid >> 5) * 2 * kRowWords : 0);
-    uint32_t* my_stream = s_rows + (tid >> 5) * 2 * kStreamRow;
+    for (int i = 0; i < (VAL ? G : 1); ++i) acc[i] = 0.0f;
+    uint32_t* my_rows = s_prev + (kCompare ? (tid >> 5) * kBufs * kRowWords : 0);
+    uint32_t* my_stream = s_rows + (tid >> 5) * kBufs * kStreamRow;
     __syncwarp();                                         // the previous sub-block's rows are no longer read
-    SubBlockAt nxt = find_subblock<G>(a, kbeg, b, hdr_bits, s, count > 0, uniform, lane, my_stream + (kbeg & 1) * kStreamRow, kStreamRow);
+    SubBlockAt nxt = find_subblock<G>(a, kbeg, b, hdr_bits, s, count > 0, uniform, lane, my_stream + (kbeg & (kBufs - 1)) * kStreamRow, kStreamRow);
     if (kCompare)
-      stage_symbol_row<kRowWords>(my_rows + (kbeg & 1) * kRowWords, a.sym_prev + (size_t)kbeg * a.sym_ld + (gs >> 5) * (size_t)(32 * G), lane);
+      stage_symbol_row<kRowWords>(my_rows + (kbeg & (kBufs - 1)) * kRowWords, a.sym_prev + (size_t)kbeg * a.sym_ld + (gs >> 5) * (size_t)(32 * G), lane);
     asm volatile("cp.async.commit_group;" ::: "memory");
     for (int k = kbeg; k < kend; ++k) {
       const SubBlockAt cur = nxt;
-      const uint32_t* prev_row = my_rows + (k & 1) * kRowWords + lane;
+      const uint32_t* prev_row = my_rows + (k & (kBufs - 1)) * kRowWords + lane;
       __syncwarp();                                       // every lane is done with the rows that are overwritten next
       if (k + 1 < kend) {
-        nxt = find_subblock<G>(a, k + 1, b, hdr_bits, s, count > 0, uniform, lane, my_stream + ((k + 1) & 1) * kStreamRow, kStreamRow);
+        nxt = find_subblock<G>(a, k + 1, b, hdr_bits, s, count > 0, uniform, lane, my_stream + ((k + 1) & (kBufs - 1)) * kStreamRow, kStreamRow);
         if (kCompare)
-          stage_symbol_row<kRowWords>(my_rows + ((k + 1) & 1) * kRowWords,
+          stage_symbol_row<kRowWords>(my_rows + ((k + 1) & (kBufs - 1)) * kRowWords,
                                       a.sym_prev + (size_t)(k + 1) * a.sym_ld + (gs >> 5) * (size_t)(32 * G), lane);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");       // one group per worker, empty after the last
@@ -728,10 +744,12 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
               if (win.avail <= 32) win.refill();
             }
             if (kCompare && (i & 3) == 0) prev4 = prev_row[(i >> 2) * 32];
-            const DecEntry e = s_lut[win.lo & mask];
+            DecEntry e;
+            if constexpr (VAL) e = s_lut[win.lo & mask];
+            else { e.len = s_len[win.lo & mask]; e.val = 0.0f; }
             win.skip(e.len & 31u);
             const float val = __fmul_rn(cur.norm, e.val);
-            acc[i] = __fadd_rn(acc[i], val);
+            if constexpr (VAL) acc[i] = __fadd_rn(acc[i], val);
             if (kCompare) {
               const float dlt = __fsub_rn(dequantize_symbol((prev4 >> (8 * (i & 3))) & 0xffu, cur.norm_prev, s_lev), val);
               sq = fma((double)dlt, (double)dlt, sq);
@@ -750,10 +768,12 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
               if (win.avail <= 32) win.refill();
             }
             if (i < count) {
-              const DecEntry e = s_lut[win.lo & mask];
+              DecEntry e;
+              if constexpr (VAL) e = s_lut[win.lo & mask];
+              else { e.len = s_len[win.lo & mask]; e.val = 0.0f; }
               win.skip(e.len & 31u);
               const float val = __fmul_rn(cur.norm, e.val);
-              acc[i] = __fadd_rn(acc[i], val);
+              if constexpr (VAL) acc[i] = __fadd_rn(acc[i], val);
               if (kCompare) {
                 const float dlt = __fsub_rn(dequantize_symbol(a.sym_prev[(size_t)k * a.sym_ld + sbase + (i >> 2) * 128 + (i & 3)], cur.norm_prev, s_lev), val);
                 sq = fma((double)dlt, (double)dlt, sq);
@@ -770,6 +790,9 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
       bad = bad || (count > 0 && used != cur.want);          // every sub-block uses exactly its length
     }
     if (count <= 0) continue;
+    if constexpr (!VAL) {
+      if (s == 0) a.norms_out[(size_t)kbeg * a.nb + b] = nxt.norm;       // the bucket's norm as the stream gives it
+    } else {
     {
       // an index that no codeword starts like left a NaN in its coordinate's sum (as a norm that is not finite does)
       bool marked = false;
@@ -821,10 +844,162 @@ __global__ void __launch_bounds__(kDecThreads, G == 128 ? 3 : (G == 64 ? 4 : 6))
         }
       }
     }
+    }   // VAL
   }
   if (kCompare || kSquare) {
     sq = warp_sum(sq);
     if (lane == 0 && sq != 0.0) atomicAdd(a.sum_sq, sq);
+  }
+  if (bad) latch_error(a.st, QGX_ERR_CORRUPT);
+}
+
+// The ordered sums of the two-pass decode: worker k's quantized coordinate is norm_k * (signed level of its symbol
+// byte), added in the order k = 0..K-1, divided by K, and the state update applied -- the same operations in the same
+// order as the one-pass kernel's.  A thread takes 16 consecutive coordinates of one sub-block (four symbol words per
+// worker; the transposed layout makes a warp's loads of one word index contiguous).  The signed level values sit in
+// shared memory once per lane (bank = lane), NaN for bytes that are no symbol: a NaN mean reports the stream.
+// SYM & 2: also adds sum_k ||vhat_k kept by the other exchange - vhat_k of this one||^2 to *sum_sq (fp32 differences,
+// fp64 sum; the kept symbols dequantized with their own table and norms); SYM & 4: sum_k ||vhat_k||^2 instead.
+struct MeanArgs {
+  const uint8_t* sym;           // [K][sym_ld], this exchange's symbol bytes (transposed layout of DecodeArgs::sym_out)
+  size_t sym_ld;
+  const float* norms;           // [K][nb], as the walk read them from the streams
+  const uint8_t* sym_prev;      // [K][sym_ld] or null
+  const float* norms_prev;      // [K][nb]
+  double* sum_sq;
+  int K;
+  size_t d;
+  int bucket;
+  size_t nb;
+  float* mean;
+  int update;
+  const float* xin;
+  float* xout;
+  const double* scalars;
+  bool vec_out;
+  DevStatus* st;
+};
+
+template <int G, int SYM>
+__global__ void __launch_bounds__(256) k_symbols_mean(const __grid_constant__ MeanArgs a, const __grid_constant__ LevelTable lt,
+                                                      const __grid_constant__ LevelTable lt_kept) {
+  constexpr bool kCompare = (SYM & 2) != 0, kSquare = (SYM & 4) != 0;
+  extern __shared__ __align__(16) float s_val[];                       // [256][32], then (comparing) the kept table [256]
+  for (int t = threadIdx.x; t < 256 * 32; t += blockDim.x) {
+    const int byte = t >> 5, idx = byte & 31;
+    const bool symbol = (byte & 0x60) == 0 && idx < lt.nlev && byte != 0x80;
+    s_val[t] = symbol ? ((byte & 0x80) ? -lt.lev[idx] : lt.lev[idx]) : __int_as_float(0x7fc00000);
+  }
+  if (kCompare) {
+    for (int t = threadIdx.x; t < 256; t += blockDim.x) {
+      const int idx = t & 31;
+      s_val[256 * 32 + t] = idx < lt_kept.nlev ? ((t & 0x80) ? -lt_kept.lev[idx] : lt_kept.lev[idx]) : 0.0f;
+    }
+  }
+  __syncthreads();
+  constexpr int kParts = G / 16;                                       // threads per sub-block
+  const uint32_t val_sa = smem_addr(s_val) + 4u * (threadIdx.x & 31u);
+  const uint32_t kept_sa = smem_addr(s_val + 256 * 32);
+  const size_t spb = (size_t)a.bucket / G, total_sub = a.nb * spb, rows = (total_sub + 31) / 32;
+  const int K = a.K;
+  const float Kf = (float)K, Kinv = 1.0f / Kf;
+  const bool k_pow2 = (K & (K - 1)) == 0;
+  const int lane = threadIdx.x & 31;
+  float gam = 1.0f;
+  if (a.update == 1) gam = (float)a.scalars[1];
+  bool bad = false;
+  double sq = 0.0;
+  const size_t ldw = a.sym_ld / 4;
+  const size_t items = rows * kParts * 32;
+  for (size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x; t < items; t += (size_t)gridDim.x * blockDim.x) {
+    const size_t rest = t >> 5, row = rest / kParts;
+    const int part = (int)(rest % kParts);
+    const size_t gs = row * 32 + (size_t)lane;
+    if (gs >= total_sub) continue;
+    const size_t b = gs / spb, lo = b * (size_t)a.bucket;
+    const int len = (int)min((size_t)a.bucket, a.d - lo);
+    const int first = (int)(gs % spb) * G + 16 * part;                 // of this thread's coordinates, within the bucket
+    const int count = max(0, min(16, len - first));
+    if (count == 0) continue;
+    const size_t word0 = row * (size_t)(8 * G) + (size_t)(4 * part) * 32 + lane;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(a.sym) + word0;
+    const uint32_t* kept = kCompare ? reinterpret_cast<const uint32_t*>(a.sym_prev) + word0 : nullptr;
+    float acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
+    auto add = [&](const uint32_t (&w)[4], const uint32_t (&p)[4], float norm, float norm_kept) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t byte = prmt(w[j], 0u, 0x4440u + (uint32_t)q);                 // byte q of the word
+          const float val = __fmul_rn(norm, __uint_as_float(lds_table32(val_sa + (byte << 7))));
+          acc[4 * j + q] = __fadd_rn(acc[4 * j + q], val);
+          if (kCompare) {
+            const uint32_t pbyte = prmt(p[j], 0u, 0x4440u + (uint32_t)q);
+            const float was = __fmul_rn(norm_kept, __uint_as_float(lds_table32(kept_sa + (pbyte << 2))));
+            const float dlt = __fsub_rn(was, val);
+            if (4 * j + q < count) sq = fma((double)dlt, (double)dlt, sq);
+          }
+          if (kSquare) { if (4 * j + q < count) sq = fma((double)val, (double)val, sq); }
+        }
+      }
+    };
+    // one worker's words and norms are asked for while the one before is added (k = K asks for nothing)
+    uint32_t w[4] = {0u, 0u, 0u, 0u}, p[4] = {0u, 0u, 0u, 0u};
+    float nrm = 0.0f, nrm_kept = 0.0f;
+    auto fetch = [&](int k, uint32_t (&fw)[4], uint32_t (&fp)[4], float* fn, float* fk) {
+      if (k >= K) return;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        fw[j] = __ldcs(words + (size_t)k * ldw + j * 32);
+        if (kCompare) fp[j] = __ldcs(kept + (size_t)k * ldw + j * 32);
+      }
+      *fn = a.norms[(size_t)k * a.nb + b];
+      if (kCompare) *fk = a.norms_prev[(size_t)k * a.nb + b];
+    };
+    fetch(0, w, p, &nrm, &nrm_kept);
+    for (int k = 0; k < K; k += 2) {
+      uint32_t w1[4] = {0u, 0u, 0u, 0u}, p1[4] = {0u, 0u, 0u, 0u};
+      float n1 = 0.0f, m1 = 0.0f;
+      fetch(k + 1, w1, p1, &n1, &m1);
+      add(w, p, nrm, nrm_kept);
+      fetch(k + 2, w, p, &nrm, &nrm_kept);
+      if (k + 1 < K) add(w1, p1, n1, m1);
+    }
+    const size_t e0 = lo + (size_t)first;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float m[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        m[q] = k_pow2 ? __fmul_rn(acc[4 * j + q], Kinv) : __fdiv_rn(acc[4 * j + q], Kf);
+        bad = bad || (4 * j + q < count && m[q] != m[q]);
+      }
+      if (4 * j + 4 <= count && a.vec_out) {
+        *reinterpret_cast<float4*>(a.mean + e0 + 4 * j) = make_float4(m[0], m[1], m[2], m[3]);
+        if (a.update != 0) {
+          const float4 x = *reinterpret_cast<const float4*>(a.xin + e0 + 4 * j);
+          const float g = a.update == 1 ? gam : 1.0f;      // update 2 subtracts the mean itself (1 * m is exact)
+          *reinterpret_cast<float4*>(a.xout + e0 + 4 * j) =
+              make_float4(__fsub_rn(x.x, __fmul_rn(g, m[0])), __fsub_rn(x.y, __fmul_rn(g, m[1])),
+                          __fsub_rn(x.z, __fmul_rn(g, m[2])), __fsub_rn(x.w, __fmul_rn(g, m[3])));
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (4 * j + q < count) {
+            a.mean[e0 + 4 * j + q] = m[q];
+            if (a.update == 1) a.xout[e0 + 4 * j + q] = __fsub_rn(a.xin[e0 + 4 * j + q], __fmul_rn(gam, m[q]));
+            if (a.update == 2) a.xout[e0 + 4 * j + q] = __fsub_rn(a.xin[e0 + 4 * j + q], m[q]);
+          }
+        }
+      }
+    }
+  }
+  if (kCompare || kSquare) {
+    sq = warp_sum(sq);
+    if ((threadIdx.x & 31) == 0 && sq != 0.0) atomicAdd(a.sum_sq, sq);
   }
   if (bad) latch_error(a.st, QGX_ERR_CORRUPT);
 }
@@ -836,7 +1011,7 @@ namespace qgx {
 
 // workspace slots of a context
 enum { WS_OFF64 = 0, WS_FLAGS = 1, WS_LUT = 2, WS_SLOT0 = 3 /* stream, bits, offsets, total: 3..6 and 7..10 */,
-       WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18, WS_SEGBITS = 19, WS_VALUES = 20 };
+       WS_NORMS = 12, WS_SYM = 13, WS_NORMS2 = 14, WS_OPVAL = 15, WS_MEAN = 16, WS_DLUT = 18, WS_SEGBITS = 19, WS_VALUES = 20, WS_SYMTMP = 21, WS_NORMSDEC = 22 };
 
 // Small vectors, second part: mean_i = (((0 + v_{0,i}) + v_{1,i}) + ...) / K in worker order (the same sequential
 // sum as in the fused decode pass), then the optional state update.
@@ -854,7 +1029,8 @@ __global__ void __launch_bounds__(256) k_sum_workers(const float* __restrict__ v
   }
 }
 
-qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct, const LevelTable& lt, int sym_mode);
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& args, const CodeTable& ct, const LevelTable& lt, int sym_mode,
+                                 bool walk_only = false);
 
 // ---- what a call derives from a quantizer configuration, kept between calls --------------------
 // Building the rounding table, the code table and the decoder table and copying the latter to the device costs
@@ -876,6 +1052,7 @@ struct TableCache {
   LaunchShape enc[3][3];                // [octets per thread 1, 2, 4][sub-block 32, 64, 128]
   LaunchShape enc_staged[3];            // [sub-block]
   LaunchShape dec[3][6];                // [sub-block][symbol mode]
+  LaunchShape dec_walk[3][6];           // the walk alone
 };
 
 // Lets a kernel use all the dynamic shared memory that the device allows, once per kernel and device.  (The
@@ -950,7 +1127,7 @@ static qgx_status cached_tables(qgx_ctx* c, const qgx_quant_cfg* cfg, const Cach
     for (size_t i = 0; i < h_lut.size(); ++i) {
       const uint16_t w = by_code[i & (((size_t)1 << ct.maxlen) - 1)];
       const uint32_t L = w >> 8, idx = w & 0xffu;
-      if (L == 0) { h_lut[i].val = std::numeric_limits<float>::quiet_NaN(); h_lut[i].len = 1u; continue; }   // no codeword starts like this
+      if (L == 0) { h_lut[i].val = std::numeric_limits<float>::quiet_NaN(); h_lut[i].len = 1u | (kBadSymbol << 8); continue; }   // no codeword starts like this
       if (idx == 0) { h_lut[i].val = 0.0f; h_lut[i].len = L; continue; }       // symbol byte 0
       const bool neg = (i >> L) & 1u;
       h_lut[i].val = neg ? -cfg->levels[idx] : cfg->levels[idx];
@@ -1168,9 +1345,47 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   da.values = nullptr;
   const bool fits = (size_t)K * d * sizeof(float) <= ((size_t)256 << 20);
   const bool small = total_sub * 2 < (size_t)c->num_sms * kDecThreads * 4;
-  if (K > 1 && fits && c->decode_split != QGX_SPLIT_NEVER && (small || c->decode_split == QGX_SPLIT_ALWAYS)) {
+  if (K > 1 && fits && c->decode_split != QGX_SPLIT_NEVER && c->decode_split != QGX_SPLIT_SYMBOLS && (small || c->decode_split == QGX_SPLIT_ALWAYS)) {
     da.values = (float*)ws_get(c, WS_VALUES, sizeof(float) * (size_t)K * d);
     if (!da.values) return QGX_ERR_CUDA;
+  }
+  // Large vectors: the walk alone with one worker per thread (twice the warps of the one-pass kernel, whose 64 running
+  // sums per thread fill the register file), every worker's symbol bytes kept, and the ordered sums from those.
+  da.norms_out = nullptr;
+  const bool in_place = (sym_mode & 3) == 3;             // compares with the kept symbols and overwrites them: one pass
+  const bool two_pass = K > 1 && !da.values && !in_place &&
+                        (c->decode_split == QGX_SPLIT_SYMBOLS || (c->decode_split == QGX_SPLIT_AUTO && !small && kTwoPassByDefault));
+  if (two_pass) {
+    if (!da.sym_out) da.sym_out = (uint8_t*)ws_get(c, WS_SYMTMP, (size_t)K * sym_ld);
+    da.norms_out = (float*)ws_get(c, WS_NORMSDEC, sizeof(float) * (size_t)K * nb);
+    if (!da.sym_out || !da.norms_out) return QGX_ERR_CUDA;
+    rc = launch_decode_average(c, da, ct, lt_kept, 0, true);
+    if (rc != QGX_OK) return rc;
+    MeanArgs ma;
+    ma.sym = da.sym_out; ma.sym_ld = sym_ld; ma.norms = da.norms_out; ma.sym_prev = da.sym_prev; ma.norms_prev = da.norms_prev;
+    ma.sum_sq = da.sum_sq; ma.K = K; ma.d = d; ma.bucket = bucket; ma.nb = nb; ma.mean = mean_out; ma.update = da.update;
+    ma.xin = da.xin; ma.xout = da.xout; ma.scalars = da.scalars; ma.vec_out = da.vec_out; ma.st = c->dstatus;
+    {
+      ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
+      const size_t rows = (total_sub + 31) / 32;
+      const size_t threads = rows * (size_t)(ct.G / 16) * 32;
+      const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>((threads + 255) / 256, (size_t)c->num_sms * 6));
+      const size_t smem = sizeof(float) * (256 * 32 + 256);
+#define QGX_LAUNCH_M(GG, SS) k_symbols_mean<GG, SS><<<grid, 256, smem, c->stream>>>(ma, lt, lt_kept)
+#define QGX_LAUNCH_MG(GG)                                  \
+  do {                                                     \
+    if (sym_mode & 2) QGX_LAUNCH_M(GG, 2);                 \
+    else if (sym_mode & 4) QGX_LAUNCH_M(GG, 4);            \
+    else QGX_LAUNCH_M(GG, 0);                              \
+  } while (0)
+      if (ct.G == 32) QGX_LAUNCH_MG(32);
+      else if (ct.G == 64) QGX_LAUNCH_MG(64);
+      else QGX_LAUNCH_MG(128);
+#undef QGX_LAUNCH_MG
+#undef QGX_LAUNCH_M
+    }
+    count_launch(c);
+    return cuda_status(cudaGetLastError());
   }
   rc = launch_decode_average(c, da, ct, lt_kept, sym_mode);
   if (rc != QGX_OK || !da.values) return rc;
@@ -1183,48 +1398,58 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   return cuda_status(cudaGetLastError());
 }
 
-template <int G, int SYM>
+template <int G, int SYM, bool VAL>
 static qgx_status launch_decode_gs(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt) {
   const size_t subs = da.nb * ((size_t)da.bucket / G);
-  const size_t total_sub = da.values ? ((subs + 31) & ~(size_t)31) * (size_t)da.K : subs;   // threads wanted
-  const size_t lut_bytes = sizeof(DecEntry) * ((size_t)2 << ct.maxlen) + DecodeSmem<G, SYM>::kBytes;   // table, then the rows
+  const size_t total_sub = (!VAL || da.values) ? ((subs + 31) & ~(size_t)31) * (size_t)da.K : subs;   // threads wanted
+  const size_t lut_bytes = (VAL ? sizeof(DecEntry) : sizeof(uint32_t)) * ((size_t)2 << ct.maxlen) + DecodeSmem<G, SYM, VAL>::kBytes;   // table, then the rows
   const size_t want = (total_sub + kDecThreads - 1) / kDecThreads;
   int per_sm = 1;
   {
     ScopedKernelTimer timer(c, QGX_KERNEL_DECODE);
-    allow_max_dynamic_smem(k_exchange_decode<G, SYM>, c->device);
-    LaunchShape& shape = table_cache(c)->dec[G == 32 ? 0 : (G == 64 ? 1 : 2)][SYM];
+    allow_max_dynamic_smem(k_exchange_decode<G, SYM, VAL>, c->device);
+    TableCache* tc = table_cache(c);
+    LaunchShape& shape = (VAL ? tc->dec : tc->dec_walk)[G == 32 ? 0 : (G == 64 ? 1 : 2)][SYM];
     if (shape.smem != lut_bytes + 1) {                       // occupancy asked once per shape, not per call
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, SYM>, kDecThreads, lut_bytes);
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exchange_decode<G, SYM, VAL>, kDecThreads, lut_bytes);
       shape.smem = lut_bytes + 1;
       shape.per_sm = per_sm < 1 ? 1 : per_sm;
     }
     per_sm = shape.per_sm;
     const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)c->num_sms * per_sm));
-    k_exchange_decode<G, SYM><<<grid, kDecThreads, lut_bytes, c->stream>>>(da, ct, lt);
+    k_exchange_decode<G, SYM, VAL><<<grid, kDecThreads, lut_bytes, c->stream>>>(da, ct, lt);
   }
   count_launch(c);
   return cuda_status(cudaGetLastError());
 }
 
-template <int G>
+template <int G, bool VAL>
 static qgx_status launch_decode_g(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt, int sym_mode) {
   switch (sym_mode) {
-    case 1: return launch_decode_gs<G, 1>(c, da, ct, lt);
-    case 2: return launch_decode_gs<G, 2>(c, da, ct, lt);
-    case 3: return launch_decode_gs<G, 3>(c, da, ct, lt);
-    case 4: return launch_decode_gs<G, 4>(c, da, ct, lt);
-    case 5: return launch_decode_gs<G, 5>(c, da, ct, lt);
-    default: return launch_decode_gs<G, 0>(c, da, ct, lt);
+    case 1: return launch_decode_gs<G, 1, VAL>(c, da, ct, lt);
+    case 2: return launch_decode_gs<G, 2, VAL>(c, da, ct, lt);
+    case 3: return launch_decode_gs<G, 3, VAL>(c, da, ct, lt);
+    case 4: return launch_decode_gs<G, 4, VAL>(c, da, ct, lt);
+    case 5: return launch_decode_gs<G, 5, VAL>(c, da, ct, lt);
+    default: return launch_decode_gs<G, 0, VAL>(c, da, ct, lt);
   }
 }
 
-qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt, int sym_mode) {
+qgx_status launch_decode_average(qgx_ctx* c, const DecodeArgs& da, const CodeTable& ct, const LevelTable& lt, int sym_mode,
+                                 bool walk_only) {
   if (!ct.has_header || da.bucket % ct.G != 0) return QGX_ERR_INVALID_ARG;
+  if (walk_only) {
+    switch (ct.G) {
+      case 32: return launch_decode_g<32, false>(c, da, ct, lt, sym_mode);
+      case 64: return launch_decode_g<64, false>(c, da, ct, lt, sym_mode);
+      case 128: return launch_decode_g<128, false>(c, da, ct, lt, sym_mode);
+      default: return QGX_ERR_INVALID_ARG;
+    }
+  }
   switch (ct.G) {
-    case 32: return launch_decode_g<32>(c, da, ct, lt, sym_mode);
-    case 64: return launch_decode_g<64>(c, da, ct, lt, sym_mode);
-    case 128: return launch_decode_g<128>(c, da, ct, lt, sym_mode);
+    case 32: return launch_decode_g<32, true>(c, da, ct, lt, sym_mode);
+    case 64: return launch_decode_g<64, true>(c, da, ct, lt, sym_mode);
+    case 128: return launch_decode_g<128, true>(c, da, ct, lt, sym_mode);
     default: return QGX_ERR_INVALID_ARG;
   }
 }
@@ -1333,7 +1558,7 @@ using namespace qgx;
 extern "C" {
 
 qgx_status qgx_set_decode_split(qgx_ctx* c, int mode) {
-  if (!c || mode < QGX_SPLIT_AUTO || mode > QGX_SPLIT_ALWAYS) return QGX_ERR_INVALID_ARG;
+  if (!c || mode < QGX_SPLIT_AUTO || mode > QGX_SPLIT_SYMBOLS) return QGX_ERR_INVALID_ARG;
   c->decode_split = mode;
   return QGX_OK;
 }

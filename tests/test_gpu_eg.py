@@ -10,12 +10,12 @@ from oracle import qgx_oracle as o
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=["one thread per sub-block", "one worker per thread"])
+@pytest.fixture(scope="module", params=["one thread per sub-block", "one worker per thread", "walk, then sums"])
 def q(request):
     """Every test runs with both ways of spreading the decode pass (small vectors would only see the second)."""
     import paper_2308_09187_b200 as qgx
     ctx = qgx.qgx_create(0)
-    qgx.qgx_set_decode_split(ctx, qgx.QGX_SPLIT_NEVER if request.param == "one thread per sub-block" else qgx.QGX_SPLIT_ALWAYS)
+    qgx.qgx_set_decode_split(ctx, {"one thread per sub-block": qgx.QGX_SPLIT_NEVER, "one worker per thread": qgx.QGX_SPLIT_ALWAYS}.get(request.param, qgx.QGX_SPLIT_SYMBOLS))
     yield qgx, ctx
     qgx.qgx_destroy(ctx)
 

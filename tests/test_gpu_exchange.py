@@ -10,13 +10,16 @@ from oracle import qgx_oracle as o
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=["one thread per sub-block", "one worker per thread", "staged encode"])
+@pytest.fixture(scope="module", params=["one thread per sub-block", "one worker per thread", "staged encode", "walk, then sums"])
 def q(request):
-    """Every test runs with both ways of spreading the decode pass (small vectors would only see the second) and
-    with the staged encode kernel (the shapes it does not take fall back to the bucket-in-registers kernel)."""
+    """Every test runs with the three ways of spreading the decode pass (one thread per sub-block over all workers;
+    one worker per thread with the values added by a second kernel; the walk alone with the sums formed from the
+    symbol bytes) and with the staged encode kernel (the shapes it does not take fall back to the
+    bucket-in-registers kernel)."""
     import paper_2308_09187_b200 as qgx
     ctx = qgx.qgx_create(0)
-    qgx.qgx_set_decode_split(ctx, qgx.QGX_SPLIT_ALWAYS if request.param == "one worker per thread" else qgx.QGX_SPLIT_NEVER)
+    split = {"one worker per thread": qgx.QGX_SPLIT_ALWAYS, "walk, then sums": qgx.QGX_SPLIT_SYMBOLS}
+    qgx.qgx_set_decode_split(ctx, split.get(request.param, qgx.QGX_SPLIT_NEVER))
     qgx.qgx_set_encode_path(ctx, qgx.QGX_ENCODE_STAGED if request.param == "staged encode" else qgx.QGX_ENCODE_REGISTERS)
     yield qgx, ctx
     qgx.qgx_destroy(ctx)
