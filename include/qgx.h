@@ -252,7 +252,10 @@ qgx_status qgx_exchange_segments(qgx_ctx *ctx, const float *v, int K, size_t d, 
  * sub-blocks are decoded one worker per thread, followed by a kernel that adds the workers' values in worker
  * order (same results, K times more threads, K * d floats of workspace, at most 256 MB); large vectors are decoded
  * by one thread per sub-block over all workers.  QGX_SPLIT_NEVER / QGX_SPLIT_ALWAYS force one way (ALWAYS still
- * falls back when the workspace would exceed 256 MB). */
+ * falls back when the workspace would exceed 256 MB).  QGX_SPLIT_SYMBOLS decodes in two passes: the walk alone, one
+ * worker per thread, writes every worker's symbol bytes (K * d bytes of workspace unless the exchange keeps its
+ * symbols anyway), and a second kernel forms the ordered sums, the squared differences and the state update from
+ * them -- same results; exchanges that compare with and overwrite the kept symbols in one go stay in one pass. */
 enum { QGX_SPLIT_AUTO = 0, QGX_SPLIT_NEVER = 1, QGX_SPLIT_ALWAYS = 2, QGX_SPLIT_SYMBOLS = 3 };
 qgx_status qgx_set_decode_split(qgx_ctx *ctx, int mode);
 /* Which kernel the encode pass of the fused calls uses (no counterpart in the paper; the streams are the same bit
