@@ -277,8 +277,8 @@ def run_ours(args):
 
 
 def other_configs(qgx, ctx):
-    """The smaller configurations, timed by the wall clock around a synchronize (they are launch- and
-    latency-bound): supplementary figures, not the headline."""
+    """The smaller configurations, timed on the device with CUDA events around the calls (the context's stream is
+    torch's current stream); they are launch- and latency-bound: supplementary figures, not the headline."""
     import numpy as np
     import torch
     import qgx_inputs as gen
@@ -287,11 +287,13 @@ def other_configs(qgx, ctx):
         for _ in range(warm):
             fn()
         torch.cuda.synchronize()
-        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         for _ in range(n):
             fn()
+        e1.record()
         torch.cuda.synchronize()
-        return (time.perf_counter() - t0) / n
+        return e0.elapsed_time(e1) * 1e-3 / n
 
     out = {}
     g = gen.c1_bilinear(T=100, device="cuda")
