@@ -13,6 +13,39 @@ qgx_status refit_from_source(qgx_ctx* c, DualSource src, int K, size_t d, qgx_qu
                              double* hist_host);
 enum { WS_OPVAL = 15, WS_MEAN = 16, WS_HIST = 17 };
 
+// sum_j m[j] x[j] of one row by one warp: fp64 accumulation, four partial sums per lane, the lanes' sums added by
+// shuffles; every lane returns the total
+__device__ __forceinline__ double gemv_row(const float* __restrict__ m, size_t ncols, const float* __restrict__ x, int lane, bool vec_ok) {
+  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+  if (vec_ok) {
+    // four loads of the row in flight, added in index order
+    constexpr int kAhead = 4;
+    for (size_t j0 = (size_t)lane * 4; j0 < ncols; j0 += 128 * kAhead) {
+      float4 mv[kAhead], xv[kAhead];
+#pragma unroll
+      for (int u = 0; u < kAhead; ++u) {
+        const size_t j = j0 + 128 * (size_t)u;
+        if (j < ncols) {
+          mv[u] = __ldcs(reinterpret_cast<const float4*>(m + j));
+          xv[u] = __ldg(reinterpret_cast<const float4*>(x + j));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kAhead; ++u) {
+        if (j0 + 128 * (size_t)u < ncols) {
+          a0 = fma((double)mv[u].x, (double)xv[u].x, a0);
+          a1 = fma((double)mv[u].y, (double)xv[u].y, a1);
+          a2 = fma((double)mv[u].z, (double)xv[u].z, a2);
+          a3 = fma((double)mv[u].w, (double)xv[u].w, a3);
+        }
+      }
+    }
+  } else {
+    for (size_t j = lane; j < ncols; j += 32) a0 = fma((double)m[j], (double)x[j], a0);
+  }
+  return warp_sum((a0 + a1) + (a2 + a3));
+}
+
 // out[row] = sign * (sum_j mat[row][j] x[j] + bias[row]); one warp per row, fp64 accumulation,
 // one rounding to fp32
 __global__ void __launch_bounds__(256) k_gemv_rows(const float* __restrict__ mat, size_t nrows, size_t ncols,
@@ -22,38 +55,46 @@ __global__ void __launch_bounds__(256) k_gemv_rows(const float* __restrict__ mat
   const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const size_t nwarps = ((size_t)gridDim.x * blockDim.x) >> 5;
   for (size_t row = warp; row < nrows; row += nwarps) {
-    const float* m = mat + row * ncols;
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-    if (vec_ok) {
-      for (size_t j = (size_t)lane * 4; j < ncols; j += 128) {
-        const float4 mv = __ldcs(reinterpret_cast<const float4*>(m + j));
-        const float4 xv = __ldg(reinterpret_cast<const float4*>(x + j));
-        a0 = fma((double)mv.x, (double)xv.x, a0);
-        a1 = fma((double)mv.y, (double)xv.y, a1);
-        a2 = fma((double)mv.z, (double)xv.z, a2);
-        a3 = fma((double)mv.w, (double)xv.w, a3);
-      }
-    } else {
-      for (size_t j = lane; j < ncols; j += 32) a0 = fma((double)m[j], (double)x[j], a0);
-    }
-    double s = warp_sum((a0 + a1) + (a2 + a3));
-    if (lane == 0) {
-      if (bias) s += (double)bias[row];
-      out[row] = (float)s;
-    }
+    const double s = gemv_row(mat + row * ncols, ncols, x, lane, vec_ok);
+    if (lane == 0) out[row] = (float)(bias ? s + (double)bias[row] : s);
   }
 }
 
-// out[col] = -(sum_i mat[i][col] x[i]): a 32 x 32 thread tile, rows strided over the 32 row
-// lanes, partial sums combined in row-lane order
-__global__ void __launch_bounds__(1024) k_gemv_cols_neg(const float* __restrict__ mat, size_t n, const float* __restrict__ x,
-                                                        float* __restrict__ out) {
+// The bilinear operator in one launch, z = (x, y): out = (M y, -M^T x).  Blocks of 32 x 32 threads; the first
+// ceil(n / 32) blocks take 32 columns each (out[n + col] = -(sum_i mat[i][col] x[i]): rows strided over the 32 row
+// lanes, partial sums combined in row-lane order), the others 32 rows each (one warp per row, as k_gemv_rows).
+__global__ void __launch_bounds__(1024) k_bilinear(const float* __restrict__ mat, size_t n, const float* __restrict__ z,
+                                                   float* __restrict__ out_all, bool vec_ok) {
   __shared__ double s_part[32][33];
   const int cx = threadIdx.x, ry = threadIdx.y;
+  const size_t col_blocks = (n + 31) / 32;
+  if (blockIdx.x >= col_blocks) {
+    const size_t row = ((size_t)blockIdx.x - col_blocks) * 32 + (size_t)ry;
+    if (row < n) {
+      const double s = gemv_row(mat + row * n, n, z + n, cx, vec_ok);
+      if (cx == 0) out_all[row] = (float)s;
+    }
+    return;
+  }
+  const float* x = z;
+  float* out = out_all + n;
   const size_t col = (size_t)blockIdx.x * 32 + cx;
   double acc = 0.0;
-  if (col < n)
-    for (size_t i = ry; i < n; i += 32) acc = fma((double)mat[i * n + col], (double)x[i], acc);
+  if (col < n) {
+    // eight loads of the column in flight, added in index order
+    constexpr int kAhead = 8;
+    for (size_t i0 = ry; i0 < n; i0 += 32 * kAhead) {
+      float mv[kAhead], xv[kAhead];
+#pragma unroll
+      for (int u = 0; u < kAhead; ++u) {
+        const size_t i = i0 + 32 * (size_t)u;
+        if (i < n) { mv[u] = mat[i * n + col]; xv[u] = x[i]; }
+      }
+#pragma unroll
+      for (int u = 0; u < kAhead; ++u)
+        if (i0 + 32 * (size_t)u < n) acc = fma((double)mv[u], (double)xv[u], acc);
+    }
+  }
   s_part[ry][cx] = acc;
   __syncthreads();
   if (ry == 0 && col < n) {
@@ -116,9 +157,8 @@ qgx_status apply_operator_impl(qgx_ctx* c, const qgx_operator* op, const float* 
     if (d % 2) return QGX_ERR_INVALID_ARG;
     const size_t n = d / 2;
     const bool vec_ok = (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(op->mat) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(x + n) & 15u) == 0);
-    k_gemv_rows<<<grid_for(c, n * 32, 256), 256, 0, c->stream>>>(op->mat, n, n, x + n, nullptr, out, vec_ok);
-    k_gemv_cols_neg<<<(unsigned)((n + 31) / 32), dim3(32, 32), 0, c->stream>>>(op->mat, n, x, out + n);
-    count_launch(c, 2);
+    k_bilinear<<<(unsigned)(2 * ((n + 31) / 32)), dim3(32, 32), 0, c->stream>>>(op->mat, n, x, out, vec_ok);
+    count_launch(c);
   } else if (op->kind == QGX_OP_DIAGONAL) {
     k_diag<<<grid_for(c, d, 256), 256, 0, c->stream>>>(op->mat, x, out, d);
     count_launch(c);
