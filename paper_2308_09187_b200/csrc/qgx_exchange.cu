@@ -82,6 +82,7 @@ struct EncodeArgs {
   float* norms;                 // [K][nb] (kept for the caller; the streams carry them too)
   unsigned long long* status;   // [K][nb], zeroed before the launch
   unsigned int* ticket;         // zeroed before the launch
+  const struct EncodeTables* tables;   // the shared-memory tables of the configuration, built once (null: every CTA builds them)
   DevStatus* st;
   size_t nb_whole;              // buckets [0, nb_whole) of every worker belong to k_encode_staged ...
   size_t b_first;               // ... and buckets [b_first, nb) to k_exchange_encode
@@ -229,6 +230,30 @@ __device__ __forceinline__ uint32_t pair_entry(uint32_t pair, float z_first, flo
   return lds_table32(pair + (__float_as_uint(t) & 0x3ffcu));
 }
 
+// The encoder's shared-memory tables as one block of global memory: built by one CTA when a configuration is first
+// used and copied by every encode CTA after that (building them costs a CTA of a small bucket more than the bucket).
+struct EncodeTables {
+  float4 bin[kBinEntries];
+  uint32_t pair[kPairLutSize];
+  EncLut lut;
+};
+static_assert(sizeof(EncodeTables) % 16 == 0, "copied in 16-byte pieces");
+
+__global__ void __launch_bounds__(512) k_build_encode_tables(const __grid_constant__ RoundTable rt, const __grid_constant__ CodeTable ct,
+                                                             EncodeTables* out) {
+  __shared__ __align__(128) float4 s_bin[kBinEntries];
+  __shared__ __align__(16) uint32_t s_pair[kPairLutSize];
+  __shared__ EncLut s_lut;
+  fill_enc_lut(&s_lut, ct);
+  fill_bin_table(s_bin, rt, true);
+  __syncthreads();
+  fill_pair_lut_signed(s_pair, &s_lut);
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBinEntries; i += blockDim.x) out->bin[i] = s_bin[i];
+  for (int i = threadIdx.x; i < kPairLutSize; i += blockDim.x) out->pair[i] = s_pair[i];
+  for (int i = threadIdx.x; i < 2 * QGX_MAX_LEVELS; i += blockDim.x) out->lut.e[i] = s_lut.e[i];
+}
+
 // One persistent CTA per SM slot; each ticket is one bucket (k = ticket % K, b = ticket / K).
 //   loads, zero the image | barrier | norm, Philox, rounding, packing, sub-block lengths, warp scans |
 //   barrier | warp offsets, bit scatter, look-back (warp 0) | barrier | copy out
@@ -242,7 +267,7 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ __align__(128) float4 s_bin[kBinEntries];
   __shared__ EncLut s_lut;
-  __shared__ uint32_t s_pair[kPairLutSize];
+  __shared__ __align__(16) uint32_t s_pair[kPairLutSize];
   __shared__ float s_lev[QGX_MAX_LEVELS];
   __shared__ double s_red[2][32];
   __shared__ uint32_t s_wtot[2][32];
@@ -258,13 +283,23 @@ k_exchange_encode(const __grid_constant__ EncodeArgs a, const __grid_constant__ 
   constexpr int kSegLanes = G / kOctet;                 // lanes per sub-block within a row of 256 coordinates
   constexpr int kSegs = 32 / kSegLanes;                 // sub-blocks per row
 
-  fill_enc_lut(&s_lut, ct);
-  fill_bin_table(s_bin, rt, true);
+  if (a.tables) {
+    const uint4* gb = reinterpret_cast<const uint4*>(a.tables->bin);
+    const uint4* gp = reinterpret_cast<const uint4*>(a.tables->pair);
+    uint4* sb = reinterpret_cast<uint4*>(s_bin);
+    uint4* sp = reinterpret_cast<uint4*>(s_pair);
+    for (int i = threadIdx.x; i < kBinEntries; i += blockDim.x) sb[i] = __ldg(gb + i);
+    for (int i = threadIdx.x; i < kPairLutSize / 4; i += blockDim.x) sp[i] = __ldg(gp + i);
+    for (int i = threadIdx.x; i < 2 * QGX_MAX_LEVELS; i += blockDim.x) s_lut.e[i] = __ldg(a.tables->lut.e + i);
+  } else {
+    fill_enc_lut(&s_lut, ct);
+    fill_bin_table(s_bin, rt, true);
+  }
   if (threadIdx.x < QGX_MAX_LEVELS) s_lev[threadIdx.x] = threadIdx.x < lt.nlev ? lt.lev[threadIdx.x] : 1.0f;
   if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
   for (int i = threadIdx.x; i < 2 * img_words; i += blockDim.x) s_dyn[i] = 0;
   __syncthreads();
-  fill_pair_lut_signed(s_pair, &s_lut);
+  if (!a.tables) fill_pair_lut_signed(s_pair, &s_lut);
   __syncthreads();
   const int nlev = lt.nlev;
   const uint32_t pair_sa = smem_addr(s_pair);
@@ -1044,6 +1079,7 @@ struct CachedTables {
   CodeTable ct;
   RoundTable rt;
   DecEntry* lut_dev;                    // 2 * kDecLutMax entries, owned
+  EncodeTables* enc_dev;                // owned; built by k_build_encode_tables
 };
 constexpr int kTableCacheSlots = 32;
 struct LaunchShape { size_t smem; int per_sm; };      // smem == 0: not asked yet
@@ -1081,8 +1117,10 @@ static void allow_max_dynamic_smem(Kernel kernel, int device) {
 void free_table_cache(qgx_ctx* c) {
   TableCache* tc = (TableCache*)c->table_cache;
   if (!tc) return;
-  for (int i = 0; i < kTableCacheSlots; ++i)
+  for (int i = 0; i < kTableCacheSlots; ++i) {
     if (tc->e[i].lut_dev) cudaFree(tc->e[i].lut_dev);
+    if (tc->e[i].enc_dev) cudaFree(tc->e[i].enc_dev);
+  }
   delete tc;
   c->table_cache = nullptr;
 }
@@ -1137,6 +1175,14 @@ static qgx_status cached_tables(qgx_ctx* c, const qgx_quant_cfg* cfg, const Cach
     // the call returns once it has been staged
     if (cudaMemcpyAsync(e->lut_dev, h_lut.data(), h_lut.size() * sizeof(DecEntry), cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
       return QGX_ERR_CUDA;
+    // the encoder's tables, built on the device by the routines that the kernels would run themselves
+    if (!e->enc_dev && cudaMalloc((void**)&e->enc_dev, sizeof(EncodeTables)) != cudaSuccess) {
+      cudaGetLastError();
+      e->enc_dev = nullptr;
+      return QGX_ERR_CUDA;
+    }
+    k_build_encode_tables<<<1, 512, 0, c->stream>>>(e->rt, e->ct, e->enc_dev);
+    if (cudaGetLastError() != cudaSuccess) return QGX_ERR_CUDA;
     e->nlev = cfg->nlev;
     e->bucket = cfg->bucket;
     std::memcpy(e->levels, cfg->levels, sizeof(e->levels));
@@ -1218,7 +1264,7 @@ qgx_status exchange_impl(qgx_ctx* c, DualSource src, int K, size_t d, const qgx_
   ea.src = src; ea.d = d; ea.bucket = bucket; ea.K = K; ea.nb = nb; ea.norm_type = cfg->norm_type; ea.xid = xid; ea.quad_base = coord_base / kQuad;
   ea.vec_ok = (d % kQuad == 0) && (src.ld % kQuad == 0) && ((reinterpret_cast<uintptr_t>(src.v) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(src.a) & 15u) == 0);
   ea.stream = stream; ea.cap_words = cap; ea.bucket_bits = bbits; ea.offsets = offs; ea.total_bits = tot; ea.norms = norms;
-  ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(tot + K); ea.st = c->dstatus;
+  ea.status = status; ea.ticket = reinterpret_cast<unsigned int*>(tot + K); ea.st = c->dstatus; ea.tables = tables->enc_dev;
   uint8_t* sym_out = nullptr;
   const uint8_t* sym_prev = nullptr;
   const size_t sym_ld = ((nb * (size_t)(bucket / ct.G) + 31) / 32) * 32 * (size_t)ct.G;   // see DecodeArgs::sym_out
