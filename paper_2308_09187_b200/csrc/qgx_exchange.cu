@@ -1182,6 +1182,7 @@ static qgx_status cached_tables(qgx_ctx* c, const qgx_quant_cfg* cfg, const Cach
       return QGX_ERR_CUDA;
     }
     k_build_encode_tables<<<1, 512, 0, c->stream>>>(e->rt, e->ct, e->enc_dev);
+    count_launch(c);
     if (cudaGetLastError() != cudaSuccess) return QGX_ERR_CUDA;
     e->nlev = cfg->nlev;
     e->bucket = cfg->bucket;
